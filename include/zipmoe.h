@@ -1,0 +1,180 @@
+/*
+ * zipmoe.h -- C ABI of the B200-native ZipMoE decode library.
+ *
+ * The library implements the compute-centric step of ZipMoE: expert weights
+ * are kept losslessly compressed and the required bf16 tensors are computed
+ * on demand instead of being transferred (paper Section 1, last paragraph).
+ * Offline, each bf16 tensor is split into an exponent stream and a
+ * sign+mantissa byte stream; the exponent stream is cut into K shards that
+ * are entropy-coded independently ("E-chunks") while the sign+mantissa bytes
+ * are stored raw ("SM-chunks") (Section 3.1, "Offline Initialization").
+ * Online, E-chunks are decompressed and re-assembled with the SM-chunks into
+ * exact bf16 (Section 3.1, "Real-time Inference"; Section 3.3,
+ * "Memory-Coalesced Tensor Recovery Kernel").  The paper runs the
+ * decompression on CPU threads with LZ4/ZSTD and leaves the compressor slot
+ * open (Section 6, "Other Compressors"); here the slot holds an order-0
+ * canonical Huffman code over exponent bytes and both steps run in one CUDA
+ * kernel for sm_100a.
+ *
+ * Conventions for every entry point
+ *   - Plain C, no exceptions, no aborts: the return value is a zipmoe_status.
+ *   - The library never allocates or frees device memory and never
+ *     synchronises a stream, except where an entry point says otherwise.
+ *     Device buffers and streams belong to the caller.
+ *   - "host" / "device" in an argument's comment says where the pointer must
+ *     point.  Sizes are in the unit named in the comment.
+ *   - The container ("blob") produced by zipmoe_encode is self-describing,
+ *     little-endian, and documented in the repository's design notes; its
+ *     payload and sign+mantissa sections are copied verbatim to the device.
+ */
+#ifndef ZIPMOE_H
+#define ZIPMOE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int zipmoe_status;
+#define ZIPMOE_OK 0
+#define ZIPMOE_ERR_INVALID_ARG (-1)      /* null pointer, bad size, bad alignment, bad option  */
+#define ZIPMOE_ERR_BAD_FORMAT (-2)       /* blob fails validation                               */
+#define ZIPMOE_ERR_BUFFER_TOO_SMALL (-3) /* caller's output buffer can not hold the result      */
+#define ZIPMOE_ERR_CUDA (-4)             /* a CUDA runtime call failed (launch, attribute, ...) */
+#define ZIPMOE_ERR_DECODE_CORRUPT (-5)   /* reported through the device status word only        */
+#define ZIPMOE_ERR_UNSUPPORTED (-6)      /* shape or option outside what the kernels handle     */
+
+#define ZIPMOE_LAYOUT_LINEAR 0u  /* a tile is tile_elems consecutive elements of the flat tensor  */
+#define ZIPMOE_LAYOUT_BLOCKED 1u /* a tile is a 16 x 256 block of the rows x cols matrix         */
+#define ZIPMOE_MAX_CODE_LEN 12u
+#define ZIPMOE_TILE_ELEMS_MAX 4096u
+/* bytes the caller must keep readable after the end of the device payload and
+ * sign+mantissa buffers (the kernels read whole 16-byte units and look a few
+ * words past the last code) */
+#define ZIPMOE_DEVICE_PAD_BYTES 256u
+
+typedef struct CUstream_st *zipmoe_stream; /* a cudaStream_t; NULL is the default stream */
+
+/* ---- encoding (host) ---------------------------------------------------- */
+
+typedef struct {
+  uint32_t chunk_elems;  /* elements per independently decodable chunk (the paper's shard): a multiple
+                            of 256, and a multiple of 4096 when larger than 4096.  0 selects 65536.    */
+  uint32_t max_code_len; /* longest Huffman code, 8..12.  0 selects 12.                                 */
+  uint32_t layout;       /* ZIPMOE_LAYOUT_LINEAR or ZIPMOE_LAYOUT_BLOCKED (needs rows % 16 == 0,
+                            cols % 256 == 0, chunk_elems >= 4096)                                       */
+  uint32_t n_threads;    /* host threads for the encoder (chunks are independent). 0 selects 1.         */
+} zipmoe_encode_opts;
+
+typedef struct {
+  uint64_t n_elems;       /* rows * cols                                                         */
+  uint32_t rows, cols;
+  uint32_t layout, chunk_elems, tile_elems, max_code_len;
+  uint32_t n_chunks;      /* K = ceil(n_tiles / (chunk_elems / tile_elems))                      */
+  uint32_t n_tiles;
+  uint64_t table_off;     /* byte offset in the blob of the 256 code lengths                     */
+  uint64_t chunk_off_off; /* byte offset of the n_chunks + 1 per-chunk bit offsets (u64)         */
+  uint64_t payload_off;   /* byte offset and size of the E-chunk section (16-byte aligned)       */
+  uint64_t payload_bytes;
+  uint64_t sm_off;        /* byte offset and size of the SM-chunk section (16-byte aligned)      */
+  uint64_t sm_bytes;
+  uint64_t total_bytes;
+} zipmoe_blob_info;
+
+/* Upper bound on the blob size for a rows x cols tensor.  (Section 3.1: the
+ * serialised form of one tensor: E-chunks, SM-chunks and metadata.)
+ * host in: opts (NULL = defaults); host out: *blob_bytes_max. */
+zipmoe_status zipmoe_encode_bound(uint64_t rows, uint64_t cols, const zipmoe_encode_opts *opts,
+                                  uint64_t *blob_bytes_max);
+
+/* Offline initialisation of one tensor (Section 3.1, "Offline Initialization"):
+ * bit-field decomposition of each bf16 into exponent byte and sign+mantissa
+ * byte, one canonical Huffman code per tensor over the exponent bytes, the
+ * exponent stream cut into chunks of chunk_elems elements with per-chunk bit
+ * offsets, sign+mantissa bytes stored raw.  Synchronous, host only, no CUDA.
+ * host in : bf16 (rows*cols bit patterns, row-major), opts (NULL = defaults)
+ * host out: blob[0 .. *blob_bytes), written only if blob_cap is large enough
+ *           (ZIPMOE_ERR_BUFFER_TOO_SMALL otherwise; *blob_bytes is then the bound). */
+zipmoe_status zipmoe_encode(const uint16_t *bf16, uint64_t rows, uint64_t cols, const zipmoe_encode_opts *opts,
+                            void *blob, uint64_t blob_cap, uint64_t *blob_bytes);
+
+/* Parse the header of a blob.  host in: blob; host out: *info. */
+zipmoe_status zipmoe_blob_info_get(const void *blob, uint64_t blob_bytes, zipmoe_blob_info *info);
+
+/* Full structural check of a blob on the host: header, complete prefix code
+ * (Kraft sum exactly 1, lengths <= max_code_len), monotone 128-bit-aligned
+ * chunk offsets, tile tables and per-lane bit counts inside their records.
+ * A blob that passes can be handed to the device decoder safely. */
+zipmoe_status zipmoe_blob_validate(const void *blob, uint64_t blob_bytes);
+
+/* ---- decode (device) ---------------------------------------------------- */
+
+/* One descriptor per chunk of a launch.  A "run" is the consecutive
+ * descriptors of one tensor (same table, consecutive chunks). */
+typedef struct {
+  uint64_t payload_off;     /* bytes from `payload` to this chunk's E-chunk (multiple of 16): its
+                               per-chunk bit offset / 8 plus where the blob's payload section sits */
+  uint64_t sm_off;          /* bytes from `sm` to the SM bytes of this chunk's first tile (mult. of 16) */
+  uint64_t out_off;         /* elements from `out_bf16` to the tensor's element 0 (multiple of 8)  */
+  uint32_t row_pitch;       /* elements between the 256-element rows of a tile: cols (blocked), 256 (linear) */
+  uint32_t tiles_per_rowblk;/* cols / 256 (blocked), 1 (linear)                                    */
+  uint32_t tile0;           /* index within the tensor of this chunk's first tile                 */
+  uint32_t n_tiles;         /* tiles in this chunk                                                 */
+  uint32_t tile_elems;      /* 256 * I, I = 1..16                                                  */
+  uint32_t last_tile_elems; /* existing elements in this chunk's last tile (1..tile_elems)         */
+  uint32_t table_id;        /* index into `tables`                                                 */
+  uint32_t tile_prefix;     /* tiles in all earlier descriptors of the launch                      */
+  uint32_t run_first_chunk; /* index in `chunks` of the run's first descriptor                     */
+  uint32_t run_first_tile;  /* tile_prefix of that descriptor                                      */
+  uint32_t run_end_tile;    /* tile_prefix + n_tiles of the run's last descriptor                  */
+  uint32_t tiles_per_chunk; /* tiles in every chunk of the run but possibly the last               */
+} zipmoe_chunk_desc;
+
+typedef struct {
+  uint8_t code_len[256];    /* canonical Huffman code lengths, 0 = unused symbol */
+} zipmoe_table;
+
+/* Fill the descriptors and the table for one blob whose payload section will
+ * sit at payload_base bytes into the device payload buffer, whose SM section
+ * at sm_base bytes into the device SM buffer, and whose tensor at out_base
+ * elements into the output (all three multiples of 16 bytes).  chunk_base and
+ * tile_base are the number of descriptors and tiles already planned for this
+ * launch.  Host only.
+ * host in : blob;  host out: descs[0 .. info.n_chunks), *table. */
+zipmoe_status zipmoe_blob_plan(const void *blob, uint64_t blob_bytes, uint64_t payload_base, uint64_t sm_base,
+                               uint64_t out_base, uint32_t table_id, uint32_t chunk_base, uint32_t tile_base,
+                               zipmoe_chunk_desc *descs, zipmoe_table *table);
+
+/* Real-time reconstruction (Section 3.1 "Real-time Inference", steps 6-7;
+ * Section 3.3 "Memory-Coalesced Tensor Recovery Kernel"): decode every
+ * chunk's exponent bytes from its E-chunk and merge them with the SM bytes
+ * into bf16, written once, in place, to out_bf16.  Chunks are independent and
+ * may belong to any number of tensors.  One kernel launch on `stream`;
+ * asynchronous; the exponent bytes never reach global memory.
+ *
+ * device in : chunks[n_chunks] (in launch order, tile_prefix ascending),
+ *             tables[n_tables], payload[payload_bytes + PAD], sm[sm_bytes + PAD]
+ * device out: out_bf16[out_elems]; status_word (nullable): left untouched on
+ *             success, set to a non-zero code when a descriptor, offset or
+ *             bit count points outside the given buffers or a wait ran out;
+ *             the kernel skips the offending tile and always terminates.
+ * n_tiles   : total tiles of the launch (sum of chunks[].n_tiles).
+ * All device pointers 16-byte aligned.  Errors found on the host (null or
+ * misaligned pointers, zero table count with non-zero chunks) are returned
+ * before anything is launched. */
+zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t n_chunks, uint32_t n_tiles,
+                            const zipmoe_table *tables, uint32_t n_tables, const uint8_t *payload,
+                            uint64_t payload_bytes, const uint8_t *sm, uint64_t sm_bytes, uint16_t *out_bf16,
+                            uint64_t out_elems, uint32_t *status_word, zipmoe_stream stream);
+
+/* Name of a status code (static string). */
+const char *zipmoe_status_string(zipmoe_status s);
+
+/* Library version, for the binding's sanity check. */
+uint32_t zipmoe_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZIPMOE_H */
