@@ -1,0 +1,312 @@
+#!/usr/bin/env python
+"""Benchmark of the ZipMoE decode hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" is one pass of the decode path over one MoE layer of compressed
+expert weights: a single zipmoe_decode launch that decompresses every E-chunk
+and re-assembles every bf16 tensor of the layer.  Prints ONE JSON line.
+
+* value      : decoded bf16 GB/s, whole job, compressed inputs resident in HBM.
+* e2e        : the same through the C ABI with HOST buffers: compressed streams
+               copied host->device from pinned memory, decode, decoded tensors
+               copied device->host, all inside the timed region.
+* roofline   : algorithmic bytes of one launch (E-chunk section + sign/mantissa
+               bytes read + bf16 written) / mean launch duration, against the
+               measured HBM copy bandwidth of this machine's B200s.
+* cpu_baseline: the CPU oracle (test infrastructure; plain C, bit-by-bit
+               decoder), one thread per host core over whole tensors, on a
+               bounded sample of the same workload.
+* --impl reference: the oracle alone, timed on the host cores.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "decoded bf16 GB/s (lossless decode of compressed MoE expert weights), 1 B200, bit-exact"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+def build_workload(name, keep_originals):
+    from paper_2601_21198_b200 import workloads
+    if name == "small_layer":
+        return workloads.small_layer(keep_originals=keep_originals)
+    if name == "large_layer":
+        return workloads.large_layer(keep_originals=keep_originals)
+    if name == "single_matrix":
+        return workloads.single_matrix(keep_originals=keep_originals)
+    raise SystemExit("unknown workload %s" % name)
+
+
+# ----------------------------------------------------------------------------- CPU oracle leg
+def oracle_seconds_per_tensor(blob):
+    from oracle import codec
+    codec.lib()
+    t0 = time.perf_counter()
+    codec.decode(blob)
+    return max(time.perf_counter() - t0, 1e-4)
+
+
+def oracle_decode_rate(blobs, n_threads, count):
+    """Decodes `count` whole tensors (cycling through blobs) with the CPU oracle on
+    n_threads threads (ctypes releases the GIL).  Returns (decoded bf16 GB/s, seconds)."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import codec
+    sample = [blobs[i % len(blobs)] for i in range(count)]
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(min(n_threads, count)) as pool:
+        sizes = list(pool.map(lambda b: codec.decode(b).size, sample))
+    dt = time.perf_counter() - t0
+    return 2.0 * sum(sizes) / dt / 1e9, dt
+
+
+def run_reference(args):
+    """The oracle as it stands, on the host cores; rank 0 only.  Each step decodes a
+    bounded sample of the layer, sized so that the whole run stays near two minutes."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from paper_2601_21198_b200 import workloads
+    cores = os.cpu_count() or 1
+    w = workloads.small_layer(n_experts=max(1, min(64, (cores + 2) // 3)), keep_originals=False)
+    per = oracle_seconds_per_tensor(w.blobs[0])
+    wall_per_step = 120.0 / max(1, args.steps + args.warmup)
+    count = int(max(1, min(4 * len(w.blobs), wall_per_step * cores / per)))
+    threads = min(cores, count)
+    for _ in range(args.warmup):
+        oracle_decode_rate(w.blobs, threads, count)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_decode_rate(w.blobs, threads, count)
+    dt_all = time.perf_counter() - t0
+    value = args.steps * count * 2.0 * 2048 * 1408 / dt_all / 1e9
+    sample = "%d tensors (2048x1408 bf16 each, 64K-element chunks) of the 64-expert layer per step" % count
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt_all / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u16", "data": "synthetic",
+        "config": {"workload": "moe64_2048x1408_chunk64K (bounded sample)", "chunk_elems": 65536},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler(threading.Thread):
+    """Samples SM clock, power and clock-event reasons through NVML (read-only)."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index, period=0.004):
+        super().__init__(daemon=True)
+        self.period, self.samples, self.stop_flag, self.ok = period, [], False, False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.max_mhz = None
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.samples.append((time.perf_counter(), mhz, reasons))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def summary(self, t0, t1):
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        window = "timed"
+        if not inside:
+            inside, window = self.samples, "warmup+timed"
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "window": "none"}
+        bits = 0
+        for s in inside:
+            bits |= s[2]
+        reasons = sorted(name for bit, name in self.REASONS.items() if bits & bit)
+        return {"sm_mhz": float(np.median([s[1] for s in inside])), "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(inside), "window": window}
+
+
+# ----------------------------------------------------------------------------- GPU leg
+def run_ours(args):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+
+    from paper_2601_21198_b200 import binding, build
+    build.build()
+    w = build_workload(args.workload, keep_originals=False)
+    plan = w.plan
+    dplan = plan.to_device(dev)
+    out = dplan.new_output()
+    stream = torch.cuda.current_stream(dev)
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    # correctness before timing: status word clean and one tensor equal to what the encoder was given
+    dplan.decode(out)
+    torch.cuda.synchronize(dev)
+    verified = int(dplan.status.item()) == 0
+    from paper_2601_21198_b200 import inputs
+    probe = inputs.small_expert_tensor(0, 0) if args.workload == "small_layer" else None
+    if probe is not None:
+        ref = torch.from_numpy(probe.view(np.int16).ravel()).to(dev)
+        verified = verified and bool(torch.equal(plan.tensor_slice(out, 0), ref))
+        del ref
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for _ in range(args.warmup):
+        dplan.decode(out)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(args.steps):
+        dplan.decode(out)
+    e1.record(stream)
+    barrier()
+    t1 = time.perf_counter()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.summary(t0, t1)
+    verified = verified and int(dplan.status.item()) == 0
+
+    # end to end: pinned host -> device, decode, device -> pinned host, every step
+    h_pay = torch.from_numpy(plan.payload).pin_memory()
+    h_sm = torch.from_numpy(plan.sm).pin_memory()
+    h_desc = torch.from_numpy(plan.descs.view(np.uint8).copy()).pin_memory()
+    h_tab = torch.from_numpy(plan.tables).pin_memory()
+    h_out = torch.empty(plan.out_elems, dtype=torch.int16).pin_memory()
+    e2e_steps = max(1, min(args.steps, 10))
+
+    def e2e_step():
+        dplan.payload.copy_(h_pay, non_blocking=True)
+        dplan.sm.copy_(h_sm, non_blocking=True)
+        dplan.descs.copy_(h_desc, non_blocking=True)
+        dplan.tables.copy_(h_tab, non_blocking=True)
+        dplan.decode(out)
+        h_out.copy_(out, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    f1.record(stream)
+    barrier()
+    e2e_ms = f0.elapsed_time(f1)
+    sampler.stop_flag = True
+
+    times = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = (float(v) for v in times.cpu())
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        bf16_bytes = w.bf16_bytes()
+        per_launch_s = ms / 1e3 / args.steps
+        alg = plan.algorithmic_bytes()
+        achieved = alg / per_launch_s / 1e9
+        line = {
+            "metric": METRIC, "value": world * bf16_bytes / per_launch_s / 1e9, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_launch_s * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u16", "data": "synthetic",
+            "config": {"workload": w.label, "tensors": len(w.blobs), "elements": w.n_elems,
+                       "chunk_elems": int(plan.infos[0].chunk_elems), "chunks": plan.n_chunks, "tiles": plan.n_tiles,
+                       "compressed_over_bf16": w.compressed_bytes() / bf16_bytes,
+                       "l2": "inputs and outputs of one step (%.2f GB) exceed L2; no flush" % (alg / 1e9),
+                       "sharding": "every rank decodes its own copy of the layer; no collective"},
+            "clocks": clocks,
+            "e2e": {"value": world * bf16_bytes / (e2e_ms / 1e3 / e2e_steps) / 1e9, "unit": UNIT,
+                    "h2d_bytes_per_step": int(h_pay.numel() + h_sm.numel() + h_desc.numel() + h_tab.numel()),
+                    "d2h_bytes_per_step": int(h_out.numel() * 2), "steps": e2e_steps},
+            "gpu_launches": args.steps,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": TRAFFIC_BYTES.get(w.label),
+                         "peak_kind": "of " + peak_kind, "algorithmic_bytes_per_launch": alg,
+                         "kernel": "zipmoe_dev::decode_kernel", "launch_ms": per_launch_s * 1e3},
+            "verified_bit_exact": verified,
+        }
+        if world == 1:
+            cores = os.cpu_count() or 1
+            count = int(max(cores, 20.0 / oracle_seconds_per_tensor(w.blobs[0])))   # ~20 s of CPU work
+            rate, dt = oracle_decode_rate(w.blobs, cores, count)
+            line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": "%d whole-tensor decodes cycling over the layer's %d tensors, %.1f s wall" % (
+                                        count, len(w.blobs), dt)}
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch, from the ncu capture summarised
+# under profiles/ (null until a capture of the current kernel exists)
+TRAFFIC_BYTES = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="small_layer", choices=["small_layer", "large_layer", "single_matrix"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

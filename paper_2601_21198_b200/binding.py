@@ -1,0 +1,227 @@
+"""Thin ctypes binding over the C ABI in include/zipmoe.h.
+
+Every function here has the name of the C entry point it forwards to and does
+argument marshalling only (numpy arrays / torch tensors -> pointers and sizes).
+`DecodePlan` lays several blobs out in contiguous host buffers and collects the
+descriptors zipmoe_blob_plan writes; it computes nothing of the codec.
+
+There is no fallback: if the CUDA library has not been built, importing this
+module raises.
+"""
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libzipmoe.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "CUDA library %s not found: build it with `python -m paper_2601_21198_b200.build` "
+        "(there is no CPU fallback)" % LIB_PATH)
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+OK = 0
+ERR_INVALID_ARG, ERR_BAD_FORMAT, ERR_BUFFER_TOO_SMALL, ERR_CUDA, ERR_DECODE_CORRUPT, ERR_UNSUPPORTED = -1, -2, -3, -4, -5, -6
+LAYOUT_LINEAR, LAYOUT_BLOCKED = 0, 1
+DEVICE_PAD_BYTES = 256
+
+_u64, _u32, _vp, _int = ctypes.c_uint64, ctypes.c_uint32, ctypes.c_void_p, ctypes.c_int
+
+
+class EncodeOpts(ctypes.Structure):
+    _fields_ = [("chunk_elems", _u32), ("max_code_len", _u32), ("layout", _u32), ("n_threads", _u32)]
+
+
+class BlobInfo(ctypes.Structure):
+    _fields_ = [("n_elems", _u64), ("rows", _u32), ("cols", _u32), ("layout", _u32), ("chunk_elems", _u32),
+                ("tile_elems", _u32), ("max_code_len", _u32), ("n_chunks", _u32), ("n_tiles", _u32),
+                ("table_off", _u64), ("chunk_off_off", _u64), ("payload_off", _u64), ("payload_bytes", _u64),
+                ("sm_off", _u64), ("sm_bytes", _u64), ("total_bytes", _u64)]
+
+
+CHUNK_DESC_DTYPE = np.dtype([
+    ("payload_off", "<u8"), ("sm_off", "<u8"), ("out_off", "<u8"), ("row_pitch", "<u4"), ("tiles_per_rowblk", "<u4"),
+    ("tile0", "<u4"), ("n_tiles", "<u4"), ("tile_elems", "<u4"), ("last_tile_elems", "<u4"), ("table_id", "<u4"),
+    ("tile_prefix", "<u4"), ("run_first_chunk", "<u4"), ("run_first_tile", "<u4"), ("run_end_tile", "<u4"),
+    ("tiles_per_chunk", "<u4")], align=True)
+assert CHUNK_DESC_DTYPE.itemsize == 72
+TABLE_BYTES = 256
+
+_lib.zipmoe_version.restype = _u32
+_lib.zipmoe_status_string.restype = ctypes.c_char_p
+_lib.zipmoe_status_string.argtypes = [_int]
+_lib.zipmoe_encode_bound.argtypes = [_u64, _u64, ctypes.POINTER(EncodeOpts), ctypes.POINTER(_u64)]
+_lib.zipmoe_encode.argtypes = [_vp, _u64, _u64, ctypes.POINTER(EncodeOpts), _vp, _u64, ctypes.POINTER(_u64)]
+_lib.zipmoe_blob_info_get.argtypes = [_vp, _u64, ctypes.POINTER(BlobInfo)]
+_lib.zipmoe_blob_validate.argtypes = [_vp, _u64]
+_lib.zipmoe_blob_plan.argtypes = [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _u32, _vp, _vp]
+_lib.zipmoe_decode.argtypes = [_vp, _u32, _u32, _vp, _u32, _vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp]
+for _f in ("zipmoe_encode_bound", "zipmoe_encode", "zipmoe_blob_info_get", "zipmoe_blob_validate",
+           "zipmoe_blob_plan", "zipmoe_decode"):
+    getattr(_lib, _f).restype = _int
+
+
+class ZipMoEError(RuntimeError):
+    def __init__(self, where, status):
+        self.status = status
+        super().__init__("%s: %s (%d)" % (where, zipmoe_status_string(status), status))
+
+
+def _check(where, status):
+    if status != OK:
+        raise ZipMoEError(where, status)
+
+
+def _ptr(a):
+    """Address of a numpy array, a torch tensor, an int, or None."""
+    if a is None:
+        return None
+    if isinstance(a, int):
+        return a
+    if isinstance(a, np.ndarray):
+        return a.ctypes.data
+    return a.data_ptr()
+
+
+def zipmoe_version():
+    return int(_lib.zipmoe_version())
+
+
+def zipmoe_status_string(status):
+    return _lib.zipmoe_status_string(int(status)).decode()
+
+
+def _opts(chunk_elems, max_code_len, layout, n_threads):
+    return EncodeOpts(int(chunk_elems), int(max_code_len), int(layout), int(n_threads))
+
+
+def zipmoe_encode_bound(rows, cols, chunk_elems=0, max_code_len=0, layout=LAYOUT_LINEAR, n_threads=0):
+    out = _u64(0)
+    o = _opts(chunk_elems, max_code_len, layout, n_threads)
+    _check("zipmoe_encode_bound", _lib.zipmoe_encode_bound(rows, cols, ctypes.byref(o), ctypes.byref(out)))
+    return out.value
+
+
+def zipmoe_encode(bf16, rows=None, cols=None, chunk_elems=0, max_code_len=0, layout=LAYOUT_LINEAR, n_threads=0):
+    """bf16 bit patterns (numpy uint16, row-major) -> blob (numpy uint8)."""
+    x = np.ascontiguousarray(bf16, dtype=np.uint16)
+    if rows is None:
+        rows, cols = (x.shape if x.ndim == 2 else (1, x.size))
+    if rows * cols != x.size:
+        raise ValueError("rows * cols != number of elements")
+    cap = zipmoe_encode_bound(rows, cols, chunk_elems, max_code_len, layout, n_threads)
+    blob = np.empty(cap, np.uint8)
+    n = _u64(0)
+    o = _opts(chunk_elems, max_code_len, layout, n_threads)
+    _check("zipmoe_encode", _lib.zipmoe_encode(_ptr(x), rows, cols, ctypes.byref(o), _ptr(blob), cap, ctypes.byref(n)))
+    return blob[: n.value].copy()
+
+
+def zipmoe_blob_info_get(blob):
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    info = BlobInfo()
+    _check("zipmoe_blob_info_get", _lib.zipmoe_blob_info_get(_ptr(blob), blob.size, ctypes.byref(info)))
+    return info
+
+
+def zipmoe_blob_validate(blob):
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    return int(_lib.zipmoe_blob_validate(_ptr(blob), blob.size))
+
+
+def zipmoe_blob_plan(blob, payload_base, sm_base, out_base, table_id, chunk_base, tile_base):
+    """Returns (descs: numpy structured array [n_chunks], table: numpy uint8 [256])."""
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    info = zipmoe_blob_info_get(blob)
+    descs = np.zeros(info.n_chunks, CHUNK_DESC_DTYPE)
+    table = np.zeros(TABLE_BYTES, np.uint8)
+    _check("zipmoe_blob_plan", _lib.zipmoe_blob_plan(_ptr(blob), blob.size, payload_base, sm_base, out_base, table_id,
+                                                     chunk_base, tile_base, _ptr(descs), _ptr(table)))
+    return descs, table
+
+
+def zipmoe_decode(chunks, n_chunks, n_tiles, tables, n_tables, payload, payload_bytes, sm, sm_bytes, out_bf16,
+                  out_elems, status_word=None, stream=None):
+    """All pointer arguments are device tensors (or raw device addresses)."""
+    _check("zipmoe_decode", _lib.zipmoe_decode(_ptr(chunks), n_chunks, n_tiles, _ptr(tables), n_tables, _ptr(payload),
+                                                payload_bytes, _ptr(sm), sm_bytes, _ptr(out_bf16), out_elems,
+                                                _ptr(status_word), _ptr(stream)))
+
+
+class DecodePlan:
+    """Host-side layout of one decode launch over several blobs: where each
+    blob's E-chunk section, SM section and output tensor sit in three contiguous
+    buffers, plus the chunk descriptors and tables from zipmoe_blob_plan."""
+
+    def __init__(self, blobs):
+        self.infos = [zipmoe_blob_info_get(b) for b in blobs]
+        pay = sm = out = 0
+        self.payload_base, self.sm_base, self.out_base = [], [], []
+        for inf in self.infos:
+            self.payload_base.append(pay)
+            self.sm_base.append(sm)
+            self.out_base.append(out)
+            pay += inf.payload_bytes                      # multiples of 16 by construction
+            sm += (inf.sm_bytes + 15) // 16 * 16
+            out += (inf.n_elems + 7) // 8 * 8
+        self.payload_bytes, self.sm_bytes, self.out_elems = pay, sm, out
+        self.payload = np.zeros(pay + DEVICE_PAD_BYTES, np.uint8)
+        self.sm = np.zeros(sm + DEVICE_PAD_BYTES, np.uint8)
+        descs, tables = [], []
+        chunk_base = tile_base = 0
+        for i, (b, inf) in enumerate(zip(blobs, self.infos)):
+            b = np.ascontiguousarray(b, dtype=np.uint8)
+            self.payload[self.payload_base[i]: self.payload_base[i] + inf.payload_bytes] = \
+                b[inf.payload_off: inf.payload_off + inf.payload_bytes]
+            self.sm[self.sm_base[i]: self.sm_base[i] + inf.sm_bytes] = b[inf.sm_off: inf.sm_off + inf.sm_bytes]
+            d, t = zipmoe_blob_plan(b, self.payload_base[i], self.sm_base[i], self.out_base[i], i, chunk_base,
+                                    tile_base)
+            descs.append(d)
+            tables.append(t)
+            chunk_base += inf.n_chunks
+            tile_base += inf.n_tiles
+        self.descs = np.concatenate(descs) if descs else np.zeros(0, CHUNK_DESC_DTYPE)
+        self.tables = np.concatenate(tables) if tables else np.zeros(0, np.uint8)
+        self.n_chunks, self.n_tiles, self.n_tables = chunk_base, tile_base, len(blobs)
+
+    def algorithmic_bytes(self):
+        """Bytes one decode must move: E-chunk section + SM bytes read, bf16 written."""
+        n = sum(inf.n_elems for inf in self.infos)
+        return self.payload_bytes + n + 2 * n
+
+    def to_device(self, device="cuda"):
+        import torch
+        return DevicePlan(self, torch.device(device))
+
+    def tensor_slice(self, out, i):
+        inf = self.infos[i]
+        return out[self.out_base[i]: self.out_base[i] + inf.n_elems]
+
+
+class DevicePlan:
+    """Device copies of a DecodePlan's buffers (torch owns the memory)."""
+
+    def __init__(self, plan, device):
+        import torch
+        self.plan = plan
+        self.device = device
+        self.descs = torch.from_numpy(plan.descs.view(np.uint8).copy()).to(device)
+        self.tables = torch.from_numpy(plan.tables).to(device)
+        self.payload = torch.from_numpy(plan.payload).to(device)
+        self.sm = torch.from_numpy(plan.sm).to(device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def new_output(self):
+        import torch
+        return torch.zeros(self.plan.out_elems, dtype=torch.int16, device=self.device)
+
+    def decode(self, out, stream=None):
+        """One zipmoe_decode launch on `stream` (a torch stream or None = current)."""
+        import torch
+        p = self.plan
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        zipmoe_decode(self.descs, p.n_chunks, p.n_tiles, self.tables, p.n_tables, self.payload, p.payload_bytes,
+                      self.sm, p.sm_bytes, out, p.out_elems, self.status, s.cuda_stream)

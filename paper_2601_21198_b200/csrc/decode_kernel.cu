@@ -1,0 +1,272 @@
+// Bulk decode kernel for sm_100a: E-chunk decompression and tensor recovery in
+// one pass (paper Section 3.1 "Real-time Inference", Section 3.3
+// "Memory-Coalesced Tensor Recovery Kernel").  The paper decompresses E-chunks
+// on CPU threads and uses the GPU only for the bit merge; here a warp decodes
+// a tile's 32 Huffman sub-streams by table lookup from shared memory and
+// merges each exponent byte with its sign+mantissa byte in registers, so the
+// decompressed exponents never reach global memory.
+//
+// Data movement per tile (256*I elements):
+//   global -> shared : the tile record (sub-stream bit counts + code bits) and
+//                      the tile's sign+mantissa bytes, each by one bulk
+//                      asynchronous copy (cp.async.bulk, completion on an
+//                      mbarrier), issued one tile ahead of the decode;
+//   shared -> regs   : 8 SM bytes per lane per iteration, code words on demand;
+//   regs   -> global : one 16-byte store per lane per iteration; a warp writes
+//                      512 contiguous bytes per iteration.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "zipmoe.h"
+#include "decode_device.cuh"
+
+namespace zipmoe_dev {
+
+constexpr int kWarps = 12;                 // warps per CTA, one CTA per SM
+constexpr int kThreads = kWarps * 32;
+constexpr int kPayBuf = 3072;              // record bytes staged per stage; longer records are read from global
+constexpr int kPaySlack = 256;             // readable bytes after a staged record
+constexpr int kSmBuf = 4096;
+constexpr int kStages = 2;
+constexpr int kWarpBytes = kStages * (kPayBuf + kPaySlack + kSmBuf);
+constexpr int kSmemBytes = kLutBytes + kWarps * kWarpBytes + kWarps * kStages * 8 + kLutScratchBytes;
+
+struct TileWork {
+  const uint8_t *rec;   // global address of the tile record
+  const uint8_t *sm;    // global address of the tile's sign+mantissa bytes
+  uint16_t *out;        // global address of the tile's first element
+  uint32_t rec_bytes, pitch, valid, iters;
+  bool ok, staged;
+};
+
+struct LaunchArgs {
+  const zipmoe_chunk_desc *chunks;
+  const zipmoe_table *tables;
+  const uint8_t *payload;
+  const uint8_t *sm;
+  uint16_t *out;
+  uint32_t *status;
+  uint64_t payload_bytes, sm_bytes, out_elems;
+  uint32_t n_chunks, n_tiles, n_tables, tiles_per_cta;
+};
+
+// Which descriptor holds global tile g: exact guess for launches whose chunks
+// all hold the same number of tiles, binary search on tile_prefix otherwise.
+__device__ uint32_t find_chunk(const LaunchArgs &a, uint32_t g) {
+  uint32_t c = (uint32_t)(((uint64_t)g * a.n_chunks) / a.n_tiles);
+  if (c >= a.n_chunks) c = a.n_chunks - 1;
+  uint32_t p = __ldg(&a.chunks[c].tile_prefix), m = __ldg(&a.chunks[c].n_tiles);
+  if (g >= p && g - p < m) return c;
+  uint32_t lo = 0, hi = a.n_chunks;  // invariant: prefix[lo] <= g (prefix[0] = 0)
+  while (hi - lo > 1) {
+    uint32_t mid = (lo + hi) >> 1;
+    if (__ldg(&a.chunks[mid].tile_prefix) <= g) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ TileWork resolve_tile(const LaunchArgs &a, uint32_t g, uint32_t run_first_chunk, uint32_t run_first_tile,
+                                 uint32_t tiles_per_chunk) {
+  TileWork w;
+  w.ok = false;
+  w.staged = false;
+  uint32_t rel = g - run_first_tile;
+  uint32_t c = run_first_chunk + rel / tiles_per_chunk, t = rel % tiles_per_chunk;
+  if (c >= a.n_chunks) return w;
+  const zipmoe_chunk_desc *d = a.chunks + c;
+  const uint64_t pay_off = __ldg(&d->payload_off), sm_off = __ldg(&d->sm_off), out_off = __ldg(&d->out_off);
+  const uint32_t pitch = __ldg(&d->row_pitch), tpr = __ldg(&d->tiles_per_rowblk), tile0 = __ldg(&d->tile0);
+  const uint32_t m = __ldg(&d->n_tiles), tile_elems = __ldg(&d->tile_elems), last = __ldg(&d->last_tile_elems);
+  if (t >= m || tpr == 0 || tile_elems == 0 || tile_elems > ZIPMOE_TILE_ELEMS_MAX || (tile_elems & 255) ||
+      last == 0 || last > tile_elems || (pitch & 7) || (pay_off & 15) || (sm_off & 15) || (out_off & 7))
+    return w;
+  if (pay_off + 4ull * (t + 2) > a.payload_bytes) return w;
+  const uint32_t *tab = reinterpret_cast<const uint32_t *>(a.payload + pay_off);
+  const uint32_t o0 = __ldg(tab + t), o1 = __ldg(tab + t + 1);
+  const uint64_t rec_off = pay_off + 16ull * o0;
+  if (o1 <= o0) return w;
+  w.rec_bytes = (o1 - o0) * 16u;
+  if (w.rec_bytes < 64 || w.rec_bytes > 64 + tile_elems / 8 * ZIPMOE_MAX_CODE_LEN + 16 ||
+      rec_off + w.rec_bytes > a.payload_bytes)
+    return w;
+  w.iters = tile_elems >> 8;
+  w.valid = (t == m - 1) ? last : tile_elems;
+  const uint32_t q = tile0 + t;
+  const uint64_t origin = out_off + (uint64_t)(q / tpr) * w.iters * pitch + (uint64_t)(q % tpr) * 256;
+  const uint32_t rows_used = (w.valid + 255) >> 8;
+  if (origin + (uint64_t)(rows_used - 1) * pitch + (w.valid - (rows_used - 1) * 256) > a.out_elems) return w;
+  const uint64_t sm_tile = sm_off + (uint64_t)t * tile_elems;
+  if (sm_tile + w.valid > a.sm_bytes) return w;
+  w.rec = a.payload + rec_off;
+  w.sm = a.sm + sm_tile;
+  w.out = a.out + origin;
+  w.pitch = pitch;
+  w.staged = w.rec_bytes <= kPayBuf;
+  w.ok = true;
+  return w;
+}
+
+__global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t *lut_raw = smem;
+  uint8_t *warp_base = smem + kLutBytes;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kLutBytes + kWarps * kWarpBytes);
+  uint8_t *lut_scratch = reinterpret_cast<uint8_t *>(bars + kWarps * kStages);
+
+  const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  uint32_t g0 = blockIdx.x * a.tiles_per_cta;
+  const uint32_t g1 = min(g0 + a.tiles_per_cta, a.n_tiles);
+  if (g0 >= g1) return;
+
+  uint8_t *my = warp_base + warp * kWarpBytes;
+  const uint32_t pay_addr = smem_addr(my);                                   // [stage][kPayBuf + kPaySlack]
+  const uint32_t sm_addr = smem_addr(my + kStages * (kPayBuf + kPaySlack));  // [stage][kSmBuf]
+  const uint32_t bar_addr = smem_addr(bars + warp * kStages);
+  const uint32_t lut_addr = smem_addr(lut_raw);
+  if (lane == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(bar_addr + 8 * s, 1);
+  }
+  fence_barrier_init();
+  __syncthreads();
+
+  uint32_t phase = 0;   // bit s = parity to wait for on stage s
+  bool dead = false;    // this warp gave up after a wait ran out
+  uint32_t c = find_chunk(a, g0);
+
+  while (g0 < g1) {
+    const zipmoe_chunk_desc *d = a.chunks + c;
+    const uint32_t table_id = __ldg(&d->table_id), run_first_chunk = __ldg(&d->run_first_chunk);
+    const uint32_t run_first_tile = __ldg(&d->run_first_tile), run_end_tile = __ldg(&d->run_end_tile);
+    const uint32_t tpc = __ldg(&d->tiles_per_chunk);
+    const uint32_t seg_end = min(g1, run_end_tile);
+    if (seg_end <= g0 || run_first_tile > g0 || tpc == 0 || table_id >= a.n_tables) {
+      report(a.status, kStatusBadDescriptor);
+      break;
+    }
+    __syncthreads();  // every warp is done with the previous table
+    build_lut<kThreads>(a.tables[table_id].code_len, lut_raw, lut_scratch, a.status);
+    __syncthreads();
+
+    uint32_t g = g0 + warp;
+    uint32_t stage = 0;
+    TileWork cur;
+    cur.ok = false;
+    if (g < seg_end && !dead) {
+      cur = resolve_tile(a, g, run_first_chunk, run_first_tile, tpc);
+      if (!cur.ok) report(a.status, kStatusBadDescriptor);
+      else if (lane == 0)
+        issue_tile_copies(cur.rec, cur.staged ? cur.rec_bytes : 0, cur.sm, (cur.valid + 15) & ~15u,
+                          pay_addr + stage * (kPayBuf + kPaySlack), sm_addr + stage * kSmBuf, bar_addr + 8 * stage);
+    }
+    for (; g < seg_end && !dead; g += kWarps) {
+      TileWork nxt;
+      nxt.ok = false;
+      const uint32_t g2 = g + kWarps;
+      if (g2 < seg_end) {
+        nxt = resolve_tile(a, g2, run_first_chunk, run_first_tile, tpc);
+        __syncwarp();  // all lanes have finished reading the other stage
+        if (!nxt.ok) report(a.status, kStatusBadDescriptor);
+        else if (lane == 0)
+          issue_tile_copies(nxt.rec, nxt.staged ? nxt.rec_bytes : 0, nxt.sm, (nxt.valid + 15) & ~15u,
+                            pay_addr + (stage ^ 1) * (kPayBuf + kPaySlack), sm_addr + (stage ^ 1) * kSmBuf,
+                            bar_addr + 8 * (stage ^ 1));
+      }
+      if (cur.ok) {
+        if (!mbar_wait_bounded(bar_addr + 8 * stage, (phase >> stage) & 1)) {
+          report(a.status, kStatusWaitTimeout);
+          // give the copies in flight one more bounded chance to land, then stop using the buffers
+          mbar_wait_bounded(bar_addr + 8 * stage, (phase >> stage) & 1);
+          if (nxt.ok) mbar_wait_bounded(bar_addr + 8 * (stage ^ 1), (phase >> (stage ^ 1)) & 1);
+          dead = true;
+          break;
+        }
+        phase ^= 1u << stage;
+        const uint32_t rec_s = pay_addr + stage * (kPayBuf + kPaySlack);
+        const uint32_t sm_s = sm_addr + stage * kSmBuf;
+        bool good;
+        if (cur.staged)
+          good = decode_tile<true>(rec_s, nullptr, cur.rec_bytes, sm_s, lut_addr, cur.out, cur.pitch, cur.valid,
+                                   cur.iters, lane);
+        else
+          good = decode_tile<false>(0, cur.rec, cur.rec_bytes, sm_s, lut_addr, cur.out, cur.pitch, cur.valid,
+                                    cur.iters, lane);
+        if (!good) report(a.status, kStatusBadBitCount);
+      }
+      cur = nxt;
+      stage ^= 1;
+    }
+    g0 = seg_end;
+    c = run_first_chunk + (run_end_tile - run_first_tile + tpc - 1) / tpc;
+    if (g0 < g1 && c >= a.n_chunks) {
+      report(a.status, kStatusBadDescriptor);
+      break;
+    }
+  }
+}
+
+}  // namespace zipmoe_dev
+
+namespace {
+struct DeviceInfo {
+  int sm_count = 0;
+  bool ready = false;
+};
+DeviceInfo g_dev[64];
+
+zipmoe_status prepare_device(int *sm_count) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ZIPMOE_ERR_CUDA;
+  if (!g_dev[dev].ready) {
+    int sms = 0, major = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ZIPMOE_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ZIPMOE_ERR_CUDA;
+    if (major != 10) return ZIPMOE_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(zipmoe_dev::decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             zipmoe_dev::kSmemBytes) != cudaSuccess)
+      return ZIPMOE_ERR_CUDA;
+    g_dev[dev].sm_count = sms;
+    g_dev[dev].ready = true;
+  }
+  *sm_count = g_dev[dev].sm_count;
+  return ZIPMOE_OK;
+}
+}  // namespace
+
+extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t n_chunks, uint32_t n_tiles,
+                                       const zipmoe_table *tables, uint32_t n_tables, const uint8_t *payload,
+                                       uint64_t payload_bytes, const uint8_t *sm, uint64_t sm_bytes,
+                                       uint16_t *out_bf16, uint64_t out_elems, uint32_t *status_word,
+                                       zipmoe_stream stream) {
+  if (n_chunks == 0 || n_tiles == 0) return (n_chunks == 0 && n_tiles == 0) ? ZIPMOE_OK : ZIPMOE_ERR_INVALID_ARG;
+  if (!chunks || !tables || n_tables == 0 || !payload || !sm || !out_bf16) return ZIPMOE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(payload) | reinterpret_cast<uintptr_t>(sm) | reinterpret_cast<uintptr_t>(out_bf16) |
+       reinterpret_cast<uintptr_t>(chunks)) & 15)
+    return ZIPMOE_ERR_INVALID_ARG;
+  if (status_word && (reinterpret_cast<uintptr_t>(status_word) & 3)) return ZIPMOE_ERR_INVALID_ARG;
+  int sms = 0;
+  zipmoe_status rc = prepare_device(&sms);
+  if (rc != ZIPMOE_OK) return rc;
+
+  zipmoe_dev::LaunchArgs a;
+  a.chunks = chunks;
+  a.tables = tables;
+  a.payload = payload;
+  a.sm = sm;
+  a.out = out_bf16;
+  a.status = status_word;
+  a.payload_bytes = payload_bytes;
+  a.sm_bytes = sm_bytes;
+  a.out_elems = out_elems;
+  a.n_chunks = n_chunks;
+  a.n_tiles = n_tiles;
+  a.n_tables = n_tables;
+  // one CTA per SM, each with a contiguous range of tiles
+  uint32_t ctas = (uint32_t)sms;
+  if (n_tiles < ctas) ctas = n_tiles;
+  a.tiles_per_cta = (n_tiles + ctas - 1) / ctas;
+  ctas = (n_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
+  zipmoe_dev::decode_kernel<<<ctas, zipmoe_dev::kThreads, zipmoe_dev::kSmemBytes,
+                              reinterpret_cast<cudaStream_t>(stream)>>>(a);
+  return cudaGetLastError() == cudaSuccess ? ZIPMOE_OK : ZIPMOE_ERR_CUDA;
+}

@@ -49,16 +49,22 @@ def single_expert_matrix(seed=0):
     return gaussian((2048, 1408), 0.02, seed)
 
 
-def small_expert_layer(n_experts=64, seed=1, hidden=2048, inter=1408):
-    """Experts of a DeepSeekV2-Lite / Qwen1.5-MoE sized layer: gate and up
-    [inter, hidden], down [hidden, inter]; per-expert std 0.02 * U(0.5, 1.5).
-    Yields (expert, name, array)."""
+SMALL_EXPERT_TENSORS = (("gate", (1408, 2048)), ("up", (1408, 2048)), ("down", (2048, 1408)))
+
+
+def small_expert_tensor(e, j, seed=1):
+    """Tensor j (0 gate, 1 up, 2 down) of expert e of a DeepSeekV2-Lite /
+    Qwen1.5-MoE sized layer: gate and up [1408, 2048], down [2048, 1408];
+    per-expert std 0.02 * U(0.5, 1.5)."""
+    std = 0.02 * float(_rng(seed + e).uniform(0.5, 1.5))
+    return gaussian(SMALL_EXPERT_TENSORS[j][1], std, 10_000 + 3 * (seed + e) + j)
+
+
+def small_expert_layer(n_experts=64, seed=1):
+    """Yields (expert, name, array) over the whole layer."""
     for e in range(n_experts):
-        scale = _rng(seed + e).uniform(0.5, 1.5)
-        std = 0.02 * float(scale)
-        yield e, "gate", gaussian((inter, hidden), std, 10_000 + 3 * (seed + e))
-        yield e, "up", gaussian((inter, hidden), std, 10_001 + 3 * (seed + e))
-        yield e, "down", gaussian((hidden, inter), std, 10_002 + 3 * (seed + e))
+        for j, (name, _) in enumerate(SMALL_EXPERT_TENSORS):
+            yield e, name, small_expert_tensor(e, j, seed)
 
 
 def outlier_matrix(rows, cols, std, seed, frac=0.001, gain=20.0):
@@ -77,13 +83,21 @@ def outlier_matrix(rows, cols, std, seed, frac=0.001, gain=20.0):
     return w
 
 
+LARGE_EXPERT_TENSORS = ("w1", "w3", "w2")
+
+
+def large_expert_tensor(e, j, seed=100, hidden=4096, inter=14336, std=0.015):
+    """Tensor j (0 w1, 1 w3: [inter, hidden]; 2 w2: [hidden, inter]) of expert e:
+    N(0, std) plus 0.1 % outlier channels at 20x."""
+    rows, cols = (inter, hidden) if j < 2 else (hidden, inter)
+    return outlier_matrix(rows, cols, std, 3 * (seed + e) + j)
+
+
 def large_expert_layer(n_experts=8, seed=100, hidden=4096, inter=14336, std=0.015):
-    """Experts with w1, w3 [inter, hidden] and w2 [hidden, inter], N(0, std)
-    plus 0.1 % outlier channels at 20x.  Yields (expert, name, array)."""
+    """Yields (expert, name, array) over the whole layer."""
     for e in range(n_experts):
-        yield e, "w1", outlier_matrix(inter, hidden, std, 3 * (seed + e))
-        yield e, "w3", outlier_matrix(inter, hidden, std, 3 * (seed + e) + 1)
-        yield e, "w2", outlier_matrix(hidden, inter, std, 3 * (seed + e) + 2)
+        for j, name in enumerate(LARGE_EXPERT_TENSORS):
+            yield e, name, large_expert_tensor(e, j, seed, hidden, inter, std)
 
 
 def special_patterns():

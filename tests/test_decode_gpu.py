@@ -1,0 +1,214 @@
+"""GPU parity: zipmoe_decode (through the C ABI) against the CPU oracle, bit for
+bit, on the same seeded inputs.  Small cases are compared element by element
+with the oracle's decode of the same blob; full-size configurations are
+compared with the original tensor (the one correct answer of a lossless codec)
+and, chunk by chunk on a sample, with the oracle's independent decode."""
+import numpy as np
+import pytest
+
+from oracle import codec
+from paper_2601_21198_b200 import build, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def zb():
+    build.build()
+    from paper_2601_21198_b200 import binding
+    return binding
+
+
+def gpu_decode(zb, blobs):
+    import torch
+    plan = zb.DecodePlan(blobs)
+    dev = plan.to_device()
+    out = dev.new_output()
+    out.fill_(0x5555)
+    dev.decode(out)
+    torch.cuda.synchronize()
+    assert int(dev.status.item()) == 0
+    host = out.cpu().numpy().view(np.uint16)
+    return plan, [plan.tensor_slice(host, i) for i in range(len(blobs))], host
+
+
+CASES = [
+    (1, 1, 0, 256), (1, 7, 0, 256), (1, 8, 0, 256), (1, 9, 0, 256), (1, 255, 0, 256), (1, 256, 0, 256), (1, 257, 0, 1024),
+    (3, 1000, 0, 1024), (1, 4095, 0, 4096), (1, 4096, 0, 4096), (1, 4097, 0, 4096), (5, 4099, 0, 16384),
+    (64, 1408, 0, 4096), (100, 1408, 0, 65536), (16, 256, 1, 4096), (48, 768, 1, 8192), (32, 4096, 1, 65536),
+    (16, 14336, 1, 262144), (333, 1031, 0, 262144),
+]
+
+
+@pytest.mark.parametrize("rows,cols,layout,chunk", CASES)
+def test_decode_matches_oracle_small(zb, rows, cols, layout, chunk):
+    x = inputs.gaussian((rows, cols), 0.02, rows * 31 + cols)
+    blob = zb.zipmoe_encode(x, layout=layout, chunk_elems=chunk)
+    _, (got,), _ = gpu_decode(zb, [blob])
+    want = codec.decode(blob)
+    assert np.array_equal(got, want)
+    assert np.array_equal(want, x.ravel())
+
+
+def test_decode_of_oracle_encoded_blobs(zb):
+    """The blob comes from the oracle's encoder (optimal length-limited code,
+    different tie-breaks): the GPU must decode it all the same."""
+    xs = [inputs.gaussian((40, 1000), 0.02, 5), inputs.gaussian((32, 512), 0.02, 6),
+          inputs.stress_tensor(1, max_elems=60000)[0]]
+    blobs = [codec.encode(xs[0], chunk_elems=4096), codec.encode(xs[1], layout=1, chunk_elems=8192),
+             codec.encode(xs[2], chunk_elems=1024, max_code_len=9)]
+    _, got, _ = gpu_decode(zb, blobs)
+    for g, x in zip(got, xs):
+        assert np.array_equal(g, x.ravel())
+
+
+def test_many_tensors_mixed_tiles_layouts_and_tables_in_one_launch(zb):
+    rng = np.random.default_rng(0)
+    xs, blobs = [], []
+    for i in range(40):
+        kind = i % 4
+        if kind == 0:
+            x = inputs.gaussian((int(rng.integers(1, 30000)),), 0.02 * (1 + i), i)
+            b = zb.zipmoe_encode(x, chunk_elems=1024)
+        elif kind == 1:
+            x = inputs.gaussian((int(rng.integers(1, 200000)),), 0.01, i)
+            b = zb.zipmoe_encode(x, chunk_elems=16384)
+        elif kind == 2:
+            x = inputs.gaussian((16 * int(rng.integers(1, 5)), 256 * int(rng.integers(1, 7))), 0.05, i)
+            b = zb.zipmoe_encode(x, layout=1, chunk_elems=8192)
+        else:
+            x = inputs.stress_tensor(i, max_elems=50000)[0]
+            b = zb.zipmoe_encode(x, chunk_elems=256)
+        xs.append(x)
+        blobs.append(b)
+    plan, got, host = gpu_decode(zb, blobs)
+    for g, x, b in zip(got, xs, blobs):
+        assert np.array_equal(g, codec.decode(b))
+        assert np.array_equal(g, x.ravel())
+    # the padding elements between tensors are never written
+    mask = np.ones(plan.out_elems, bool)
+    for i, inf in enumerate(plan.infos):
+        mask[plan.out_base[i]: plan.out_base[i] + inf.n_elems] = False
+    assert (host[mask] == 0x5555).all()
+
+
+def test_every_bit_pattern_and_special_values(zb):
+    rng = np.random.default_rng(1)
+    allp = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    rng.shuffle(allp)
+    sp = np.tile(inputs.special_patterns(), 7)
+    blobs = [zb.zipmoe_encode(allp, chunk_elems=c) for c in (256, 1024, 4096, 65536)] + \
+            [zb.zipmoe_encode(sp, chunk_elems=256)]
+    _, got, _ = gpu_decode(zb, blobs)
+    for g in got[:4]:
+        assert np.array_equal(g, allp)
+    assert np.array_equal(got[4], sp)
+
+
+def test_long_records_take_the_unstaged_path(zb):
+    """Near-uniform exponents: 8-bit codes, tile records of 4160 bytes, longer than
+    the staged-record buffer."""
+    x = inputs.stress_tensor(2, max_elems=300000)[0]
+    assert x.size > 20000
+    blob = zb.zipmoe_encode(x, chunk_elems=16384)
+    assert blob[64:320].min() >= 7
+    _, (got,), _ = gpu_decode(zb, [blob])
+    assert np.array_equal(got, codec.decode(blob)) and np.array_equal(got, x)
+
+
+def test_stress_set_sample(zb):
+    xs, blobs = [], []
+    for i in range(0, 96):
+        x, fam, chunk = inputs.stress_tensor(i, max_elems=1 << 18)
+        xs.append(x)
+        blobs.append(zb.zipmoe_encode(x, chunk_elems=chunk))
+    _, got, _ = gpu_decode(zb, blobs)
+    for i, (g, x) in enumerate(zip(got, xs)):
+        assert np.array_equal(g, x), i
+    for i in (0, 1, 2, 3, 50):
+        assert np.array_equal(got[i], codec.decode(blobs[i]))
+
+
+def test_empty_launch_and_bad_arguments(zb):
+    import torch
+    zb.zipmoe_decode(None, 0, 0, None, 0, None, 0, None, 0, None, 0)       # nothing to do: OK
+    t = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(zb.ZipMoEError):
+        zb.zipmoe_decode(t, 1, 1, None, 1, t, 16, t, 16, t, 8)               # null tables
+    with pytest.raises(zb.ZipMoEError):
+        zb.zipmoe_decode(t, 1, 1, t, 1, t.data_ptr() + 4, 16, t, 16, t, 8)   # misaligned payload
+
+
+def test_out_of_range_descriptors_set_the_status_word_and_write_nothing(zb):
+    """The kernel checks every offset against the buffer sizes it was given: a
+    descriptor that points outside is reported and its tiles are skipped."""
+    import torch
+    x = inputs.gaussian((3, 5000), 0.02, 8)
+    plan = zb.DecodePlan([zb.zipmoe_encode(x, chunk_elems=4096)])
+    for field, value in [("payload_off", plan.payload_bytes + 4096), ("sm_off", plan.sm_bytes),
+                         ("out_off", plan.out_elems), ("table_id", 5)]:
+        bad = zb.DecodePlan.__new__(zb.DecodePlan)
+        bad.__dict__.update(plan.__dict__)
+        bad.descs = plan.descs.copy()
+        bad.descs[field][1] = value
+        dev = bad.to_device()
+        out = dev.new_output()
+        out.fill_(0x5555)
+        dev.decode(out)
+        torch.cuda.synchronize()
+        assert int(dev.status.item()) != 0, field
+        host = out.cpu().numpy().view(np.uint16)
+        assert (host[4096:8192] == 0x5555).all(), field
+
+
+def test_single_matrix_config_full(zb):
+    from paper_2601_21198_b200 import workloads
+    w = workloads.single_matrix()
+    dev = w.plan.to_device()
+    out = dev.new_output()
+    dev.decode(out)
+    got = out.cpu().numpy().view(np.uint16)
+    assert int(dev.status.item()) == 0
+    assert np.array_equal(got, codec.decode(w.blobs[0]))
+    assert np.array_equal(got, w.originals[0].ravel())
+
+
+def _check_full_workload(zb, w, n_sample_chunks):
+    """Whole output against the originals on the device; sampled chunks against
+    the oracle's independent decode of the same blob."""
+    import torch
+    dev = w.plan.to_device()
+    out = dev.new_output()
+    dev.decode(out)
+    torch.cuda.synchronize()
+    assert int(dev.status.item()) == 0
+    for i, x in enumerate(w.originals):
+        ref = torch.from_numpy(x.view(np.int16).ravel()).cuda()
+        assert torch.equal(w.plan.tensor_slice(out, i), ref), w.names[i]
+        del ref
+    rng = np.random.default_rng(123)
+    for _ in range(n_sample_chunks):
+        i = int(rng.integers(len(w.blobs)))
+        inf = w.plan.infos[i]
+        k = int(rng.integers(inf.n_chunks))
+        want = np.zeros(inf.n_elems, np.uint16)
+        codec.decode_chunk(w.blobs[i], k, want)
+        got = w.plan.tensor_slice(out, i).cpu().numpy().view(np.uint16)
+        touched = want != 0
+        assert touched.sum() > 0.9 * min(inf.chunk_elems, inf.n_elems - k * inf.chunk_elems)
+        assert np.array_equal(got[touched], want[touched])
+
+
+def test_small_expert_layer_config_full(zb):
+    from paper_2601_21198_b200 import workloads
+    _check_full_workload(zb, workloads.small_layer(), 24)
+
+
+def test_large_expert_layer_config_full(zb):
+    from paper_2601_21198_b200 import workloads
+    _check_full_workload(zb, workloads.large_layer(), 8)
+
+
+def test_large_expert_layer_blocked_layout(zb):
+    from paper_2601_21198_b200 import workloads
+    _check_full_workload(zb, workloads.large_layer(n_experts=1, layout=1), 6)
