@@ -44,12 +44,12 @@ def measured_peaks():
     return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
 
 
-def build_workload(name, keep_originals):
+def build_workload(name, keep_originals, experts=None):
     from paper_2601_21198_b200 import workloads
     if name == "small_layer":
-        return workloads.small_layer(keep_originals=keep_originals)
+        return workloads.small_layer(n_experts=experts or 64, keep_originals=keep_originals)
     if name == "large_layer":
-        return workloads.large_layer(keep_originals=keep_originals)
+        return workloads.large_layer(n_experts=experts or 8, keep_originals=keep_originals)
     if name == "single_matrix":
         return workloads.single_matrix(keep_originals=keep_originals)
     raise SystemExit("unknown workload %s" % name)
@@ -174,7 +174,7 @@ def run_ours(args):
 
     from paper_2601_21198_b200 import binding, build
     build.build()
-    w = build_workload(args.workload, keep_originals=False)
+    w = build_workload(args.workload, keep_originals=False, experts=args.experts)
     plan = w.plan
     dplan = plan.to_device(dev)
     out = dplan.new_output()
@@ -300,6 +300,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="small_layer", choices=["small_layer", "large_layer", "single_matrix"])
+    ap.add_argument("--experts", type=int, default=None,
+                    help="fewer experts than the configuration names (profiling captures on a small case only)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

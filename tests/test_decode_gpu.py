@@ -108,8 +108,7 @@ def test_every_bit_pattern_and_special_values(zb):
 def test_long_records_take_the_unstaged_path(zb):
     """Near-uniform exponents: 8-bit codes, tile records of 4160 bytes, longer than
     the staged-record buffer."""
-    x = inputs.stress_tensor(2, max_elems=300000)[0]
-    assert x.size > 20000
+    x = np.random.default_rng(2).integers(0, 1 << 16, 50021, dtype=np.uint16)
     blob = zb.zipmoe_encode(x, chunk_elems=16384)
     assert blob[64:320].min() >= 7
     _, (got,), _ = gpu_decode(zb, [blob])
