@@ -44,14 +44,14 @@ def measured_peaks():
     return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
 
 
-def build_workload(name, keep_originals, experts=None):
+def build_workload(name, keep_originals, experts=None, max_code_len=0):
     from paper_2601_21198_b200 import workloads
     if name == "small_layer":
-        return workloads.small_layer(n_experts=experts or 64, keep_originals=keep_originals)
+        return workloads.small_layer(n_experts=experts or 64, keep_originals=keep_originals, max_code_len=max_code_len)
     if name == "large_layer":
-        return workloads.large_layer(n_experts=experts or 8, keep_originals=keep_originals)
+        return workloads.large_layer(n_experts=experts or 8, keep_originals=keep_originals, max_code_len=max_code_len)
     if name == "single_matrix":
-        return workloads.single_matrix(keep_originals=keep_originals)
+        return workloads.single_matrix(keep_originals=keep_originals, max_code_len=max_code_len)
     raise SystemExit("unknown workload %s" % name)
 
 
@@ -174,7 +174,7 @@ def run_ours(args):
 
     from paper_2601_21198_b200 import binding, build
     build.build()
-    w = build_workload(args.workload, keep_originals=False, experts=args.experts)
+    w = build_workload(args.workload, keep_originals=False, experts=args.experts, max_code_len=args.max_code_len)
     plan = w.plan
     dplan = plan.to_device(dev)
     out = dplan.new_output()
@@ -260,7 +260,8 @@ def run_ours(args):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_launch_s * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u16", "data": "synthetic",
             "config": {"workload": w.label, "tensors": len(w.blobs), "elements": w.n_elems,
-                       "chunk_elems": int(plan.infos[0].chunk_elems), "chunks": plan.n_chunks, "tiles": plan.n_tiles,
+                       "chunk_elems": int(plan.infos[0].chunk_elems),
+                       "max_code_len": int(plan.infos[0].max_code_len), "chunks": plan.n_chunks, "tiles": plan.n_tiles,
                        "compressed_over_bf16": w.compressed_bytes() / bf16_bytes,
                        "l2": "inputs and outputs of one step (%.2f GB) exceed L2; no flush" % (alg / 1e9),
                        "sharding": "every rank decodes its own copy of the layer; no collective"},
@@ -300,6 +301,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="small_layer", choices=["small_layer", "large_layer", "single_matrix"])
+    ap.add_argument("--max-code-len", type=int, default=0, help="longest Huffman code the encoder may use (8..12)")
     ap.add_argument("--experts", type=int, default=None,
                     help="fewer experts than the configuration names (profiling captures on a small case only)")
     args = ap.parse_args()

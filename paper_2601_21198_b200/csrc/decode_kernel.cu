@@ -23,20 +23,22 @@
 
 namespace zipmoe_dev {
 
-constexpr int kWarps = 12;                 // warps per CTA, one CTA per SM
+constexpr int kWarps = 20;                 // warps per CTA, one CTA per SM
 constexpr int kThreads = kWarps * 32;
-constexpr int kPayBuf = 3072;              // record bytes staged per stage; longer records are read from global
-constexpr int kPaySlack = 256;             // readable bytes after a staged record
-constexpr int kSmBuf = 4096;
-constexpr int kStages = 2;
-constexpr int kWarpBytes = kStages * (kPayBuf + kPaySlack + kSmBuf);
-constexpr int kSmemBytes = kLutBytes + kWarps * kWarpBytes + kWarps * kStages * 8 + kLutScratchBytes;
+constexpr int kPayBuf = 2048;              // record bytes staged per stage; longer records are read from global
+constexpr int kPaySlack = 64;              // readable bytes after a staged record (a lane looks two words ahead)
+constexpr int kPayStage = kPayBuf + kPaySlack;
+constexpr int kPayStages = 2;
+constexpr int kBarsPerWarp = kPayStages + kSmPieces;   // two record stages, four sign+mantissa slots
+constexpr int kWarpBytes = kPayStages * kPayStage + kSmPieces * kSmPieceBytes;
+constexpr int kSmemBytes = kLutBytes + kWarps * kWarpBytes + kWarps * kBarsPerWarp * 8 + kLutScratchBytes;
+static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
 
 struct TileWork {
   const uint8_t *rec;   // global address of the tile record
   const uint8_t *sm;    // global address of the tile's sign+mantissa bytes
   uint16_t *out;        // global address of the tile's first element
-  uint32_t rec_bytes, pitch, valid, iters;
+  uint32_t rec_bytes, pitch, valid, iters, pieces;
   bool ok, staged;
 };
 
@@ -91,6 +93,7 @@ __device__ TileWork resolve_tile(const LaunchArgs &a, uint32_t g, uint32_t run_f
       rec_off + w.rec_bytes > a.payload_bytes)
     return w;
   w.iters = tile_elems >> 8;
+  w.pieces = (w.iters + 3) >> 2;
   w.valid = (t == m - 1) ? last : tile_elems;
   const uint32_t q = tile0 + t;
   const uint64_t origin = out_off + (uint64_t)(q / tpr) * w.iters * pitch + (uint64_t)(q % tpr) * 256;
@@ -107,30 +110,95 @@ __device__ TileWork resolve_tile(const LaunchArgs &a, uint32_t g, uint32_t run_f
   return w;
 }
 
+// Per-warp asynchronous pipeline.  A warp decodes its tiles one after the other;
+// the record of the next tile is copied into the other record stage while the
+// current one is decoded, and piece p of the next tile's sign+mantissa bytes is
+// copied into slot p as soon as the current tile is done with its piece p.
+struct WarpPipe {
+  uint32_t pay_addr, sm_addr, bar_addr;   // shared addresses: record stages, SM slots, barriers
+  uint32_t phase;                         // bit b = parity to wait for on barrier b
+  uint32_t pending;                       // bit b = a copy on barrier b has been started and not waited for
+  uint32_t lane;
+
+  __device__ __forceinline__ uint32_t bar(uint32_t b) const { return bar_addr + 8 * b; }
+  __device__ __forceinline__ bool wait(uint32_t b) {
+    if (!mbar_wait_bounded(bar(b), (phase >> b) & 1u)) return false;
+    phase ^= 1u << b;
+    pending &= ~(1u << b);
+    return true;
+  }
+  // all lanes call these; one lane starts the copy
+  __device__ __forceinline__ void load_record(const TileWork &t, uint32_t stage) {
+    if (!t.staged) return;
+    if (lane == 0) bulk_load(pay_addr + stage * kPayStage, t.rec, t.rec_bytes, bar(stage));
+    pending |= 1u << stage;
+  }
+  __device__ __forceinline__ void load_sm_piece(const TileWork &t, uint32_t p) {
+    const uint32_t all = (t.valid + 15u) & ~15u;
+    const uint32_t bytes = min(kSmPieceBytes, all - p * kSmPieceBytes);
+    if (lane == 0) bulk_load(sm_addr + p * kSmPieceBytes, t.sm + p * kSmPieceBytes, bytes, bar(kPayStages + p));
+    pending |= 1u << (kPayStages + p);
+  }
+  // after a wait ran out: give what is still in flight one short, bounded chance to land
+  __device__ __forceinline__ void drain() {
+    for (uint32_t b = 0; b < (uint32_t)kBarsPerWarp; ++b)
+      if (pending & (1u << b)) mbar_wait_bounded(bar(b), (phase >> b) & 1u, 1u << 14);
+  }
+};
+
+struct SmFeed {
+  WarpPipe &pipe;
+  const TileWork &nxt;
+  uint32_t &nxt_issued;   // pieces of the next tile already started
+  __device__ __forceinline__ uint32_t begin(uint32_t p) {
+    if (!pipe.wait(kPayStages + p)) return 0xFFFFFFFFu;
+    return pipe.sm_addr + p * kSmPieceBytes;
+  }
+  __device__ __forceinline__ void end(uint32_t p) {
+    __syncwarp();   // every lane has read the slot
+    if (nxt.ok && p == nxt_issued && p < nxt.pieces) {
+      pipe.load_sm_piece(nxt, p);
+      ++nxt_issued;
+    }
+  }
+};
+
+struct GlobalSink {
+  uint16_t *out;
+  uint32_t pitch;
+  __device__ __forceinline__ void group(uint32_t i, uint32_t lane, const uint4 &v) const {
+    __stcs(reinterpret_cast<uint4 *>(out + (size_t)i * pitch + lane * 8), v);
+  }
+  __device__ __forceinline__ void elem(uint32_t i, uint32_t lane, uint32_t j, uint16_t v) const {
+    out[(size_t)i * pitch + lane * 8 + j] = v;
+  }
+};
+
 __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t *lut_raw = smem;
   uint8_t *warp_base = smem + kLutBytes;
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kLutBytes + kWarps * kWarpBytes);
-  uint8_t *lut_scratch = reinterpret_cast<uint8_t *>(bars + kWarps * kStages);
+  uint8_t *lut_scratch = reinterpret_cast<uint8_t *>(bars + kWarps * kBarsPerWarp);
 
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint32_t g0 = blockIdx.x * a.tiles_per_cta;
   const uint32_t g1 = min(g0 + a.tiles_per_cta, a.n_tiles);
   if (g0 >= g1) return;
 
-  uint8_t *my = warp_base + warp * kWarpBytes;
-  const uint32_t pay_addr = smem_addr(my);                                   // [stage][kPayBuf + kPaySlack]
-  const uint32_t sm_addr = smem_addr(my + kStages * (kPayBuf + kPaySlack));  // [stage][kSmBuf]
-  const uint32_t bar_addr = smem_addr(bars + warp * kStages);
-  const uint32_t lut_addr = smem_addr(lut_raw);
-  if (lane == 0) {
-    for (int s = 0; s < kStages; ++s) mbar_init(bar_addr + 8 * s, 1);
-  }
+  WarpPipe pipe;
+  pipe.pay_addr = smem_addr(warp_base + warp * kWarpBytes);
+  pipe.sm_addr = pipe.pay_addr + kPayStages * kPayStage;
+  pipe.bar_addr = smem_addr(bars + warp * kBarsPerWarp);
+  pipe.phase = 0;
+  pipe.pending = 0;
+  pipe.lane = lane;
+  const uint32_t lane_lut = smem_addr(lut_raw), wide_lut = lane_lut + kLaneLutBytes;
+  if (lane == 0)
+    for (int b = 0; b < kBarsPerWarp; ++b) mbar_init(pipe.bar(b), 1);
   fence_barrier_init();
   __syncthreads();
 
-  uint32_t phase = 0;   // bit s = parity to wait for on stage s
   bool dead = false;    // this warp gave up after a wait ran out
   uint32_t c = find_chunk(a, g0);
 
@@ -145,8 +213,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
       break;
     }
     __syncthreads();  // every warp is done with the previous table
-    build_lut<kThreads>(a.tables[table_id].code_len, lut_raw, lut_scratch, a.status);
-    __syncthreads();
+    const bool escape = build_lut<kThreads>(a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) >
+                        (uint32_t)kLaneLutBits;
 
     uint32_t g = g0 + warp;
     uint32_t stage = 0;
@@ -155,44 +223,61 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
     if (g < seg_end && !dead) {
       cur = resolve_tile(a, g, run_first_chunk, run_first_tile, tpc);
       if (!cur.ok) report(a.status, kStatusBadDescriptor);
-      else if (lane == 0)
-        issue_tile_copies(cur.rec, cur.staged ? cur.rec_bytes : 0, cur.sm, (cur.valid + 15) & ~15u,
-                          pay_addr + stage * (kPayBuf + kPaySlack), sm_addr + stage * kSmBuf, bar_addr + 8 * stage);
+      else {
+        pipe.load_record(cur, stage);
+        for (uint32_t p = 0; p < cur.pieces; ++p) pipe.load_sm_piece(cur, p);
+      }
     }
     for (; g < seg_end && !dead; g += kWarps) {
       TileWork nxt;
       nxt.ok = false;
+      uint32_t nxt_issued = 0;
       const uint32_t g2 = g + kWarps;
       if (g2 < seg_end) {
         nxt = resolve_tile(a, g2, run_first_chunk, run_first_tile, tpc);
-        __syncwarp();  // all lanes have finished reading the other stage
         if (!nxt.ok) report(a.status, kStatusBadDescriptor);
-        else if (lane == 0)
-          issue_tile_copies(nxt.rec, nxt.staged ? nxt.rec_bytes : 0, nxt.sm, (nxt.valid + 15) & ~15u,
-                            pay_addr + (stage ^ 1) * (kPayBuf + kPaySlack), sm_addr + (stage ^ 1) * kSmBuf,
-                            bar_addr + 8 * (stage ^ 1));
+        else pipe.load_record(nxt, stage ^ 1);   // that stage was released by the __syncwarp below
       }
       if (cur.ok) {
-        if (!mbar_wait_bounded(bar_addr + 8 * stage, (phase >> stage) & 1)) {
-          report(a.status, kStatusWaitTimeout);
-          // give the copies in flight one more bounded chance to land, then stop using the buffers
-          mbar_wait_bounded(bar_addr + 8 * stage, (phase >> stage) & 1);
-          if (nxt.ok) mbar_wait_bounded(bar_addr + 8 * (stage ^ 1), (phase >> (stage ^ 1)) & 1);
+        uint32_t rc = 0;
+        if (cur.staged && !pipe.wait(stage)) rc = kStatusWaitTimeout;
+        if (rc == 0) {
+          const uint32_t rec_s = pipe.pay_addr + stage * kPayStage;
+          SmFeed feed{pipe, nxt, nxt_issued};
+          GlobalSink sink{cur.out, cur.pitch};
+          if (cur.staged) {
+            rc = escape ? decode_tile<true, true>(rec_s, nullptr, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
+                                                  cur.iters, lane, feed, sink)
+                        : decode_tile<true, false>(rec_s, nullptr, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
+                                                   cur.iters, lane, feed, sink);
+          } else {
+            rc = escape ? decode_tile<false, true>(0, cur.rec, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
+                                                   cur.iters, lane, feed, sink)
+                        : decode_tile<false, false>(0, cur.rec, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
+                                                    cur.iters, lane, feed, sink);
+          }
+        }
+        if (rc == kStatusWaitTimeout) {
+          report(a.status, rc);
+          pipe.drain();
           dead = true;
           break;
         }
-        phase ^= 1u << stage;
-        const uint32_t rec_s = pay_addr + stage * (kPayBuf + kPaySlack);
-        const uint32_t sm_s = sm_addr + stage * kSmBuf;
-        bool good;
-        if (cur.staged)
-          good = decode_tile<true>(rec_s, nullptr, cur.rec_bytes, sm_s, lut_addr, cur.out, cur.pitch, cur.valid,
-                                   cur.iters, lane);
-        else
-          good = decode_tile<false>(0, cur.rec, cur.rec_bytes, sm_s, lut_addr, cur.out, cur.pitch, cur.valid,
-                                    cur.iters, lane);
-        if (!good) report(a.status, kStatusBadBitCount);
+        if (rc == kStatusBadBitCount) {
+          // nothing was decoded: take the tile's sign+mantissa pieces off the barriers
+          report(a.status, rc);
+          for (uint32_t p = 0; p < cur.pieces && !dead; ++p)
+            if (!pipe.wait(kPayStages + p)) dead = true;
+          if (dead) {
+            report(a.status, kStatusWaitTimeout);
+            pipe.drain();
+            break;
+          }
+        }
       }
+      __syncwarp();   // every lane is done with the current record stage and SM slots
+      if (nxt.ok)
+        for (; nxt_issued < nxt.pieces; ++nxt_issued) pipe.load_sm_piece(nxt, nxt_issued);
       cur = nxt;
       stage ^= 1;
     }

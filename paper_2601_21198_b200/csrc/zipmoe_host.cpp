@@ -221,7 +221,7 @@ zipmoe_status zipmoe_encode_bound(uint64_t rows, uint64_t cols, const zipmoe_enc
 
 zipmoe_status zipmoe_encode(const uint16_t *bf16, uint64_t rows, uint64_t cols, const zipmoe_encode_opts *opts,
                             void *blob_v, uint64_t blob_cap, uint64_t *blob_bytes) {
-  if (!blob_bytes || (!bf16 && rows * cols) || !blob_v) return ZIPMOE_ERR_INVALID_ARG;
+  if (!blob_bytes || (!bf16 && rows != 0 && cols != 0) || !blob_v) return ZIPMOE_ERR_INVALID_ARG;
   Opts o;
   Geometry g;
   zipmoe_status rc = resolve_opts(opts, &o);

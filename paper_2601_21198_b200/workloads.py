@@ -13,7 +13,7 @@ def host_threads():
     return max(1, min(32, (os.cpu_count() or 1)))
 
 
-def _encode_all(named_tensors, chunk_elems, layout, keep_originals):
+def _encode_all(named_tensors, chunk_elems, layout, keep_originals, max_code_len=0):
     """named_tensors: iterable of (name, thunk -> uint16 array).  Tensors are
     drawn and encoded on a small thread pool (numpy and the encoder release the
     GIL); returns (names, blobs, originals or None)."""
@@ -27,7 +27,8 @@ def _encode_all(named_tensors, chunk_elems, layout, keep_originals):
         x = thunk()
         rows, cols = (x.shape if x.ndim == 2 else (1, x.size))
         lay = layout if (layout == binding.LAYOUT_LINEAR or (rows % 16 == 0 and cols % 256 == 0)) else 0
-        blob = binding.zipmoe_encode(x, rows, cols, chunk_elems=chunk_elems, layout=lay, n_threads=inner)
+        blob = binding.zipmoe_encode(x, rows, cols, chunk_elems=chunk_elems, layout=lay, n_threads=inner,
+                                     max_code_len=max_code_len)
         return name, blob, (x if keep_originals else None)
 
     with ThreadPoolExecutor(outer) as pool:
@@ -54,22 +55,23 @@ class Workload:
         return sum(b.size for b in self.blobs)
 
 
-def single_matrix(keep_originals=True):
+def single_matrix(keep_originals=True, max_code_len=0):
     """One 2048x1408 expert matrix, 4096-element chunks."""
     items = [("expert0", lambda: inputs.single_expert_matrix(0))]
-    return Workload("single_2048x1408_chunk4096", *_encode_all(items, 4096, 0, keep_originals))
+    return Workload("single_2048x1408_chunk4096", *_encode_all(items, 4096, 0, keep_originals, max_code_len))
 
 
-def small_layer(n_experts=64, keep_originals=True, layout=0):
+def small_layer(n_experts=64, keep_originals=True, layout=0, max_code_len=0):
     """64 experts x {gate, up [1408,2048]; down [2048,1408]}, 64K-element chunks (~1.1 GB bf16)."""
     items = []
     for e in range(n_experts):
         for j, (name, _) in enumerate(inputs.SMALL_EXPERT_TENSORS):
             items.append(("e%d.%s" % (e, name), lambda e=e, j=j: inputs.small_expert_tensor(e, j)))
-    return Workload("moe%d_2048x1408_chunk64K" % n_experts, *_encode_all(items, 65536, layout, keep_originals))
+    return Workload("moe%d_2048x1408_chunk64K" % n_experts, *_encode_all(items, 65536, layout, keep_originals, max_code_len))
 
 
-def large_layer(n_experts=8, keep_originals=True, layout=0, hidden=4096, inter=14336, chunk_elems=262144):
+def large_layer(n_experts=8, keep_originals=True, layout=0, hidden=4096, inter=14336, chunk_elems=262144,
+                max_code_len=0):
     """8 experts x {w1, w3 [14336,4096]; w2 [4096,14336]} with outlier channels, 256K-element chunks (~2.8 GB bf16)."""
     items = []
     for e in range(n_experts):
@@ -77,7 +79,7 @@ def large_layer(n_experts=8, keep_originals=True, layout=0, hidden=4096, inter=1
             items.append(("e%d.%s" % (e, name),
                           lambda e=e, j=j: inputs.large_expert_tensor(e, j, hidden=hidden, inter=inter)))
     label = "moe%d_%dx%d_chunk%dK" % (n_experts, inter, hidden, chunk_elems // 1024)
-    return Workload(label, *_encode_all(items, chunk_elems, layout, keep_originals))
+    return Workload(label, *_encode_all(items, chunk_elems, layout, keep_originals, max_code_len))
 
 
 def stress_set(n_tensors=4096, chunk_elems=None, keep_originals=True, max_elems=4 << 20):
