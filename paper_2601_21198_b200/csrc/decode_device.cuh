@@ -194,13 +194,50 @@ __device__ uint32_t build_lut(const uint8_t *code_len, uint8_t *lut_raw, uint8_t
 // ---- tile decoder -------------------------------------------------------------
 template <bool STAGED>
 struct WordSource {
-  uint32_t base_s;           // shared address of the bit area (STAGED)
-  const uint32_t *base_g;    // global address of the bit area (!STAGED)
-  __device__ __forceinline__ uint32_t word(uint32_t idx) const {
-    if (STAGED) return lds_u32(base_s + 4 * idx);
-    return __ldg(base_g + idx);
+  uint32_t at_s;             // shared address of the next unread word (STAGED)
+  const uint32_t *at_g;      // global address of the next unread word (!STAGED)
+  __device__ __forceinline__ uint32_t pop() {
+    if (STAGED) {
+      const uint32_t v = lds_u32(at_s);
+      at_s += 4;
+      return v;
+    }
+    return __ldg(at_g++);
+  }
+  // If bit 5 of pos is set (a whole word has been consumed): b_hi <- b_lo,
+  // b_lo <- next word, clear the bit.  Predicated, no branch.
+  __device__ __forceinline__ void advance(uint32_t &pos, uint32_t &b_hi, uint32_t &b_lo) {
+    if (STAGED) {
+      asm volatile(
+          "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
+          "and.b32 t, %0, 32;\n\t"
+          "setp.ne.u32 p, t, 0;\n\t"
+          "@p mov.b32 %1, %2;\n\t"
+          "@p ld.shared.u32 %2, [%3];\n\t"
+          "@p add.u32 %3, %3, 4;\n\t"
+          "@p xor.b32 %0, %0, 32;\n\t}"
+          : "+r"(pos), "+r"(b_hi), "+r"(b_lo), "+r"(at_s));
+    } else {
+      asm volatile(
+          "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
+          "and.b32 t, %0, 32;\n\t"
+          "setp.ne.u32 p, t, 0;\n\t"
+          "@p mov.b32 %1, %2;\n\t"
+          "@p ld.global.nc.u32 %2, [%3];\n\t"
+          "@p add.u64 %3, %3, 4;\n\t"
+          "@p xor.b32 %0, %0, 32;\n\t}"
+          : "+r"(pos), "+r"(b_hi), "+r"(b_lo), "+l"(at_g));
+    }
   }
 };
+
+// a*b + c on the multiply-add pipe (keeps pure integer adds and shifts-by-constant
+// off the ALU pipe, which the variable shifts and logic ops of the decoder fill)
+__device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
 
 // Decodes one tile with the 32 lanes of a warp.
 //   record  : in shared memory at rec_s (STAGED) or in global memory at rec_g;
@@ -211,17 +248,20 @@ struct WordSource {
 //             sink.elem(i, lane, j, v) one bf16 of the short last group of a
 //             linear tensor.
 // The code bits of a lane form a stream of u32 words consumed from bit 31 down.
-// The lane keeps a 64-bit window (hi:lo) whose top bits are the next code bits.
-// `used` counts, in its low 7 bits, the bits shifted out since the window was
-// last full; whole table entries are added to it (their low 4 bits are the code
-// length, bits 4..6 are zero), so bits 7 and up are meaningless.  A new word is
-// shifted in whenever 32 bits are free, which is checked after every four codes:
-// the window then holds at least 33 bits, enough for four codes of at most 8
-// bits.  A code longer than 8 bits (ESCAPE only) shows as a zero entry of the
-// lane table and is resolved through the wide table with its own checks.
+// The lane keeps two consecutive words of it (b_hi:b_lo) and the bit position
+// `pos` of the next code inside them (pos mod 64 < 32 between batches).  A batch
+// takes the 32 bits at pos into one register and decodes from its top:
+//   FAST  (no code longer than 8 bits): four codes per batch, looked up in the
+//         lane table with the top 8 bits;
+//   !FAST (codes up to 12 bits): two codes per batch, looked up in the wide
+//         table with the top 12 bits.
+// Whole table entries are added to pos: their low 4 bits are the code length and
+// bits 4..6 are zero, so the low 7 bits of pos stay exact and the rest is
+// ignored (the funnel shifts take the shift amount mod 32).  When bit 5 of pos
+// is set a whole word has been consumed and the next one is shifted in.
 // Returns 0 on success, else a status code (warp-uniform); on
 // kStatusBadBitCount nothing has been written.
-template <bool STAGED, bool ESCAPE, class Feed, class Sink>
+template <bool STAGED, bool FAST, class Feed, class Sink>
 __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *rec_g, uint32_t rec_bytes,
                                                 uint32_t lane_lut, uint32_t wide_lut, uint32_t valid, uint32_t iters,
                                                 uint32_t lane, Feed &feed, Sink &sink) {
@@ -239,69 +279,91 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
   const uint32_t start = incl - my_bits;
 
   WordSource<STAGED> src;
-  src.base_s = rec_s + 64;
-  src.base_g = reinterpret_cast<const uint32_t *>(rec_g + 64);
-  uint32_t next = start >> 5;
-  uint32_t used = start & 31;
-  const uint32_t w0 = src.word(next), w1 = src.word(next + 1);
-  next += 2;
-  uint32_t hi = __funnelshift_l(w1, w0, used);
-  uint32_t lo = w1 << used;
+  src.at_s = rec_s + 64 + 4 * (start >> 5);
+  src.at_g = reinterpret_cast<const uint32_t *>(rec_g + 64) + (start >> 5);
+  uint32_t pos = start & 31;
+  uint32_t b_hi = src.pop(), b_lo = src.pop();
   const uint32_t my_lut = lane_lut + 4 * lane;
 
-  auto refill = [&]() {   // shift one word in when 32 bits are free
-    if (used & 32u) {
-      const uint32_t w = src.word(next++);
-      used ^= 32u;
-      hi |= __funnelshift_l(w, 0u, used);      // w >> (32 - used mod 32), 0 when used mod 32 == 0
-      lo |= __funnelshift_l(0u, w, used);      // w << (used mod 32)
-    }
+  auto advance = [&]() { src.advance(pos, b_hi, b_lo); };   // shift the next word in once one is consumed
+  auto lookup = [&](uint32_t w) -> uint32_t {   // entry for the code at the top of w: (symbol << 7) | length
+    if (FAST) return lds_u32(mad_u32(w >> (32 - kLaneLutBits), 128u, my_lut));
+    return lds_u16(mad_u32(w >> (32 - kWideLutBits), 2u, wide_lut));
   };
-  auto consume = [&](uint32_t e) {   // shifts use the low 5 bits of e = the code length
-    hi = __funnelshift_l(lo, hi, e);
-    lo = __funnelshift_l(0u, lo, e);
-    used += e;
+  auto pair = [&](uint32_t &ea, uint32_t &eb) {   // two codes from the 32 bits at pos
+    uint32_t w = __funnelshift_l(b_lo, b_hi, pos);
+    ea = lookup(w);
+    w = __funnelshift_l(0u, w, ea);
+    eb = lookup(w);
+    pos += ea + eb;
+    advance();
   };
-  auto take = [&]() -> uint32_t {   // decode one code: returns (symbol << 7) | length
-    uint32_t e = lds_u32(my_lut + ((hi >> (32 - kLaneLutBits)) << 7));
-    consume(e);
-    if (ESCAPE) {
-      if (e == 0) {
-        refill();
-        e = lds_u16(wide_lut + ((hi >> (32 - kWideLutBits)) << 1));
-        consume(e);
-        refill();
-      }
-    }
+  auto quad = [&](uint32_t &ea, uint32_t &eb, uint32_t &ec, uint32_t &ed) {   // four codes of at most 8 bits
+    uint32_t w = __funnelshift_l(b_lo, b_hi, pos);
+    ea = lookup(w);
+    w = __funnelshift_l(0u, w, ea);
+    eb = lookup(w);
+    w = __funnelshift_l(0u, w, eb);
+    ec = lookup(w);
+    w = __funnelshift_l(0u, w, ec);
+    ed = lookup(w);
+    pos += (ea + eb) + (ec + ed);
+    advance();
+  };
+  auto single = [&]() -> uint32_t {
+    const uint32_t e = lookup(__funnelshift_l(b_lo, b_hi, pos));
+    pos += e;
+    advance();
     return e;
   };
 
   constexpr uint32_t kKeep = 0x807F807Fu;   // sign and mantissa bits of two bf16
+  auto group = [&](uint32_t sm_at) -> uint4 {   // the 8 bf16 of one iteration of this lane
+    const uint2 smv = lds_v2(sm_at);
+    uint32_t e0, e1, e2, e3, e4, e5, e6, e7;
+    if (FAST) {
+      quad(e0, e1, e2, e3);
+      quad(e4, e5, e6, e7);
+    } else {
+      pair(e0, e1);
+      pair(e2, e3);
+      pair(e4, e5);
+      pair(e6, e7);
+    }
+    uint4 o;
+    o.x = (__byte_perm(smv.x, 0, 0x1100) & kKeep) | (mad_u32(e1, 65536u, e0) & ~kKeep);
+    o.y = (__byte_perm(smv.x, 0, 0x3322) & kKeep) | (mad_u32(e3, 65536u, e2) & ~kKeep);
+    o.z = (__byte_perm(smv.y, 0, 0x1100) & kKeep) | (mad_u32(e5, 65536u, e4) & ~kKeep);
+    o.w = (__byte_perm(smv.y, 0, 0x3322) & kKeep) | (mad_u32(e7, 65536u, e6) & ~kKeep);
+    return o;
+  };
+
   const uint32_t pieces = (iters + 3) >> 2;
+  if (valid == iters * 256u && (iters & 3u) == 0) {
+    // every group exists and pieces are whole: four unrolled iterations per piece
+    for (uint32_t p = 0; p < pieces; ++p) {
+      const uint32_t sm_s = feed.begin(p);
+      if (sm_s == 0xFFFFFFFFu) return kStatusWaitTimeout;
+      const uint32_t sm_lane = sm_s + lane * 8;
+#pragma unroll
+      for (uint32_t k = 0; k < 4; ++k) sink.group(4 * p + k, lane, group(sm_lane + k * 256));
+      feed.end(p);
+    }
+    return 0;
+  }
   for (uint32_t p = 0; p < pieces; ++p) {
     const uint32_t sm_s = feed.begin(p);
     if (sm_s == 0xFFFFFFFFu) return kStatusWaitTimeout;
     const uint32_t i_end = min(iters, 4 * p + 4);
 #pragma unroll 1
     for (uint32_t i = 4 * p; i < i_end; ++i) {
-      const uint32_t pos = (i * 32 + lane) * 8;
-      if (pos + 8 <= valid) {
-        const uint2 smv = lds_v2(sm_s + ((i & 3) * 32 + lane) * 8);
-        const uint32_t e0 = take(), e1 = take(), e2 = take(), e3 = take();
-        refill();
-        const uint32_t e4 = take(), e5 = take(), e6 = take(), e7 = take();
-        refill();
-        uint4 o;
-        o.x = (__byte_perm(smv.x, 0, 0x1100) & kKeep) | (__byte_perm(e0, e1, 0x5410) & ~kKeep);
-        o.y = (__byte_perm(smv.x, 0, 0x3322) & kKeep) | (__byte_perm(e2, e3, 0x5410) & ~kKeep);
-        o.z = (__byte_perm(smv.y, 0, 0x1100) & kKeep) | (__byte_perm(e4, e5, 0x5410) & ~kKeep);
-        o.w = (__byte_perm(smv.y, 0, 0x3322) & kKeep) | (__byte_perm(e6, e7, 0x5410) & ~kKeep);
-        sink.group(i, lane, o);
-      } else if (pos < valid) {   // the one short group at the end of a linear tensor
-        const uint32_t cnt = valid - pos;
+      const uint32_t pos_e = (i * 32 + lane) * 8;
+      if (pos_e + 8 <= valid) {
+        sink.group(i, lane, group(sm_s + ((i & 3) * 32 + lane) * 8));
+      } else if (pos_e < valid) {   // the one short group at the end of a linear tensor
+        const uint32_t cnt = valid - pos_e;
         for (uint32_t j = 0; j < cnt; ++j) {
-          const uint32_t e = take();
-          refill();
+          const uint32_t e = single();
           const uint32_t at = ((i & 3) * 32 + lane) * 8 + j;
           const uint32_t smb = (lds_u32(sm_s + (at & ~3u)) >> (8 * (at & 3u))) & 0xFFu;
           sink.elem(i, lane, j, (uint16_t)(((smb & 0x80u) << 8) | (e & 0x7F80u) | (smb & 0x7Fu)));

@@ -213,8 +213,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
       break;
     }
     __syncthreads();  // every warp is done with the previous table
-    const bool escape = build_lut<kThreads>(a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) >
-                        (uint32_t)kLaneLutBits;
+    const bool fast = build_lut<kThreads>(a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <=
+                      (uint32_t)kLaneLutBits;
 
     uint32_t g = g0 + warp;
     uint32_t stage = 0;
@@ -246,12 +246,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
           SmFeed feed{pipe, nxt, nxt_issued};
           GlobalSink sink{cur.out, cur.pitch};
           if (cur.staged) {
-            rc = escape ? decode_tile<true, true>(rec_s, nullptr, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
+            rc = fast ? decode_tile<true, true>(rec_s, nullptr, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
                                                   cur.iters, lane, feed, sink)
                         : decode_tile<true, false>(rec_s, nullptr, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
                                                    cur.iters, lane, feed, sink);
           } else {
-            rc = escape ? decode_tile<false, true>(0, cur.rec, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
+            rc = fast ? decode_tile<false, true>(0, cur.rec, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
                                                    cur.iters, lane, feed, sink)
                         : decode_tile<false, false>(0, cur.rec, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
                                                     cur.iters, lane, feed, sink);
