@@ -61,7 +61,9 @@ typedef struct CUstream_st *zipmoe_stream; /* a cudaStream_t; NULL is the defaul
 typedef struct {
   uint32_t chunk_elems;  /* elements per independently decodable chunk (the paper's shard): a multiple
                             of 256, and a multiple of 4096 when larger than 4096.  0 selects 65536.    */
-  uint32_t max_code_len; /* longest Huffman code, 8..12.  0 selects 12.                                 */
+  uint32_t max_code_len; /* longest Huffman code, 8..12.  0 selects 8: the decoder's fastest path (codes of
+                            at most 8 bits resolve in a bank-conflict-free table, four per 32-bit window);
+                            12 gives ~0.06-0.1 bit/element smaller output and decodes ~20 % slower.      */
   uint32_t layout;       /* ZIPMOE_LAYOUT_LINEAR or ZIPMOE_LAYOUT_BLOCKED (needs rows % 16 == 0,
                             cols % 256 == 0, chunk_elems >= 4096)                                       */
   uint32_t n_threads;    /* host threads for the encoder (chunks are independent). 0 selects 1.         */
@@ -129,6 +131,7 @@ typedef struct {
   uint32_t run_first_tile;  /* tile_prefix of that descriptor                                      */
   uint32_t run_end_tile;    /* tile_prefix + n_tiles of the run's last descriptor                  */
   uint32_t tiles_per_chunk; /* tiles in every chunk of the run but possibly the last               */
+  uint32_t reserved[2];     /* zero; pads the descriptor to 80 bytes (five 16-byte loads)          */
 } zipmoe_chunk_desc;
 
 typedef struct {

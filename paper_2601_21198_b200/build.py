@@ -34,7 +34,8 @@ def build(force=False, verbose=False):
     if not force and not needs_build():
         return LIB
     tmp = LIB + ".tmp%d" % os.getpid()
-    cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
+    extra = os.environ.get("ZIPMOE_NVCC_EXTRA", "").split()   # e.g. -DZIPMOE_WARPS=20 when tuning
+    cmd = [_nvcc()] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + \
           [os.path.join(CSRC, s) for s in SOURCES] + ["-o", tmp, "-lcudart"]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

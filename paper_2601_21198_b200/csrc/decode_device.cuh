@@ -11,21 +11,19 @@
 
 namespace zipmoe_dev {
 
-// Two lookup tables per Huffman code:
-//  * the lane table resolves codes of up to 8 bits.  It is indexed by the next
-//    8 code bits and replicated for each of the 32 lanes, entry (v, lane) at
-//    word v*32 + lane, so that lane l only ever touches bank l: the
-//    data-dependent lookups of a warp are free of bank conflicts.  Entry =
-//    (symbol << 7) | length, or 0 when the 8 bits are the prefix of a longer code;
-//  * the wide table (u16 entries, indexed by the next 12 bits) resolves any
-//    code.  It is only built, and only consulted after a 0 entry, for codes
-//    whose longest length exceeds 8.
+// One of two lookup tables per Huffman code, in the same shared-memory region:
+//  * a code whose longest length is at most 8 bits gets the lane table: indexed
+//    by the next 8 code bits and replicated for each of the 32 lanes, entry
+//    (v, lane) at word v*32 + lane, so that lane l only ever touches bank l and
+//    the data-dependent lookups of a warp are free of bank conflicts;
+//  * any other code gets the wide table: u16 entries indexed by the next 12 bits.
+// Entry = (symbol << 7) | length in both.
 constexpr int kLaneLutBits = 8;
 constexpr int kLaneLutBytes = (1 << kLaneLutBits) * 32 * 4;   // 32 KB
 constexpr int kWideLutBits = ZIPMOE_MAX_CODE_LEN;
 constexpr int kWideLutEntries = 1 << kWideLutBits;
 constexpr int kWideLutBytes = kWideLutEntries * 2;            // 8 KB
-constexpr int kLutBytes = kLaneLutBytes + kWideLutBytes;
+constexpr int kLutBytes = kLaneLutBytes;                      // the wide table overlays the lane table
 constexpr int kLutScratchBytes = 256 + 16 * 4 + 8 * 16 * 4 + 256 * 2 + 256 * 4 + 16;
 
 constexpr uint32_t kStatusBadDescriptor = 1;  // a descriptor, offset or table points outside the buffers
@@ -33,8 +31,9 @@ constexpr uint32_t kStatusBadBitCount = 2;    // a tile's lane bit counts overru
 constexpr uint32_t kStatusWaitTimeout = 3;    // an asynchronous copy did not complete in time
 constexpr uint32_t kStatusBadTable = 4;       // code lengths do not form a complete prefix code
 
-constexpr uint32_t kSmPieceBytes = 1024;      // sign+mantissa bytes of four iterations
-constexpr uint32_t kSmPieces = 4;             // pieces of a full tile = slots of a warp's ring
+constexpr uint32_t kPieceIters = 8;           // iterations served by one piece of sign+mantissa bytes
+constexpr uint32_t kSmPieceBytes = kPieceIters * 256;
+constexpr uint32_t kSmPieces = 16 / kPieceIters;   // pieces of a full tile = sign+mantissa slots of a warp
 
 __device__ __forceinline__ void report(uint32_t *status, uint32_t code) {
   if (status) atomicCAS(status, 0u, code);
@@ -111,7 +110,7 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
 // Returns the longest code length (0 for an invalid table).  An incomplete or
 // over-full code is reported and leaves zero entries in the holes: decoding
 // then yields garbage but stays in bounds.
-// Layout of lut_raw: lane table (kLaneLutBytes) then wide table (kWideLutBytes).
+// lut_raw holds the lane table when the result is <= 8, the wide table otherwise.
 template <int THREADS>
 __device__ uint32_t build_lut(const uint8_t *code_len, uint8_t *lut_raw, uint8_t *scratch, uint32_t *status) {
   static_assert(THREADS >= 256 && THREADS % 32 == 0, "one thread per symbol");
@@ -122,7 +121,7 @@ __device__ uint32_t build_lut(const uint8_t *code_len, uint8_t *lut_raw, uint8_t
   uint32_t *s_short = reinterpret_cast<uint32_t *>(s_start + 256);    // [256] lane-table entry of each 8-bit prefix
   uint32_t *s_max = s_short + 256;                                    // [1] longest length
   uint32_t *lane_lut = reinterpret_cast<uint32_t *>(lut_raw);
-  uint16_t *wide_lut = reinterpret_cast<uint16_t *>(lut_raw + kLaneLutBytes);
+  uint16_t *wide_lut = reinterpret_cast<uint16_t *>(lut_raw);
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   uint32_t len = 0;
@@ -186,7 +185,8 @@ __device__ uint32_t build_lut(const uint8_t *code_len, uint8_t *lut_raw, uint8_t
   }
   __syncthreads();
   // replicate the 8-bit table once per lane
-  for (uint32_t k = tid; k < (1u << kLaneLutBits) * 32; k += THREADS) lane_lut[k] = s_short[k >> 5];
+  if (longest <= (uint32_t)kLaneLutBits)
+    for (uint32_t k = tid; k < (1u << kLaneLutBits) * 32; k += THREADS) lane_lut[k] = s_short[k >> 5];
   __syncthreads();
   return longest;
 }
@@ -241,7 +241,8 @@ __device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) 
 
 // Decodes one tile with the 32 lanes of a warp.
 //   record  : in shared memory at rec_s (STAGED) or in global memory at rec_g;
-//   SM bytes: arrive in pieces of four iterations; feed.begin(p) waits for piece
+//   lut     : shared address of the lane table (FAST) or the wide table (!FAST);
+//   SM bytes: arrive in pieces of kPieceIters iterations; feed.begin(p) waits for piece
 //             p and returns its shared address (0xFFFFFFFF when the wait ran
 //             out), feed.end(p) tells that the warp is done reading it;
 //   output  : sink.group(i, lane, v) takes the 8 bf16 of iteration i, lane;
@@ -263,7 +264,7 @@ __device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) 
 // kStatusBadBitCount nothing has been written.
 template <bool STAGED, bool FAST, class Feed, class Sink>
 __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *rec_g, uint32_t rec_bytes,
-                                                uint32_t lane_lut, uint32_t wide_lut, uint32_t valid, uint32_t iters,
+                                                uint32_t lut, uint32_t valid, uint32_t iters,
                                                 uint32_t lane, Feed &feed, Sink &sink) {
   uint32_t my_bits;
   if (STAGED) my_bits = lds_u16(rec_s + 2 * lane);
@@ -283,12 +284,12 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
   src.at_g = reinterpret_cast<const uint32_t *>(rec_g + 64) + (start >> 5);
   uint32_t pos = start & 31;
   uint32_t b_hi = src.pop(), b_lo = src.pop();
-  const uint32_t my_lut = lane_lut + 4 * lane;
+  const uint32_t my_lut = lut + 4 * lane;
 
   auto advance = [&]() { src.advance(pos, b_hi, b_lo); };   // shift the next word in once one is consumed
   auto lookup = [&](uint32_t w) -> uint32_t {   // entry for the code at the top of w: (symbol << 7) | length
     if (FAST) return lds_u32(mad_u32(w >> (32 - kLaneLutBits), 128u, my_lut));
-    return lds_u16(mad_u32(w >> (32 - kWideLutBits), 2u, wide_lut));
+    return lds_u16(mad_u32(w >> (32 - kWideLutBits), 2u, lut));
   };
   auto pair = [&](uint32_t &ea, uint32_t &eb) {   // two codes from the 32 bits at pos
     uint32_t w = __funnelshift_l(b_lo, b_hi, pos);
@@ -338,15 +339,15 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
     return o;
   };
 
-  const uint32_t pieces = (iters + 3) >> 2;
-  if (valid == iters * 256u && (iters & 3u) == 0) {
-    // every group exists and pieces are whole: four unrolled iterations per piece
+  const uint32_t pieces = (iters + kPieceIters - 1) / kPieceIters;
+  if (valid == iters * 256u && (iters % kPieceIters) == 0) {
+    // every group exists and pieces are whole: unrolled iterations, addresses are immediates
     for (uint32_t p = 0; p < pieces; ++p) {
       const uint32_t sm_s = feed.begin(p);
       if (sm_s == 0xFFFFFFFFu) return kStatusWaitTimeout;
       const uint32_t sm_lane = sm_s + lane * 8;
 #pragma unroll
-      for (uint32_t k = 0; k < 4; ++k) sink.group(4 * p + k, lane, group(sm_lane + k * 256));
+      for (uint32_t k = 0; k < kPieceIters; ++k) sink.group(kPieceIters * p + k, lane, group(sm_lane + k * 256));
       feed.end(p);
     }
     return 0;
@@ -354,17 +355,17 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
   for (uint32_t p = 0; p < pieces; ++p) {
     const uint32_t sm_s = feed.begin(p);
     if (sm_s == 0xFFFFFFFFu) return kStatusWaitTimeout;
-    const uint32_t i_end = min(iters, 4 * p + 4);
+    const uint32_t i_end = min(iters, kPieceIters * (p + 1));
 #pragma unroll 1
-    for (uint32_t i = 4 * p; i < i_end; ++i) {
+    for (uint32_t i = kPieceIters * p; i < i_end; ++i) {
       const uint32_t pos_e = (i * 32 + lane) * 8;
       if (pos_e + 8 <= valid) {
-        sink.group(i, lane, group(sm_s + ((i & 3) * 32 + lane) * 8));
+        sink.group(i, lane, group(sm_s + ((i % kPieceIters) * 32 + lane) * 8));
       } else if (pos_e < valid) {   // the one short group at the end of a linear tensor
         const uint32_t cnt = valid - pos_e;
         for (uint32_t j = 0; j < cnt; ++j) {
           const uint32_t e = single();
-          const uint32_t at = ((i & 3) * 32 + lane) * 8 + j;
+          const uint32_t at = ((i % kPieceIters) * 32 + lane) * 8 + j;
           const uint32_t smb = (lds_u32(sm_s + (at & ~3u)) >> (8 * (at & 3u))) & 0xFFu;
           sink.elem(i, lane, j, (uint16_t)(((smb & 0x80u) << 8) | (e & 0x7F80u) | (smb & 0x7Fu)));
         }

@@ -23,13 +23,16 @@
 
 namespace zipmoe_dev {
 
-constexpr int kWarps = 20;                 // warps per CTA, one CTA per SM
+#ifndef ZIPMOE_WARPS
+#define ZIPMOE_WARPS 20
+#endif
+constexpr int kWarps = ZIPMOE_WARPS;                 // warps per CTA, one CTA per SM
 constexpr int kThreads = kWarps * 32;
 constexpr int kPayBuf = 2048;              // record bytes staged per stage; longer records are read from global
 constexpr int kPaySlack = 64;              // readable bytes after a staged record (a lane looks two words ahead)
 constexpr int kPayStage = kPayBuf + kPaySlack;
 constexpr int kPayStages = 2;
-constexpr int kBarsPerWarp = kPayStages + kSmPieces;   // two record stages, four sign+mantissa slots
+constexpr int kBarsPerWarp = kPayStages + kSmPieces;   // two record stages, one barrier per sign+mantissa slot
 constexpr int kWarpBytes = kPayStages * kPayStage + kSmPieces * kSmPieceBytes;
 constexpr int kSmemBytes = kLutBytes + kWarps * kWarpBytes + kWarps * kBarsPerWarp * 8 + kLutScratchBytes;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
@@ -68,20 +71,23 @@ __device__ uint32_t find_chunk(const LaunchArgs &a, uint32_t g) {
   return lo;
 }
 
-__device__ TileWork resolve_tile(const LaunchArgs &a, uint32_t g, uint32_t run_first_chunk, uint32_t run_first_tile,
-                                 uint32_t tiles_per_chunk) {
+static_assert(sizeof(zipmoe_chunk_desc) == 80, "descriptor is read as five 16-byte words");
+
+// Everything the decoder needs about tile t of descriptor c, with every offset
+// checked against the sizes of the buffers the launch was given.
+__device__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_t t) {
   TileWork w;
   w.ok = false;
   w.staged = false;
-  uint32_t rel = g - run_first_tile;
-  uint32_t c = run_first_chunk + rel / tiles_per_chunk, t = rel % tiles_per_chunk;
   if (c >= a.n_chunks) return w;
-  const zipmoe_chunk_desc *d = a.chunks + c;
-  const uint64_t pay_off = __ldg(&d->payload_off), sm_off = __ldg(&d->sm_off), out_off = __ldg(&d->out_off);
-  const uint32_t pitch = __ldg(&d->row_pitch), tpr = __ldg(&d->tiles_per_rowblk), tile0 = __ldg(&d->tile0);
-  const uint32_t m = __ldg(&d->n_tiles), tile_elems = __ldg(&d->tile_elems), last = __ldg(&d->last_tile_elems);
+  const uint4 *d = reinterpret_cast<const uint4 *>(a.chunks + c);
+  const uint4 d0 = __ldg(d), d1 = __ldg(d + 1), d2 = __ldg(d + 2), d3 = __ldg(d + 3);
+  const uint64_t pay_off = ((uint64_t)d0.y << 32) | d0.x, sm_off = ((uint64_t)d0.w << 32) | d0.z;
+  const uint64_t out_off = ((uint64_t)d1.y << 32) | d1.x;
+  const uint32_t pitch = d1.z, tpr = d1.w, tile0 = d2.x, m = d2.y, tile_elems = d2.z, last = d2.w;
+  (void)d3;
   if (t >= m || tpr == 0 || tile_elems == 0 || tile_elems > ZIPMOE_TILE_ELEMS_MAX || (tile_elems & 255) ||
-      last == 0 || last > tile_elems || (pitch & 7) || (pay_off & 15) || (sm_off & 15) || (out_off & 7))
+      last == 0 || last > tile_elems || ((pitch & 7) | (pay_off & 15) | (sm_off & 15) | (out_off & 7)))
     return w;
   if (pay_off + 4ull * (t + 2) > a.payload_bytes) return w;
   const uint32_t *tab = reinterpret_cast<const uint32_t *>(a.payload + pay_off);
@@ -93,10 +99,12 @@ __device__ TileWork resolve_tile(const LaunchArgs &a, uint32_t g, uint32_t run_f
       rec_off + w.rec_bytes > a.payload_bytes)
     return w;
   w.iters = tile_elems >> 8;
-  w.pieces = (w.iters + 3) >> 2;
+  w.pieces = (w.iters + kPieceIters - 1) / kPieceIters;
   w.valid = (t == m - 1) ? last : tile_elems;
   const uint32_t q = tile0 + t;
-  const uint64_t origin = out_off + (uint64_t)(q / tpr) * w.iters * pitch + (uint64_t)(q % tpr) * 256;
+  uint64_t origin = out_off;
+  if (tpr == 1) origin += (uint64_t)q * w.iters * pitch;   // linear layout: no division
+  else origin += (uint64_t)(q / tpr) * w.iters * pitch + (uint64_t)(q % tpr) * 256;
   const uint32_t rows_used = (w.valid + 255) >> 8;
   if (origin + (uint64_t)(rows_used - 1) * pitch + (w.valid - (rows_used - 1) * 256) > a.out_elems) return w;
   const uint64_t sm_tile = sm_off + (uint64_t)t * tile_elems;
@@ -193,7 +201,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
   pipe.phase = 0;
   pipe.pending = 0;
   pipe.lane = lane;
-  const uint32_t lane_lut = smem_addr(lut_raw), wide_lut = lane_lut + kLaneLutBytes;
+  const uint32_t lut = smem_addr(lut_raw);
   if (lane == 0)
     for (int b = 0; b < kBarsPerWarp; ++b) mbar_init(pipe.bar(b), 1);
   fence_barrier_init();
@@ -218,10 +226,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
 
     uint32_t g = g0 + warp;
     uint32_t stage = 0;
+    // descriptor and tile-in-chunk of this warp's next tile, stepped without divisions
+    uint32_t tc = run_first_chunk + (g - run_first_tile) / tpc, tt = (g - run_first_tile) % tpc;
+    auto step = [&]() {
+      tt += kWarps;
+      while (tt >= tpc) {
+        tt -= tpc;
+        ++tc;
+      }
+    };
     TileWork cur;
     cur.ok = false;
     if (g < seg_end && !dead) {
-      cur = resolve_tile(a, g, run_first_chunk, run_first_tile, tpc);
+      cur = resolve_tile(a, tc, tt);
       if (!cur.ok) report(a.status, kStatusBadDescriptor);
       else {
         pipe.load_record(cur, stage);
@@ -234,7 +251,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
       uint32_t nxt_issued = 0;
       const uint32_t g2 = g + kWarps;
       if (g2 < seg_end) {
-        nxt = resolve_tile(a, g2, run_first_chunk, run_first_tile, tpc);
+        step();
+        nxt = resolve_tile(a, tc, tt);
         if (!nxt.ok) report(a.status, kStatusBadDescriptor);
         else pipe.load_record(nxt, stage ^ 1);   // that stage was released by the __syncwarp below
       }
@@ -246,14 +264,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
           SmFeed feed{pipe, nxt, nxt_issued};
           GlobalSink sink{cur.out, cur.pitch};
           if (cur.staged) {
-            rc = fast ? decode_tile<true, true>(rec_s, nullptr, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
+            rc = fast ? decode_tile<true, true>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid,
                                                   cur.iters, lane, feed, sink)
-                        : decode_tile<true, false>(rec_s, nullptr, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
+                        : decode_tile<true, false>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid,
                                                    cur.iters, lane, feed, sink);
           } else {
-            rc = fast ? decode_tile<false, true>(0, cur.rec, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
+            rc = fast ? decode_tile<false, true>(0, cur.rec, cur.rec_bytes, lut, cur.valid,
                                                    cur.iters, lane, feed, sink)
-                        : decode_tile<false, false>(0, cur.rec, cur.rec_bytes, lane_lut, wide_lut, cur.valid,
+                        : decode_tile<false, false>(0, cur.rec, cur.rec_bytes, lut, cur.valid,
                                                     cur.iters, lane, feed, sink);
           }
         }

@@ -53,7 +53,7 @@ struct Opts {
 
 zipmoe_status resolve_opts(const zipmoe_encode_opts *o, Opts *r) {
   r->chunk_elems = (o && o->chunk_elems) ? o->chunk_elems : 65536u;
-  r->max_code_len = (o && o->max_code_len) ? o->max_code_len : ZIPMOE_MAX_CODE_LEN;
+  r->max_code_len = (o && o->max_code_len) ? o->max_code_len : 8u;
   r->layout = o ? o->layout : ZIPMOE_LAYOUT_LINEAR;
   r->n_threads = (o && o->n_threads) ? o->n_threads : 1u;
   if (r->max_code_len < 8 || r->max_code_len > ZIPMOE_MAX_CODE_LEN) return ZIPMOE_ERR_INVALID_ARG;
@@ -461,6 +461,7 @@ zipmoe_status zipmoe_blob_plan(const void *blob_v, uint64_t bytes, uint64_t payl
     d.run_first_tile = tile_base;
     d.run_end_tile = tile_base + g.n_tiles;
     d.tiles_per_chunk = g.tiles_per_chunk;
+    d.reserved[0] = d.reserved[1] = 0;
   }
   return ZIPMOE_OK;
 }

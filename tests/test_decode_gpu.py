@@ -40,10 +40,11 @@ CASES = [
 ]
 
 
+@pytest.mark.parametrize("max_code_len", [8, 12])
 @pytest.mark.parametrize("rows,cols,layout,chunk", CASES)
-def test_decode_matches_oracle_small(zb, rows, cols, layout, chunk):
+def test_decode_matches_oracle_small(zb, rows, cols, layout, chunk, max_code_len):
     x = inputs.gaussian((rows, cols), 0.02, rows * 31 + cols)
-    blob = zb.zipmoe_encode(x, layout=layout, chunk_elems=chunk)
+    blob = zb.zipmoe_encode(x, layout=layout, chunk_elems=chunk, max_code_len=max_code_len)
     _, (got,), _ = gpu_decode(zb, [blob])
     want = codec.decode(blob)
     assert np.array_equal(got, want)
@@ -120,7 +121,7 @@ def test_stress_set_sample(zb):
     for i in range(0, 96):
         x, fam, chunk = inputs.stress_tensor(i, max_elems=1 << 18)
         xs.append(x)
-        blobs.append(zb.zipmoe_encode(x, chunk_elems=chunk))
+        blobs.append(zb.zipmoe_encode(x, chunk_elems=chunk, max_code_len=(8, 12, 10)[i % 3]))
     _, got, _ = gpu_decode(zb, blobs)
     for i, (g, x) in enumerate(zip(got, xs)):
         assert np.array_equal(g, x), i
@@ -205,7 +206,7 @@ def test_small_expert_layer_config_full(zb):
 
 def test_large_expert_layer_config_full(zb):
     from paper_2601_21198_b200 import workloads
-    _check_full_workload(zb, workloads.large_layer(), 8)
+    _check_full_workload(zb, workloads.large_layer(max_code_len=12), 8)
 
 
 def test_large_expert_layer_blocked_layout(zb):
