@@ -171,6 +171,52 @@ zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t n_chunks, 
                             uint64_t payload_bytes, const uint8_t *sm, uint64_t sm_bytes, uint16_t *out_bf16,
                             uint64_t out_elems, uint32_t *status_word, zipmoe_stream stream);
 
+/* ---- fused decode + routed expert FFN (device) ----------------------------- */
+
+/* The compressed experts of one MoE layer.  A HOST struct holding DEVICE
+ * pointers.  Expert e has three tensors, encoded with ZIPMOE_LAYOUT_BLOCKED:
+ * tensor 3e+0 = w1 (gate) [inter, hidden], 3e+1 = w3 (up) [inter, hidden],
+ * 3e+2 = w2 (down) [hidden, inter], all [out, in] row-major before encoding.
+ * `chunks` holds the descriptors zipmoe_blob_plan wrote for the 3E blobs (their
+ * out_off is not used), `tensor_first_chunk[3e+j]` the index of each tensor's
+ * first descriptor, `tables` the code lengths its table_id refers to. */
+typedef struct {
+  uint32_t n_experts, hidden, inter, n_chunks;   /* hidden, inter: multiples of 256; inter/256 a multiple of 4 */
+  const zipmoe_chunk_desc *chunks;               /* device [n_chunks]                                          */
+  const uint32_t *tensor_first_chunk;            /* device [3 * n_experts]                                     */
+  const zipmoe_table *tables;                    /* device [n_tables]                                          */
+  uint32_t n_tables, reserved;
+  const uint8_t *payload;                        /* device, payload_bytes + ZIPMOE_DEVICE_PAD_BYTES            */
+  uint64_t payload_bytes;
+  const uint8_t *sm;                             /* device, sm_bytes + ZIPMOE_DEVICE_PAD_BYTES                 */
+  uint64_t sm_bytes;
+} zipmoe_compressed_experts;
+
+/* Scratch the fused call needs for T tokens with k experts each (routing lists,
+ * fp32 gate/up activations, bf16 intermediate, fp32 partial outputs).  Host only. */
+zipmoe_status zipmoe_ffn_workspace_bytes(uint32_t T, uint32_t k, const zipmoe_compressed_experts *experts,
+                                         uint64_t *workspace_bytes);
+
+/* Expert execution on compressed weights (Section 3.3: the GPU work p_n for the
+ * tokens routed to expert n, here without ever materialising the expert): for
+ * every token t and choice j with e = topk_ids[t, j]:
+ *     g = W1_e x_t,  u = W3_e x_t,  h = bf16(SiLU(g) * u),  y = W2_e h
+ *     out[t] = bf16( sum_j topk_weights[t, j] * y )
+ * bf16 inputs, fp32 accumulation on the tensor cores (tcgen05, accumulators in
+ * tensor memory), weights decoded tile by tile into shared memory.  The paper
+ * does not define the expert network; this is the gated FFN of the models it
+ * evaluates.  Five kernels on `stream`, asynchronous.
+ * device in : tokens [T, hidden] bf16 patterns; topk_ids [T, k] (each token's ids
+ *             distinct); topk_weights [T, k] fp32 or NULL (= 1.0)
+ * device out: out [T, hidden] bf16 patterns; workspace: scratch of at least
+ *             zipmoe_ffn_workspace_bytes, 16-byte aligned; status_word as for
+ *             zipmoe_decode.
+ * Limits: T <= 64, k <= 8, n_experts <= 256 (ZIPMOE_ERR_UNSUPPORTED otherwise). */
+zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32_t T, const int32_t *topk_ids,
+                                       const float *topk_weights, uint32_t k,
+                                       const zipmoe_compressed_experts *experts, uint16_t *out, void *workspace,
+                                       uint64_t workspace_bytes, uint32_t *status_word, zipmoe_stream stream);
+
 /* Name of a status code (static string). */
 const char *zipmoe_status_string(zipmoe_status s);
 

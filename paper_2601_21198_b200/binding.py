@@ -50,6 +50,12 @@ CHUNK_DESC_DTYPE = np.dtype([
 assert CHUNK_DESC_DTYPE.itemsize == 80
 TABLE_BYTES = 256
 
+class CompressedExperts(ctypes.Structure):
+    _fields_ = [("n_experts", _u32), ("hidden", _u32), ("inter", _u32), ("n_chunks", _u32), ("chunks", _vp),
+                ("tensor_first_chunk", _vp), ("tables", _vp), ("n_tables", _u32), ("reserved", _u32),
+                ("payload", _vp), ("payload_bytes", _u64), ("sm", _vp), ("sm_bytes", _u64)]
+
+
 _lib.zipmoe_version.restype = _u32
 _lib.zipmoe_status_string.restype = ctypes.c_char_p
 _lib.zipmoe_status_string.argtypes = [_int]
@@ -59,7 +65,10 @@ _lib.zipmoe_blob_info_get.argtypes = [_vp, _u64, ctypes.POINTER(BlobInfo)]
 _lib.zipmoe_blob_validate.argtypes = [_vp, _u64]
 _lib.zipmoe_blob_plan.argtypes = [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _u32, _vp, _vp]
 _lib.zipmoe_decode.argtypes = [_vp, _u32, _u32, _vp, _u32, _vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp]
-for _f in ("zipmoe_encode_bound", "zipmoe_encode", "zipmoe_blob_info_get", "zipmoe_blob_validate",
+_lib.zipmoe_ffn_workspace_bytes.argtypes = [_u32, _u32, ctypes.POINTER(CompressedExperts), ctypes.POINTER(_u64)]
+_lib.zipmoe_decode_expert_ffn.argtypes = [_vp, _u32, _vp, _vp, _u32, ctypes.POINTER(CompressedExperts), _vp, _vp, _u64,
+                                          _vp, _vp]
+for _f in ("zipmoe_ffn_workspace_bytes", "zipmoe_decode_expert_ffn", "zipmoe_encode_bound", "zipmoe_encode", "zipmoe_blob_info_get", "zipmoe_blob_validate",
            "zipmoe_blob_plan", "zipmoe_decode"):
     getattr(_lib, _f).restype = _int
 
@@ -151,6 +160,20 @@ def zipmoe_decode(chunks, n_chunks, n_tiles, tables, n_tables, payload, payload_
                                                 _ptr(status_word), _ptr(stream)))
 
 
+def zipmoe_ffn_workspace_bytes(T, k, experts):
+    out = _u64(0)
+    _check("zipmoe_ffn_workspace_bytes", _lib.zipmoe_ffn_workspace_bytes(T, k, ctypes.byref(experts), ctypes.byref(out)))
+    return out.value
+
+
+def zipmoe_decode_expert_ffn(tokens, T, topk_ids, topk_weights, k, experts, out, workspace, workspace_bytes,
+                             status_word=None, stream=None):
+    """Pointer arguments are device tensors (or raw device addresses); `experts` is a CompressedExperts."""
+    _check("zipmoe_decode_expert_ffn",
+           _lib.zipmoe_decode_expert_ffn(_ptr(tokens), T, _ptr(topk_ids), _ptr(topk_weights), k, ctypes.byref(experts),
+                                         _ptr(out), _ptr(workspace), workspace_bytes, _ptr(status_word), _ptr(stream)))
+
+
 class DecodePlan:
     """Host-side layout of one decode launch over several blobs: where each
     blob's E-chunk section, SM section and output tensor sit in three contiguous
@@ -225,3 +248,39 @@ class DevicePlan:
         s = torch.cuda.current_stream(self.device) if stream is None else stream
         zipmoe_decode(self.descs, p.n_chunks, p.n_tiles, self.tables, p.n_tables, self.payload, p.payload_bytes,
                       self.sm, p.sm_bytes, out, p.out_elems, self.status, s.cuda_stream)
+
+
+class DeviceExperts:
+    """The compressed experts of one layer on the device: blobs[3*e + j] (j: 0 w1, 1 w3, 2 w2, blocked
+    layout) laid out by DecodePlan, plus the CompressedExperts struct the fused call takes."""
+
+    def __init__(self, blobs, hidden, inter, device="cuda"):
+        import torch
+        assert len(blobs) % 3 == 0
+        self.plan = DecodePlan(blobs)
+        self.dev = self.plan.to_device(device)
+        first = np.cumsum([0] + [inf.n_chunks for inf in self.plan.infos])[:-1].astype(np.uint32)
+        self.tensor_first_chunk = torch.from_numpy(first.view(np.int32).copy()).to(self.dev.device)
+        p, d = self.plan, self.dev
+        self.struct = CompressedExperts(len(blobs) // 3, hidden, inter, p.n_chunks, d.descs.data_ptr(),
+                                        self.tensor_first_chunk.data_ptr(), d.tables.data_ptr(), p.n_tables, 0,
+                                        d.payload.data_ptr(), p.payload_bytes, d.sm.data_ptr(), p.sm_bytes)
+        self.hidden, self.inter = hidden, inter
+        self._ws = {}
+
+    def ffn(self, tokens, topk_ids, topk_weights, out=None, stream=None):
+        """tokens [T, hidden] int16 (bf16 patterns), topk_ids [T, k] int32, topk_weights [T, k] float32 or None:
+        device tensors.  Returns out [T, hidden] int16."""
+        import torch
+        T, k = topk_ids.shape
+        key = (T, k)
+        if key not in self._ws:
+            n = zipmoe_ffn_workspace_bytes(T, k, self.struct)
+            self._ws[key] = torch.empty(n, dtype=torch.uint8, device=self.dev.device)
+        ws = self._ws[key]
+        if out is None:
+            out = torch.empty(T, self.hidden, dtype=torch.int16, device=self.dev.device)
+        s = torch.cuda.current_stream(self.dev.device) if stream is None else stream
+        zipmoe_decode_expert_ffn(tokens, T, topk_ids, topk_weights, k, self.struct, out, ws, ws.numel(),
+                                 self.dev.status, s.cuda_stream)
+        return out

@@ -35,6 +35,10 @@ constexpr uint32_t kPieceIters = 8;           // iterations served by one piece 
 constexpr uint32_t kSmPieceBytes = kPieceIters * 256;
 constexpr uint32_t kSmPieces = 16 / kPieceIters;   // pieces of a full tile = sign+mantissa slots of a warp
 
+constexpr int kPayBuf = 2048;        // record bytes staged in shared memory; longer records are read from global
+constexpr int kPaySlack = 64;        // readable bytes after a staged record (a lane looks two words ahead)
+constexpr int kPayStage = kPayBuf + kPaySlack;
+
 __device__ __forceinline__ void report(uint32_t *status, uint32_t code) {
   if (status) atomicCAS(status, 0u, code);
 }
@@ -105,15 +109,14 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
 // Builds the tables of one canonical Huffman code from its 256 code lengths.
 // Canonical rule: symbols ordered by (length, symbol value) take consecutive
 // code values; the first code of length L+1 is (first code of length L + count
-// of length L) * 2.  Called by all THREADS threads of the CTA (THREADS >= 256);
+// of length L) * 2.  Called by all THREADS threads of the CTA (a multiple of 32, >= 256);
 // the caller synchronises before the call, and the call ends with a barrier.
 // Returns the longest code length (0 for an invalid table).  An incomplete or
 // over-full code is reported and leaves zero entries in the holes: decoding
 // then yields garbage but stays in bounds.
 // lut_raw holds the lane table when the result is <= 8, the wide table otherwise.
-template <int THREADS>
-__device__ uint32_t build_lut(const uint8_t *code_len, uint8_t *lut_raw, uint8_t *scratch, uint32_t *status) {
-  static_assert(THREADS >= 256 && THREADS % 32 == 0, "one thread per symbol");
+__device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint8_t *code_len, uint8_t *lut_raw,
+                                              uint8_t *scratch, uint32_t *status) {
   uint8_t *s_len = scratch;                                           // [256]
   uint32_t *s_first = reinterpret_cast<uint32_t *>(scratch + 256);    // [16] left-aligned 12-bit start of each length
   uint32_t *s_wcnt = s_first + 16;                                    // [8][16] per-warp symbol counts by length
@@ -191,6 +194,88 @@ __device__ uint32_t build_lut(const uint8_t *code_len, uint8_t *lut_raw, uint8_t
   return longest;
 }
 
+// ---- descriptors -> tiles --------------------------------------------------
+struct TileWork {
+  const uint8_t *rec;   // global address of the tile record
+  const uint8_t *sm;    // global address of the tile's sign+mantissa bytes
+  uint16_t *out;        // global address of the tile's first element
+  uint32_t rec_bytes, pitch, valid, iters, pieces;
+  bool ok, staged;
+};
+
+struct LaunchArgs {
+  const zipmoe_chunk_desc *chunks;
+  const zipmoe_table *tables;
+  const uint8_t *payload;
+  const uint8_t *sm;
+  uint16_t *out;
+  uint32_t *status;
+  uint64_t payload_bytes, sm_bytes, out_elems;
+  uint32_t n_chunks, n_tiles, n_tables, tiles_per_cta;
+};
+
+// Which descriptor holds global tile g: exact guess for launches whose chunks
+// all hold the same number of tiles, binary search on tile_prefix otherwise.
+__device__ inline uint32_t find_chunk(const LaunchArgs &a, uint32_t g) {
+  uint32_t c = (uint32_t)(((uint64_t)g * a.n_chunks) / a.n_tiles);
+  if (c >= a.n_chunks) c = a.n_chunks - 1;
+  uint32_t p = __ldg(&a.chunks[c].tile_prefix), m = __ldg(&a.chunks[c].n_tiles);
+  if (g >= p && g - p < m) return c;
+  uint32_t lo = 0, hi = a.n_chunks;  // invariant: prefix[lo] <= g (prefix[0] = 0)
+  while (hi - lo > 1) {
+    uint32_t mid = (lo + hi) >> 1;
+    if (__ldg(&a.chunks[mid].tile_prefix) <= g) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+static_assert(sizeof(zipmoe_chunk_desc) == 80, "descriptor is read as five 16-byte words");
+
+// Everything the decoder needs about tile t of descriptor c, with every offset
+// checked against the sizes of the buffers the launch was given.
+__device__ inline TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_t t) {
+  TileWork w;
+  w.ok = false;
+  w.staged = false;
+  if (c >= a.n_chunks) return w;
+  const uint4 *d = reinterpret_cast<const uint4 *>(a.chunks + c);
+  const uint4 d0 = __ldg(d), d1 = __ldg(d + 1), d2 = __ldg(d + 2), d3 = __ldg(d + 3);
+  const uint64_t pay_off = ((uint64_t)d0.y << 32) | d0.x, sm_off = ((uint64_t)d0.w << 32) | d0.z;
+  const uint64_t out_off = ((uint64_t)d1.y << 32) | d1.x;
+  const uint32_t pitch = d1.z, tpr = d1.w, tile0 = d2.x, m = d2.y, tile_elems = d2.z, last = d2.w;
+  (void)d3;
+  if (t >= m || tpr == 0 || tile_elems == 0 || tile_elems > ZIPMOE_TILE_ELEMS_MAX || (tile_elems & 255) ||
+      last == 0 || last > tile_elems || ((pitch & 7) | (pay_off & 15) | (sm_off & 15) | (out_off & 7)))
+    return w;
+  if (pay_off + 4ull * (t + 2) > a.payload_bytes) return w;
+  const uint32_t *tab = reinterpret_cast<const uint32_t *>(a.payload + pay_off);
+  const uint32_t o0 = __ldg(tab + t), o1 = __ldg(tab + t + 1);
+  const uint64_t rec_off = pay_off + 16ull * o0;
+  if (o1 <= o0) return w;
+  w.rec_bytes = (o1 - o0) * 16u;
+  if (w.rec_bytes < 64 || w.rec_bytes > 64 + tile_elems / 8 * ZIPMOE_MAX_CODE_LEN + 16 ||
+      rec_off + w.rec_bytes > a.payload_bytes)
+    return w;
+  w.iters = tile_elems >> 8;
+  w.pieces = (w.iters + kPieceIters - 1) / kPieceIters;
+  w.valid = (t == m - 1) ? last : tile_elems;
+  const uint32_t q = tile0 + t;
+  uint64_t origin = out_off;
+  if (tpr == 1) origin += (uint64_t)q * w.iters * pitch;   // linear layout: no division
+  else origin += (uint64_t)(q / tpr) * w.iters * pitch + (uint64_t)(q % tpr) * 256;
+  const uint32_t rows_used = (w.valid + 255) >> 8;
+  if (origin + (uint64_t)(rows_used - 1) * pitch + (w.valid - (rows_used - 1) * 256) > a.out_elems) return w;
+  const uint64_t sm_tile = sm_off + (uint64_t)t * tile_elems;
+  if (sm_tile + w.valid > a.sm_bytes) return w;
+  w.rec = a.payload + rec_off;
+  w.sm = a.sm + sm_tile;
+  w.out = a.out + origin;
+  w.pitch = pitch;
+  w.staged = w.rec_bytes <= kPayBuf;
+  w.ok = true;
+  return w;
+}
+
 // ---- tile decoder -------------------------------------------------------------
 template <bool STAGED>
 struct WordSource {
@@ -239,15 +324,7 @@ __device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) 
   return d;
 }
 
-// Decodes one tile with the 32 lanes of a warp.
-//   record  : in shared memory at rec_s (STAGED) or in global memory at rec_g;
-//   lut     : shared address of the lane table (FAST) or the wide table (!FAST);
-//   SM bytes: arrive in pieces of kPieceIters iterations; feed.begin(p) waits for piece
-//             p and returns its shared address (0xFFFFFFFF when the wait ran
-//             out), feed.end(p) tells that the warp is done reading it;
-//   output  : sink.group(i, lane, v) takes the 8 bf16 of iteration i, lane;
-//             sink.elem(i, lane, j, v) one bf16 of the short last group of a
-//             linear tensor.
+// One lane's view of a tile record: its sub-stream of code bits and the table.
 // The code bits of a lane form a stream of u32 words consumed from bit 31 down.
 // The lane keeps two consecutive words of it (b_hi:b_lo) and the bit position
 // `pos` of the next code inside them (pos mod 64 < 32 between batches).  A batch
@@ -260,46 +337,51 @@ __device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) 
 // bits 4..6 are zero, so the low 7 bits of pos stay exact and the rest is
 // ignored (the funnel shifts take the shift amount mod 32).  When bit 5 of pos
 // is set a whole word has been consumed and the next one is shifted in.
-// Returns 0 on success, else a status code (warp-uniform); on
-// kStatusBadBitCount nothing has been written.
-template <bool STAGED, bool FAST, class Feed, class Sink>
-__device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *rec_g, uint32_t rec_bytes,
-                                                uint32_t lut, uint32_t valid, uint32_t iters,
-                                                uint32_t lane, Feed &feed, Sink &sink) {
-  uint32_t my_bits;
-  if (STAGED) my_bits = lds_u16(rec_s + 2 * lane);
-  else my_bits = __ldg(reinterpret_cast<const uint16_t *>(rec_g) + lane);
-  uint32_t incl = my_bits;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-    if (lane >= (uint32_t)d) incl += t;
-  }
-  const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-  if (64u * 8u + total > rec_bytes * 8u) return kStatusBadBitCount;
-  const uint32_t start = incl - my_bits;
-
+template <bool STAGED, bool FAST>
+struct LaneDecoder {
   WordSource<STAGED> src;
-  src.at_s = rec_s + 64 + 4 * (start >> 5);
-  src.at_g = reinterpret_cast<const uint32_t *>(rec_g + 64) + (start >> 5);
-  uint32_t pos = start & 31;
-  uint32_t b_hi = src.pop(), b_lo = src.pop();
-  const uint32_t my_lut = lut + 4 * lane;
+  uint32_t pos, b_hi, b_lo, lut, my_lut;
 
-  auto advance = [&]() { src.advance(pos, b_hi, b_lo); };   // shift the next word in once one is consumed
-  auto lookup = [&](uint32_t w) -> uint32_t {   // entry for the code at the top of w: (symbol << 7) | length
+  // record in shared memory at rec_s (STAGED) or in global memory at rec_g; lut =
+  // shared address of the lane table (FAST) or the wide table (!FAST).  Turns the
+  // record's 32 bit counts into this lane's start by a warp-shuffle prefix sum.
+  // Returns false (warp-uniform) if the counts overrun the record.
+  __device__ __forceinline__ bool init(uint32_t rec_s, const uint8_t *rec_g, uint32_t rec_bytes, uint32_t lut_addr,
+                                       uint32_t lane) {
+    uint32_t my_bits;
+    if (STAGED) my_bits = lds_u16(rec_s + 2 * lane);
+    else my_bits = __ldg(reinterpret_cast<const uint16_t *>(rec_g) + lane);
+    uint32_t incl = my_bits;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+      if (lane >= (uint32_t)d) incl += t;
+    }
+    const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    if (64u * 8u + total > rec_bytes * 8u) return false;
+    const uint32_t start = incl - my_bits;
+    src.at_s = rec_s + 64 + 4 * (start >> 5);
+    src.at_g = reinterpret_cast<const uint32_t *>(rec_g + 64) + (start >> 5);
+    pos = start & 31;
+    b_hi = src.pop();
+    b_lo = src.pop();
+    lut = lut_addr;
+    my_lut = lut_addr + 4 * lane;
+    return true;
+  }
+  __device__ __forceinline__ uint32_t lookup(uint32_t w) const {   // (symbol << 7) | length of the code at the top of w
     if (FAST) return lds_u32(mad_u32(w >> (32 - kLaneLutBits), 128u, my_lut));
     return lds_u16(mad_u32(w >> (32 - kWideLutBits), 2u, lut));
-  };
-  auto pair = [&](uint32_t &ea, uint32_t &eb) {   // two codes from the 32 bits at pos
+  }
+  __device__ __forceinline__ void pair(uint32_t &ea, uint32_t &eb) {   // two codes from the 32 bits at pos
     uint32_t w = __funnelshift_l(b_lo, b_hi, pos);
     ea = lookup(w);
     w = __funnelshift_l(0u, w, ea);
     eb = lookup(w);
     pos += ea + eb;
-    advance();
-  };
-  auto quad = [&](uint32_t &ea, uint32_t &eb, uint32_t &ec, uint32_t &ed) {   // four codes of at most 8 bits
+    src.advance(pos, b_hi, b_lo);
+  }
+  __device__ __forceinline__ void quad(uint32_t &ea, uint32_t &eb, uint32_t &ec, uint32_t &ed) {   // four codes <= 8 bits
     uint32_t w = __funnelshift_l(b_lo, b_hi, pos);
     ea = lookup(w);
     w = __funnelshift_l(0u, w, ea);
@@ -309,18 +391,17 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
     w = __funnelshift_l(0u, w, ec);
     ed = lookup(w);
     pos += (ea + eb) + (ec + ed);
-    advance();
-  };
-  auto single = [&]() -> uint32_t {
+    src.advance(pos, b_hi, b_lo);
+  }
+  __device__ __forceinline__ uint32_t single() {
     const uint32_t e = lookup(__funnelshift_l(b_lo, b_hi, pos));
     pos += e;
-    advance();
+    src.advance(pos, b_hi, b_lo);
     return e;
-  };
-
-  constexpr uint32_t kKeep = 0x807F807Fu;   // sign and mantissa bits of two bf16
-  auto group = [&](uint32_t sm_at) -> uint4 {   // the 8 bf16 of one iteration of this lane
-    const uint2 smv = lds_v2(sm_at);
+  }
+  // the next 8 elements of this lane merged with their sign+mantissa bytes: 8 bf16
+  __device__ __forceinline__ uint4 group(const uint2 smv) {
+    constexpr uint32_t kKeep = 0x807F807Fu;   // sign and mantissa bits of two bf16
     uint32_t e0, e1, e2, e3, e4, e5, e6, e7;
     if (FAST) {
       quad(e0, e1, e2, e3);
@@ -337,7 +418,28 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
     o.z = (__byte_perm(smv.y, 0, 0x1100) & kKeep) | (mad_u32(e5, 65536u, e4) & ~kKeep);
     o.w = (__byte_perm(smv.y, 0, 0x3322) & kKeep) | (mad_u32(e7, 65536u, e6) & ~kKeep);
     return o;
-  };
+  }
+};
+
+// Decodes one tile with the 32 lanes of a warp.
+//   record  : in shared memory at rec_s (STAGED) or in global memory at rec_g;
+//   lut     : shared address of the lane table (FAST) or the wide table (!FAST);
+//   SM bytes: arrive in pieces of kPieceIters iterations; feed.begin(p) waits for piece
+//             p and returns its shared address (0xFFFFFFFF when the wait ran
+//             out), feed.end(p) tells that the warp is done reading it;
+//   output  : sink.group(i, lane, v) takes the 8 bf16 of iteration i, lane;
+//             sink.elem(i, lane, j, v) one bf16 of the short last group of a
+//             linear tensor.
+// Returns 0 on success, else a status code (warp-uniform); on
+// kStatusBadBitCount nothing has been written.
+template <bool STAGED, bool FAST, class Feed, class Sink>
+__device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *rec_g, uint32_t rec_bytes,
+                                                uint32_t lut, uint32_t valid, uint32_t iters,
+                                                uint32_t lane, Feed &feed, Sink &sink) {
+  LaneDecoder<STAGED, FAST> dec;
+  if (!dec.init(rec_s, rec_g, rec_bytes, lut, lane)) return kStatusBadBitCount;
+  auto group = [&](uint32_t sm_at) -> uint4 { return dec.group(lds_v2(sm_at)); };
+  auto single = [&]() -> uint32_t { return dec.single(); };
 
   const uint32_t pieces = (iters + kPieceIters - 1) / kPieceIters;
   if (valid == iters * 256u && (iters % kPieceIters) == 0) {

@@ -28,95 +28,11 @@ namespace zipmoe_dev {
 #endif
 constexpr int kWarps = ZIPMOE_WARPS;                 // warps per CTA, one CTA per SM
 constexpr int kThreads = kWarps * 32;
-constexpr int kPayBuf = 2048;              // record bytes staged per stage; longer records are read from global
-constexpr int kPaySlack = 64;              // readable bytes after a staged record (a lane looks two words ahead)
-constexpr int kPayStage = kPayBuf + kPaySlack;
 constexpr int kPayStages = 2;
 constexpr int kBarsPerWarp = kPayStages + kSmPieces;   // two record stages, one barrier per sign+mantissa slot
 constexpr int kWarpBytes = kPayStages * kPayStage + kSmPieces * kSmPieceBytes;
 constexpr int kSmemBytes = kLutBytes + kWarps * kWarpBytes + kWarps * kBarsPerWarp * 8 + kLutScratchBytes;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
-
-struct TileWork {
-  const uint8_t *rec;   // global address of the tile record
-  const uint8_t *sm;    // global address of the tile's sign+mantissa bytes
-  uint16_t *out;        // global address of the tile's first element
-  uint32_t rec_bytes, pitch, valid, iters, pieces;
-  bool ok, staged;
-};
-
-struct LaunchArgs {
-  const zipmoe_chunk_desc *chunks;
-  const zipmoe_table *tables;
-  const uint8_t *payload;
-  const uint8_t *sm;
-  uint16_t *out;
-  uint32_t *status;
-  uint64_t payload_bytes, sm_bytes, out_elems;
-  uint32_t n_chunks, n_tiles, n_tables, tiles_per_cta;
-};
-
-// Which descriptor holds global tile g: exact guess for launches whose chunks
-// all hold the same number of tiles, binary search on tile_prefix otherwise.
-__device__ uint32_t find_chunk(const LaunchArgs &a, uint32_t g) {
-  uint32_t c = (uint32_t)(((uint64_t)g * a.n_chunks) / a.n_tiles);
-  if (c >= a.n_chunks) c = a.n_chunks - 1;
-  uint32_t p = __ldg(&a.chunks[c].tile_prefix), m = __ldg(&a.chunks[c].n_tiles);
-  if (g >= p && g - p < m) return c;
-  uint32_t lo = 0, hi = a.n_chunks;  // invariant: prefix[lo] <= g (prefix[0] = 0)
-  while (hi - lo > 1) {
-    uint32_t mid = (lo + hi) >> 1;
-    if (__ldg(&a.chunks[mid].tile_prefix) <= g) lo = mid; else hi = mid;
-  }
-  return lo;
-}
-
-static_assert(sizeof(zipmoe_chunk_desc) == 80, "descriptor is read as five 16-byte words");
-
-// Everything the decoder needs about tile t of descriptor c, with every offset
-// checked against the sizes of the buffers the launch was given.
-__device__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_t t) {
-  TileWork w;
-  w.ok = false;
-  w.staged = false;
-  if (c >= a.n_chunks) return w;
-  const uint4 *d = reinterpret_cast<const uint4 *>(a.chunks + c);
-  const uint4 d0 = __ldg(d), d1 = __ldg(d + 1), d2 = __ldg(d + 2), d3 = __ldg(d + 3);
-  const uint64_t pay_off = ((uint64_t)d0.y << 32) | d0.x, sm_off = ((uint64_t)d0.w << 32) | d0.z;
-  const uint64_t out_off = ((uint64_t)d1.y << 32) | d1.x;
-  const uint32_t pitch = d1.z, tpr = d1.w, tile0 = d2.x, m = d2.y, tile_elems = d2.z, last = d2.w;
-  (void)d3;
-  if (t >= m || tpr == 0 || tile_elems == 0 || tile_elems > ZIPMOE_TILE_ELEMS_MAX || (tile_elems & 255) ||
-      last == 0 || last > tile_elems || ((pitch & 7) | (pay_off & 15) | (sm_off & 15) | (out_off & 7)))
-    return w;
-  if (pay_off + 4ull * (t + 2) > a.payload_bytes) return w;
-  const uint32_t *tab = reinterpret_cast<const uint32_t *>(a.payload + pay_off);
-  const uint32_t o0 = __ldg(tab + t), o1 = __ldg(tab + t + 1);
-  const uint64_t rec_off = pay_off + 16ull * o0;
-  if (o1 <= o0) return w;
-  w.rec_bytes = (o1 - o0) * 16u;
-  if (w.rec_bytes < 64 || w.rec_bytes > 64 + tile_elems / 8 * ZIPMOE_MAX_CODE_LEN + 16 ||
-      rec_off + w.rec_bytes > a.payload_bytes)
-    return w;
-  w.iters = tile_elems >> 8;
-  w.pieces = (w.iters + kPieceIters - 1) / kPieceIters;
-  w.valid = (t == m - 1) ? last : tile_elems;
-  const uint32_t q = tile0 + t;
-  uint64_t origin = out_off;
-  if (tpr == 1) origin += (uint64_t)q * w.iters * pitch;   // linear layout: no division
-  else origin += (uint64_t)(q / tpr) * w.iters * pitch + (uint64_t)(q % tpr) * 256;
-  const uint32_t rows_used = (w.valid + 255) >> 8;
-  if (origin + (uint64_t)(rows_used - 1) * pitch + (w.valid - (rows_used - 1) * 256) > a.out_elems) return w;
-  const uint64_t sm_tile = sm_off + (uint64_t)t * tile_elems;
-  if (sm_tile + w.valid > a.sm_bytes) return w;
-  w.rec = a.payload + rec_off;
-  w.sm = a.sm + sm_tile;
-  w.out = a.out + origin;
-  w.pitch = pitch;
-  w.staged = w.rec_bytes <= kPayBuf;
-  w.ok = true;
-  return w;
-}
 
 // Per-warp asynchronous pipeline.  A warp decodes its tiles one after the other;
 // the record of the next tile is copied into the other record stage while the
@@ -221,7 +137,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
       break;
     }
     __syncthreads();  // every warp is done with the previous table
-    const bool fast = build_lut<kThreads>(a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <=
+    const bool fast = build_lut(kThreads, a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <=
                       (uint32_t)kLaneLutBits;
 
     uint32_t g = g0 + warp;

@@ -1,0 +1,543 @@
+// Fused decode + routed expert FFN for sm_100a.  The paper's step is the GPU
+// execution of the tokens routed to an expert once its tensors are recovered
+// (Section 3.3, p_n in the scheduler's notation); here the recovery and the
+// three projections are one pass: every weight tile is decoded from its E-chunk
+// and SM-chunk straight into a shared-memory operand tile and consumed by
+// tcgen05 tensor-core MMAs, so decoded weights never reach global memory.
+//
+// One kernel, ffn_matmul_kernel, computes  Y[slot, row] = sum_k W[row, k] * X[slot, k]
+// for the token slots routed to one expert and a group of 16-row strips of one
+// compressed matrix W (blocked layout: tiles of 16 rows x 256 columns):
+//   * each decode warp owns one strip and walks its tiles along K.  A tile is
+//     decoded in two halves of 8 rows; a half is written as the B operand
+//     (N = 8, K-major, no swizzle) into the warp's own buffer and multiplied at
+//     once by 16 MMAs (M = 64 token rows, K = 16 each) issued by one lane; the
+//     accumulators of a strip are 16 fp32 columns of tensor memory;
+//   * one loader warp stages the activations of the current K step (64 x 256
+//     bf16, the A operand) in a two-stage ring shared by all decode warps;
+//   * at the end four warps read the accumulators back (tcgen05.ld) and store Y.
+// The host wrapper runs it for W1 and W3 (gate, up), applies SiLU(g)*u, runs it
+// for W2 with K split four ways, and combines the experts of every token.
+// Every wait on a barrier is bounded; a wait that runs out is reported through
+// the status word and the kernel still runs to its end and frees tensor memory.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <type_traits>
+
+#include "zipmoe.h"
+#include "decode_device.cuh"
+
+namespace zipmoe_dev {
+
+constexpr int kFfnMaxWarps = 20;                         // decode warps per CTA (plus one loader warp)
+constexpr int kFfnMaxThreads = (kFfnMaxWarps + 1) * 32;
+constexpr uint32_t kBLbo = 144;                          // bytes between the 8x8 cores of a half-tile along K: 128 + 16 of
+                                                         // padding, so that the 32 lanes' 16-byte stores spread over all banks
+constexpr uint32_t kBBufBytes = 32 * kBLbo;              // one half-tile: 8 rows x 256 columns
+constexpr uint32_t kXGroupBytes = 4096;                  // 8 token rows x 256 columns of bf16, cores 128 bytes apart
+constexpr uint32_t kFfnWarpBytes = 2 * kPayStage + kBBufBytes;
+constexpr uint32_t kFfnBarsPerWarp = 3;                  // two record stages, one "MMAs of my buffer are done"
+constexpr uint32_t kDownSplits = 4;                      // K splits of the down projection
+
+struct FfnArgs {
+  LaunchArgs la;                       // descriptors, tables, payload and SM buffers of all expert tensors
+  const uint32_t *tensor_first_chunk;  // [3E] first descriptor of tensor e*3 + {0 w1, 1 w3, 2 w2}
+  const uint32_t *expert_offset;       // [E+1] first slot of each expert
+  const uint32_t *slot_token;          // [S] token of each slot, or null when X rows are the slots themselves
+  const uint16_t *x;                   // bf16 activations, row pitch K
+  float *y;                            // [gridDim.z][S][rows]
+  uint32_t rows, K;                    // the matrix is [rows, K]
+  uint32_t tensor_in_expert;           // 0 (then grid z adds 0 or 1: w1, w3) or 2 (w2, grid z is the K split)
+  uint32_t steps_per_split;            // K steps of 256 per CTA
+  uint32_t n_warps, groups, S;         // decode warps, 8-row groups of token rows held per stage, total slots
+};
+
+__host__ __device__ inline uint32_t ffn_smem_bytes(uint32_t n_warps, uint32_t groups) {
+  return 2 * groups * kXGroupBytes + kLutBytes + kLutScratchBytes + n_warps * kFfnWarpBytes +
+         (n_warps * kFfnBarsPerWarp + 4) * 8 + 16;
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void sts_v4(uint32_t addr, const uint4 &v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// K-major, no-swizzle shared-memory matrix descriptor: 8x8 cores (8 rows of 16
+// bytes, contiguous), `lbo` bytes between cores along K, `sbo` bytes between
+// 8-row groups.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, one CTA
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// the barrier gets one arrival once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const FfnArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const uint32_t NW = a.n_warps, G = a.groups;
+  const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t e = blockIdx.y, z = blockIdx.z;
+  const uint32_t off = __ldg(a.expert_offset + e);
+  uint32_t Te = __ldg(a.expert_offset + e + 1) - off;
+  if (Te == 0) return;   // nothing routed to this expert
+  if (Te > 8 * G) {      // more slots than the stage holds (a token listing the same expert twice)
+    report(a.la.status, kStatusBadDescriptor);
+    Te = 8 * G;
+  }
+
+  uint8_t *x_raw = smem;                                   // [2][G][4096]
+  uint8_t *lut_raw = x_raw + 2 * G * kXGroupBytes;
+  uint8_t *lut_scratch = lut_raw + kLutBytes;
+  uint8_t *warp_raw = lut_scratch + kLutScratchBytes;      // [NW][2 record stages | half-tile buffer]
+  uint64_t *bars = reinterpret_cast<uint64_t *>(warp_raw + NW * kFfnWarpBytes);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NW * kFfnBarsPerWarp + 4);
+  const uint32_t bar0 = smem_addr(bars);
+  const uint32_t x_full = bar0 + 8 * (NW * kFfnBarsPerWarp), x_empty = x_full + 16;   // two barriers each
+  const uint32_t x_addr = smem_addr(x_raw), lut = smem_addr(lut_raw);
+  const bool is_loader = warp == NW;
+
+  const uint32_t n_strips = a.rows >> 4, strip = blockIdx.x * NW + warp;
+  const bool has_strip = !is_loader && strip < n_strips;
+  const uint32_t tensor = e * 3 + a.tensor_in_expert + (a.tensor_in_expert == 2 ? 0 : z);
+  const uint32_t split = a.tensor_in_expert == 2 ? z : 0;
+  const uint32_t steps_total = a.K >> 8;
+  const uint32_t s0 = split * a.steps_per_split, s1 = min(s0 + a.steps_per_split, steps_total);
+
+  uint32_t tmem_cols = 32;
+  while (tmem_cols < 16 * NW) tmem_cols <<= 1;
+  if (tid == 0) {
+    for (uint32_t b = 0; b < NW * kFfnBarsPerWarp; ++b) mbar_init(bar0 + 8 * b, 1);
+    mbar_init(x_full, 1);
+    mbar_init(x_full + 8, 1);
+    mbar_init(x_empty, NW);
+    mbar_init(x_empty + 8, NW);
+  }
+  fence_barrier_init();
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)),
+                 "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  // the tensor: blocked layout, 16 x 256 tiles, one Huffman table
+  const uint32_t c0 = __ldg(a.tensor_first_chunk + tensor);
+  bool ok = c0 < a.la.n_chunks;
+  uint32_t table_id = 0, tpc = 1;
+  if (ok) {
+    const zipmoe_chunk_desc *d = a.la.chunks + c0;
+    table_id = __ldg(&d->table_id);
+    tpc = __ldg(&d->tiles_per_chunk);
+    ok = table_id < a.la.n_tables && tpc != 0 && __ldg(&d->row_pitch) == a.K &&
+         __ldg(&d->tiles_per_rowblk) == steps_total && __ldg(&d->tile_elems) == ZIPMOE_TILE_ELEMS_MAX &&
+         __ldg(&d->tile0) == 0;
+  }
+  if (!ok) report(a.la.status, kStatusBadDescriptor);
+  bool fast = true;
+  if (ok) fast = build_lut(blockDim.x, a.la.tables[table_id].code_len, lut_raw, lut_scratch, a.la.status) <=
+                 (uint32_t)kLaneLutBits;
+  // (build_lut ends with a CTA barrier)
+
+  if (ok && is_loader) {
+    // ---- activations: one K step (8G token rows x 256 columns) per stage ----
+    for (uint32_t s = s0; s < s1; ++s) {
+      const uint32_t b = (s - s0) & 1, n = (s - s0) >> 1;
+      if (n > 0 && !mbar_wait_bounded(x_empty + 8 * b, (n - 1) & 1)) {
+        report(a.la.status, kStatusWaitTimeout);
+        break;
+      }
+      const uint32_t stage = x_addr + b * G * kXGroupBytes;
+      for (uint32_t idx = lane; idx < 8 * G * 32; idx += 32) {
+        const uint32_t rr = idx & 7, g = (idx >> 3) % G, k8 = idx / (8 * G), row = 8 * g + rr;
+        const uint16_t *src = a.x;
+        uint32_t src_bytes = 0;   // rows past the expert's last slot are filled with zeros
+        if (row < Te) {
+          const uint32_t xr = a.slot_token ? __ldg(a.slot_token + off + row) : off + row;
+          src = a.x + (size_t)xr * a.K + s * 256 + k8 * 8;
+          src_bytes = 16;
+        }
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(stage + g * kXGroupBytes + k8 * 128 + rr * 16),
+                     "l"(src), "r"(src_bytes)
+                     : "memory");
+      }
+      asm volatile("cp.async.wait_all;" ::: "memory");
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(x_full + 8 * b);
+    }
+  } else if (ok && !is_loader) {
+    // ---- one strip of 16 rows: decode tile after tile along K, multiply half-tile by half-tile ----
+    const uint32_t my = smem_addr(warp_raw + warp * kFfnWarpBytes);
+    const uint32_t buf = my + 2 * kPayStage;
+    const uint32_t rec_bar = bar0 + 8 * (warp * kFfnBarsPerWarp), mma_bar = rec_bar + 16;
+    const uint32_t d_tmem = tmem + 16 * warp;
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 17) | (4u << 24);   // bf16 x bf16 -> fp32, N=8, M=64
+    uint32_t rec_phase = 0, mma_phase = 0;
+    bool mma_pending = false, failed = !has_strip;
+    LaunchArgs la = a.la;
+    la.out = nullptr;
+    la.out_elems = ~0ull;
+
+    uint32_t tc = 0, tt = 0;
+    TileWork cur;
+    cur.ok = false;
+    uint2 smA[8], smB[8];
+    if (has_strip) {
+      const uint32_t q = strip * steps_total + s0;
+      tc = c0 + q / tpc;
+      tt = q % tpc;
+      cur = resolve_tile(la, tc, tt);
+      if (!cur.ok || cur.valid != ZIPMOE_TILE_ELEMS_MAX) {
+        report(a.la.status, kStatusBadDescriptor);
+        failed = true;
+      } else {
+        if (cur.staged && lane == 0) bulk_load(my, cur.rec, cur.rec_bytes, rec_bar);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) smA[k] = __ldg(reinterpret_cast<const uint2 *>(cur.sm + k * 256) + lane);
+      }
+    }
+    uint32_t stage = 0;
+    for (uint32_t s = s0; s < s1; ++s) {
+      const uint32_t xb = (s - s0) & 1, xn = (s - s0) >> 1;
+      TileWork nxt;
+      nxt.ok = false;
+      if (!failed && s + 1 < s1) {
+        if (++tt >= tpc) {
+          tt = 0;
+          ++tc;
+        }
+        nxt = resolve_tile(la, tc, tt);
+        if (!nxt.ok || nxt.valid != ZIPMOE_TILE_ELEMS_MAX) {
+          report(a.la.status, kStatusBadDescriptor);
+          nxt.ok = false;
+        } else if (nxt.staged && lane == 0) {
+          bulk_load(my + (stage ^ 1) * kPayStage, nxt.rec, nxt.rec_bytes, rec_bar + 8 * (stage ^ 1));
+        }
+      }
+      bool step_done = false;
+      if (!failed) {
+        bool good = true;
+        if (cur.staged) {
+          good = mbar_wait_bounded(rec_bar + 8 * stage, (rec_phase >> stage) & 1);
+          rec_phase ^= 1u << stage;
+          if (!good) report(a.la.status, kStatusWaitTimeout);
+        }
+        // both halves of the tile, for every combination of record location and table kind
+        auto run = [&](auto staged_c, auto fast_c) -> bool {
+          LaneDecoder<decltype(staged_c)::value, decltype(fast_c)::value> dec;
+          if (!dec.init(my + stage * kPayStage, cur.rec, cur.rec_bytes, lut, lane)) {
+            report(a.la.status, kStatusBadBitCount);
+            return false;
+          }
+#pragma unroll
+          for (int k = 0; k < 8; ++k) smB[k] = __ldg(reinterpret_cast<const uint2 *>(cur.sm + (8 + k) * 256) + lane);
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            if (mma_pending) {   // the MMAs that read the buffer must be done before it is overwritten
+              if (!mbar_wait_bounded(mma_bar, mma_phase)) {
+                report(a.la.status, kStatusWaitTimeout);
+                return false;
+              }
+              mma_phase ^= 1;
+              mma_pending = false;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) sts_v4(buf + lane * kBLbo + k * 16, dec.group(half ? smB[k] : smA[k]));
+            if (half == 0 && nxt.ok) {
+#pragma unroll
+              for (int k = 0; k < 8; ++k) smA[k] = __ldg(reinterpret_cast<const uint2 *>(nxt.sm + k * 256) + lane);
+            }
+            fence_async_smem();   // the stores above must be visible to the tensor core's reads
+            __syncwarp();
+            if (half == 0 && !mbar_wait_bounded(x_full + 8 * xb, xn & 1)) {
+              report(a.la.status, kStatusWaitTimeout);
+              return false;
+            }
+            if (lane == 0) {
+              tc_fence_after();
+              const uint32_t xs = x_addr + xb * G * kXGroupBytes;
+#pragma unroll
+              for (uint32_t j = 0; j < 16; ++j)
+                mma_bf16(d_tmem + 8 * half, smem_desc(xs + j * 256, 128, kXGroupBytes),
+                         smem_desc(buf + j * 2 * kBLbo, kBLbo, kBBufBytes), idesc, (s > s0 || j > 0) ? 1u : 0u);
+              mma_commit(mma_bar);
+              if (half == 1) mma_commit(x_empty + 8 * xb);
+            }
+            mma_pending = true;
+            __syncwarp();
+          }
+          return true;
+        };
+        if (good) {
+          if (cur.staged) good = fast ? run(std::true_type{}, std::true_type{}) : run(std::true_type{}, std::false_type{});
+          else good = fast ? run(std::false_type{}, std::true_type{}) : run(std::false_type{}, std::false_type{});
+        }
+        if (good) step_done = true;
+        else failed = true;
+        if (!nxt.ok && s + 1 < s1) failed = true;
+      }
+      if (!step_done) {
+        // keep the stage ring moving for the other warps: wait for the step, then release it
+        mbar_wait_bounded(x_full + 8 * xb, xn & 1);
+        if (lane == 0) mbar_arrive(x_empty + 8 * xb);
+      }
+      cur = nxt;
+      stage ^= 1;
+    }
+    if (mma_pending && !mbar_wait_bounded(mma_bar, mma_phase)) report(a.la.status, kStatusWaitTimeout);
+  }
+
+  // ---- accumulators -> Y ----
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (ok && warp < 4) {
+    // a warp reads the 32 tensor-memory lanes of its quarter; with M = 64, D row 16q + i is lane 32q + i (i < 16)
+    const uint32_t row = 16 * warp + lane;
+    float *yrow = a.y + ((size_t)z * a.S + off + row) * a.rows;
+    for (uint32_t w = 0; w < NW; ++w) {
+      const uint32_t st = blockIdx.x * NW + w;
+      if (st >= n_strips) break;
+      uint32_t r[16];
+      const uint32_t taddr = tmem + ((32 * warp) << 16) + 16 * w;
+      asm volatile(
+          "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+          : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+            "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+          : "r"(taddr)
+          : "memory");
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (lane < 16 && row < Te) {
+        float4 *dst = reinterpret_cast<float4 *>(yrow + 16 * st);
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+          dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                               __uint_as_float(r[4 * v + 3]));
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
+}
+
+// ---- routing: slots grouped by expert ---------------------------------------------------
+// slot_of[t*k + j] = slot of the j-th choice of token t (0xFFFFFFFF for an id out of range);
+// slots of an expert are consecutive, in token order.
+__global__ void route_kernel(const int32_t *topk_ids, uint32_t S, uint32_t k, uint32_t E, uint32_t max_per_expert,
+                             uint32_t *expert_offset, uint32_t *slot_token, uint32_t *slot_of, uint32_t *status) {
+  extern __shared__ uint32_t cnt[];   // [E] counts, then [E] cursors
+  uint32_t *cursor = cnt + E;
+  for (uint32_t i = threadIdx.x; i < 2 * E; i += blockDim.x) cnt[i] = 0;
+  __syncthreads();
+  for (uint32_t i = threadIdx.x; i < S; i += blockDim.x) {
+    const int32_t ex = topk_ids[i];
+    if (ex >= 0 && (uint32_t)ex < E) atomicAdd(&cnt[ex], 1u);
+    else report(status, kStatusBadDescriptor);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t run = 0;
+    for (uint32_t x = 0; x < E; ++x) {
+      expert_offset[x] = run;
+      cursor[x] = run;
+      if (cnt[x] > max_per_expert) report(status, kStatusBadDescriptor);
+      run += cnt[x];
+    }
+    expert_offset[E] = run;
+    for (uint32_t i = 0; i < S; ++i) {
+      const int32_t ex = topk_ids[i];
+      uint32_t slot = 0xFFFFFFFFu;
+      if (ex >= 0 && (uint32_t)ex < E) {
+        slot = cursor[ex]++;
+        slot_token[slot] = i / k;
+      }
+      slot_of[i] = slot;
+    }
+  }
+}
+
+// h = bf16(SiLU(g) * u), g and u fp32 [S][I]
+__global__ void swiglu_kernel(const float *g, const float *u, uint16_t *h, uint64_t n) {
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    const float gv = g[i];
+    const float hv = gv / (1.0f + __expf(-gv)) * u[i];
+    h[i] = __bfloat16_as_ushort(__float2bfloat16_rn(hv));
+  }
+}
+
+// out[t] = bf16( sum_j w[t,j] * sum_split y[split][slot_of[t,j]] )
+__global__ void combine_kernel(const float *y, const uint32_t *slot_of, const float *topk_weights, uint32_t T,
+                               uint32_t k, uint32_t S, uint32_t H, uint32_t splits, uint16_t *out) {
+  const uint32_t t = blockIdx.y;
+  for (uint32_t c = blockIdx.x * blockDim.x + threadIdx.x; c < H; c += gridDim.x * blockDim.x) {
+    float acc = 0.f;
+    for (uint32_t j = 0; j < k; ++j) {
+      const uint32_t slot = slot_of[t * k + j];
+      if (slot == 0xFFFFFFFFu) continue;
+      float v = 0.f;
+      for (uint32_t sp = 0; sp < splits; ++sp) v += y[((size_t)sp * S + slot) * H + c];
+      acc += (topk_weights ? topk_weights[t * k + j] : 1.0f) * v;
+    }
+    out[(size_t)t * H + c] = __bfloat16_as_ushort(__float2bfloat16_rn(acc));
+  }
+}
+
+}  // namespace zipmoe_dev
+
+namespace {
+
+struct FfnPlan {
+  uint32_t S, groups, n_warps, smem;
+  uint64_t off_offsets, off_slot_token, off_slot_of, off_gu, off_h, off_y, total;
+};
+
+zipmoe_status make_plan(uint32_t T, uint32_t k, const zipmoe_compressed_experts *ex, FfnPlan *p) {
+  if (!ex || T == 0 || k == 0 || T > 64 || k > 8 || ex->n_experts == 0 || ex->n_experts > 256) return ZIPMOE_ERR_UNSUPPORTED;
+  if (ex->hidden == 0 || ex->inter == 0 || ex->hidden % 256 || ex->inter % 256) return ZIPMOE_ERR_UNSUPPORTED;
+  if ((ex->inter / 256) % zipmoe_dev::kDownSplits) return ZIPMOE_ERR_UNSUPPORTED;
+  p->S = T * k;
+  p->groups = (T + 7) / 8;
+  uint32_t nw = zipmoe_dev::kFfnMaxWarps;
+  while (nw > 8 && zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) --nw;   // the table builder needs 256 threads
+  if (zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) return ZIPMOE_ERR_UNSUPPORTED;
+  p->n_warps = nw;
+  p->smem = zipmoe_dev::ffn_smem_bytes(nw, p->groups);
+  auto up = [](uint64_t v) { return (v + 255) / 256 * 256; };
+  uint64_t at = 0;
+  p->off_offsets = at; at = up(at + 4ull * (ex->n_experts + 1));
+  p->off_slot_token = at; at = up(at + 4ull * p->S);
+  p->off_slot_of = at; at = up(at + 4ull * p->S);
+  p->off_gu = at; at = up(at + 2ull * p->S * ex->inter * 4);
+  p->off_h = at; at = up(at + (uint64_t)p->S * ex->inter * 2);
+  p->off_y = at; at = up(at + (uint64_t)zipmoe_dev::kDownSplits * p->S * ex->hidden * 4);
+  p->total = at;
+  return ZIPMOE_OK;
+}
+
+bool g_ffn_ready[64];
+
+}  // namespace
+
+extern "C" zipmoe_status zipmoe_ffn_workspace_bytes(uint32_t T, uint32_t k, const zipmoe_compressed_experts *experts,
+                                                    uint64_t *workspace_bytes) {
+  if (!workspace_bytes) return ZIPMOE_ERR_INVALID_ARG;
+  FfnPlan p;
+  zipmoe_status rc = make_plan(T, k, experts, &p);
+  if (rc != ZIPMOE_OK) return rc;
+  *workspace_bytes = p.total;
+  return ZIPMOE_OK;
+}
+
+extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32_t T, const int32_t *topk_ids,
+                                                  const float *topk_weights, uint32_t k,
+                                                  const zipmoe_compressed_experts *ex, uint16_t *out, void *workspace,
+                                                  uint64_t workspace_bytes, uint32_t *status_word,
+                                                  zipmoe_stream stream_) {
+  using namespace zipmoe_dev;
+  FfnPlan p;
+  zipmoe_status rc = make_plan(T, k, ex, &p);
+  if (rc != ZIPMOE_OK) return rc;
+  if (!tokens || !topk_ids || !out || !workspace || !ex->chunks || !ex->tensor_first_chunk || !ex->tables ||
+      !ex->payload || !ex->sm || ex->n_chunks == 0 || ex->n_tables == 0)
+    return ZIPMOE_ERR_INVALID_ARG;
+  if (workspace_bytes < p.total) return ZIPMOE_ERR_BUFFER_TOO_SMALL;
+  if ((reinterpret_cast<uintptr_t>(tokens) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(workspace) |
+       reinterpret_cast<uintptr_t>(ex->payload) | reinterpret_cast<uintptr_t>(ex->sm) |
+       reinterpret_cast<uintptr_t>(ex->chunks)) & 15)
+    return ZIPMOE_ERR_INVALID_ARG;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ZIPMOE_ERR_CUDA;
+  if (!g_ffn_ready[dev]) {
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ZIPMOE_ERR_CUDA;
+    if (major != 10) return ZIPMOE_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(ffn_matmul_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+      return ZIPMOE_ERR_CUDA;
+    g_ffn_ready[dev] = true;
+  }
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  uint8_t *ws = static_cast<uint8_t *>(workspace);
+  uint32_t *expert_offset = reinterpret_cast<uint32_t *>(ws + p.off_offsets);
+  uint32_t *slot_token = reinterpret_cast<uint32_t *>(ws + p.off_slot_token);
+  uint32_t *slot_of = reinterpret_cast<uint32_t *>(ws + p.off_slot_of);
+  float *gu = reinterpret_cast<float *>(ws + p.off_gu);
+  uint16_t *h = reinterpret_cast<uint16_t *>(ws + p.off_h);
+  float *y = reinterpret_cast<float *>(ws + p.off_y);
+  const uint32_t E = ex->n_experts, H = ex->hidden, I = ex->inter, S = p.S;
+
+  route_kernel<<<1, 256, 2 * E * sizeof(uint32_t), stream>>>(topk_ids, S, k, E, 8 * p.groups, expert_offset, slot_token,
+                                                             slot_of, status_word);
+
+  FfnArgs a;
+  a.la.chunks = ex->chunks;
+  a.la.tables = ex->tables;
+  a.la.payload = ex->payload;
+  a.la.sm = ex->sm;
+  a.la.out = nullptr;
+  a.la.status = status_word;
+  a.la.payload_bytes = ex->payload_bytes;
+  a.la.sm_bytes = ex->sm_bytes;
+  a.la.out_elems = ~0ull;
+  a.la.n_chunks = ex->n_chunks;
+  a.la.n_tiles = 0;
+  a.la.n_tables = ex->n_tables;
+  a.la.tiles_per_cta = 0;
+  a.tensor_first_chunk = ex->tensor_first_chunk;
+  a.expert_offset = expert_offset;
+  a.n_warps = p.n_warps;
+  a.groups = p.groups;
+  a.S = S;
+  const uint32_t threads = (p.n_warps + 1) * 32;
+
+  // gate and up: Y[z] = W_{1,3} X over the full K = H
+  a.slot_token = slot_token;
+  a.x = tokens;
+  a.y = gu;
+  a.rows = I;
+  a.K = H;
+  a.tensor_in_expert = 0;
+  a.steps_per_split = H / 256;
+  dim3 grid_gu((I / 16 + p.n_warps - 1) / p.n_warps, E, 2);
+  ffn_matmul_kernel<<<grid_gu, threads, p.smem, stream>>>(a);
+
+  const uint64_t n_h = (uint64_t)S * I;
+  const unsigned act_blocks = (unsigned)((n_h + 1023) / 1024 < 592 ? (n_h + 1023) / 1024 : 592);
+  swiglu_kernel<<<act_blocks, 256, 0, stream>>>(gu, gu + n_h, h, n_h);
+
+  // down: partial Y[split] = W_2[:, split] H[:, split]
+  a.slot_token = nullptr;
+  a.x = h;
+  a.y = y;
+  a.rows = H;
+  a.K = I;
+  a.tensor_in_expert = 2;
+  a.steps_per_split = I / 256 / kDownSplits;
+  dim3 grid_dn((H / 16 + p.n_warps - 1) / p.n_warps, E, kDownSplits);
+  ffn_matmul_kernel<<<grid_dn, threads, p.smem, stream>>>(a);
+
+  combine_kernel<<<dim3((H + 255) / 256, T), 256, 0, stream>>>(y, slot_of, topk_weights, T, k, S, H, kDownSplits, out);
+  return cudaGetLastError() == cudaSuccess ? ZIPMOE_OK : ZIPMOE_ERR_CUDA;
+}

@@ -1,0 +1,134 @@
+"""GPU parity of the fused decode + expert FFN (zipmoe_decode_expert_ffn through
+the C ABI) against the CPU oracle's FFN on the oracle's decoded weights.
+Tolerance (bf16 inputs, fp32 accumulation): every element within 1e-2 of the
+oracle -- or within one bf16 spacing of it where that spacing is larger (an
+output of magnitude >= 2 is 2^-6 = 0.0156 away from its neighbours, so a single
+rounding flip of the final bf16 already exceeds 1e-2) -- and relative Frobenius
+error <= 2e-2."""
+import numpy as np
+import pytest
+
+from oracle import codec, ffn as offn
+from paper_2601_21198_b200 import build, inputs
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, REL_FRO = 1e-2, 2e-2
+
+
+@pytest.fixture(scope="module")
+def zb():
+    build.build()
+    from paper_2601_21198_b200 import binding
+    return binding
+
+
+def make_layer(zb, E, H, I, seed, std=0.03, max_code_len=0):
+    ws, blobs = [], []
+    for e in range(E):
+        for j in range(3):
+            shape = (I, H) if j < 2 else (H, I)
+            w = inputs.gaussian(shape, std * (1 + 0.3 * ((e + j) % 3)), seed + 3 * e + j)
+            ws.append(w)
+            blobs.append(zb.zipmoe_encode(w, layout=zb.LAYOUT_BLOCKED, chunk_elems=65536, max_code_len=max_code_len))
+    return ws, blobs
+
+
+def oracle_out(ws_decoded, tok, ids, wts, rows):
+    w1 = {e: ws_decoded[3 * e] for e in set(ids[rows].ravel().tolist())}
+    w3 = {e: ws_decoded[3 * e + 1] for e in w1}
+    w2 = {e: ws_decoded[3 * e + 2] for e in w1}
+    out, y = offn.expert_ffn(tok[rows], ids[rows], None if wts is None else wts[rows], w1, w3, w2)
+    return offn.bf16_to_f64(out), y
+
+
+def check(got_bits, want, label):
+    got = offn.bf16_to_f64(got_bits)
+    err = np.abs(got - want)
+    bound = np.maximum(MAX_ABS, np.abs(want) * 2.0 ** -7)      # one bf16 spacing is at most 2^-7 |x|
+    rel = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30)
+    assert (err <= bound).all() and rel <= REL_FRO, (label, err.max(), rel)
+
+
+@pytest.mark.parametrize("T", [1, 5, 16, 64])
+@pytest.mark.parametrize("max_code_len", [8, 12])
+def test_small_experts_match_oracle(zb, T, max_code_len):
+    import torch
+    E, H, I, k = 4, 512, 1024, 2
+    ws, blobs = make_layer(zb, E, H, I, seed=50, max_code_len=max_code_len)
+    decoded = [codec.decode(b).reshape(w.shape) for b, w in zip(blobs, ws)]
+    for d, w in zip(decoded, ws):
+        assert np.array_equal(d, w)
+    ex = zb.DeviceExperts(blobs, H, I)
+    tok = inputs.tokens(T, H, seed=T)
+    ids, wts = inputs.routing(T, n_experts=E, k=k, seed=T)
+    for weights in (wts, None):
+        out = ex.ffn(torch.from_numpy(tok.view(np.int16)).cuda(), torch.from_numpy(ids).cuda(),
+                     None if weights is None else torch.from_numpy(weights).cuda())
+        torch.cuda.synchronize()
+        assert int(ex.dev.status.item()) == 0
+        want, _ = oracle_out(decoded, tok, ids, weights, np.arange(T))
+        check(out.cpu().numpy().view(np.uint16), want, (T, max_code_len, weights is None))
+
+
+def test_single_expert_k1_and_unused_experts(zb):
+    import torch
+    E, H, I = 3, 256, 1024
+    ws, blobs = make_layer(zb, E, H, I, seed=80)
+    ex = zb.DeviceExperts(blobs, H, I)
+    tok = inputs.tokens(7, H, seed=3)
+    ids = np.full((7, 1), 1, np.int32)            # every token to expert 1; experts 0 and 2 idle
+    out = ex.ffn(torch.from_numpy(tok.view(np.int16)).cuda(), torch.from_numpy(ids).cuda(), None)
+    torch.cuda.synchronize()
+    assert int(ex.dev.status.item()) == 0
+    want, _ = oracle_out(ws, tok, ids, None, np.arange(7))
+    check(out.cpu().numpy().view(np.uint16), want, "k1")
+
+
+def test_bad_arguments(zb):
+    import torch
+    E, H, I = 1, 256, 1024
+    ws, blobs = make_layer(zb, E, H, I, seed=90)
+    ex = zb.DeviceExperts(blobs, H, I)
+    tok = torch.zeros(65, H, dtype=torch.int16, device="cuda")
+    ids = torch.zeros(65, 1, dtype=torch.int32, device="cuda")
+    with pytest.raises(zb.ZipMoEError):
+        ex.ffn(tok, ids, None)                     # T > 64
+    bad = zb.CompressedExperts.from_buffer_copy(ex.struct)
+    bad.inter = 1000
+    with pytest.raises(zb.ZipMoEError):
+        zb.zipmoe_ffn_workspace_bytes(4, 2, bad)   # inter not a multiple of 256
+
+
+@pytest.mark.parametrize("T", [1, 16, 64])
+def test_large_experts_config(zb, T):
+    """8 experts of 4096 -> 14336 -> 4096 (256K-element chunks), top-2 of 8 with Zipf(1.2) popularity.
+    The oracle FFN is evaluated on a sample of the tokens (tokens are independent)."""
+    import torch
+    from paper_2601_21198_b200 import workloads
+    w = _large_layer(workloads)
+    ex = _large_experts(zb, w)
+    tok = inputs.tokens(T, 4096, seed=100 + T)
+    ids, wts = inputs.routing(T, n_experts=8, k=2, seed=T)
+    out = ex.ffn(torch.from_numpy(tok.view(np.int16)).cuda(), torch.from_numpy(ids).cuda(),
+                 torch.from_numpy(wts).cuda())
+    torch.cuda.synchronize()
+    assert int(ex.dev.status.item()) == 0
+    rows = np.arange(T) if T <= 4 else np.random.default_rng(T).choice(T, 4, replace=False)
+    want, _ = oracle_out(w.originals, tok, ids, wts, rows)
+    check(out.cpu().numpy().view(np.uint16)[rows], want, ("large", T))
+
+
+_cache = {}
+
+
+def _large_layer(workloads):
+    if "w" not in _cache:
+        _cache["w"] = workloads.large_layer(layout=1)
+    return _cache["w"]
+
+
+def _large_experts(zb, w):
+    if "ex" not in _cache:
+        _cache["ex"] = zb.DeviceExperts(w.blobs, 4096, 14336)
+    return _cache["ex"]
