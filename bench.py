@@ -159,6 +159,85 @@ class ClockSampler(threading.Thread):
                 "samples": len(inside), "window": window}
 
 
+# ----------------------------------------------------------------------------- fused expert FFN
+def bench_ffn(dev, iters=20, cpu_tokens=2):
+    """Fused decode + expert SwiGLU FFN on 8 experts of 4096 -> 14336 -> 4096 (top-2 of 8, Zipf(1.2)
+    popularity) for T = 1, 16, 64 tokens, against decode-then-GEMM: zipmoe_decode of the routed experts
+    into bf16 followed by torch matmuls on the same stream.  Also times the CPU oracle's FFN on a few tokens."""
+    import torch
+    from paper_2601_21198_b200 import binding, inputs, workloads
+    w = workloads.large_layer(layout=binding.LAYOUT_BLOCKED, keep_originals=True)
+    ex = binding.DeviceExperts(w.blobs, 4096, 14336, dev)
+    per_expert = [binding.DecodePlan(w.blobs[3 * e: 3 * e + 3]).to_device(dev) for e in range(8)]
+    dense = [p.new_output() for p in per_expert]
+    expert_bytes = [sum(i.payload_bytes + i.n_elems for i in p.plan.infos) for p in per_expert]
+    stream = torch.cuda.current_stream(dev)
+    out = {}
+    for T in (1, 16, 64):
+        tok = inputs.tokens(T, 4096, seed=100 + T)
+        ids, wts = inputs.routing(T, n_experts=8, k=2, seed=T)
+        d_tok = torch.from_numpy(tok.view(np.int16)).to(dev)
+        d_ids = torch.from_numpy(ids).to(dev)
+        d_wts = torch.from_numpy(wts).to(dev)
+        active = sorted(set(ids.ravel().tolist()))
+        y = ex.ffn(d_tok, d_ids, d_wts)
+
+        def fused():
+            ex.ffn(d_tok, d_ids, d_wts, out=y)
+
+        x_bf = d_tok.view(torch.bfloat16)
+        sel = {e: (torch.from_numpy(np.nonzero(ids == e)[0]).to(dev), torch.from_numpy(wts[ids == e]).to(dev))
+               for e in active}
+        acc = torch.zeros(T, 4096, dtype=torch.float32, device=dev)
+
+        def unfused():
+            acc.zero_()
+            for e in active:
+                per_expert[e].decode(dense[e])
+                p = per_expert[e].plan
+                w1 = p.tensor_slice(dense[e], 0).view(torch.bfloat16).view(14336, 4096)
+                w3 = p.tensor_slice(dense[e], 1).view(torch.bfloat16).view(14336, 4096)
+                w2 = p.tensor_slice(dense[e], 2).view(torch.bfloat16).view(4096, 14336)
+                rows, wt = sel[e]
+                xe = x_bf[rows]
+                h = torch.nn.functional.silu(xe @ w1.T) * (xe @ w3.T)
+                acc.index_add_(0, rows, (h @ w2.T).float() * wt[:, None])
+            return acc.to(torch.bfloat16)
+
+        def timed(fn):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize(dev)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(iters):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize(dev)
+            return a.elapsed_time(b) / iters * 1e3      # microseconds
+
+        ref = unfused().float()
+        diff = (y.view(torch.bfloat16).float() - ref).abs().max().item()
+        us_f, us_u = timed(fused), timed(unfused)
+        nbytes = sum(expert_bytes[e] for e in active)
+        out["T%d" % T] = {"us": us_f, "tokens_per_s": T / us_f * 1e6, "active_experts": len(active),
+                          "compressed_gbs": nbytes / us_f / 1e3, "decode_then_gemm_us": us_u,
+                          "speedup_vs_decode_then_gemm": us_u / us_f, "max_abs_diff_vs_decode_then_gemm": diff,
+                          "status": int(ex.dev.status.item())}
+    # CPU oracle FFN on a few tokens of the T = 16 case (fp64 numpy)
+    from oracle import ffn as offn
+    tok = inputs.tokens(16, 4096, seed=116)
+    ids, wts = inputs.routing(16, n_experts=8, k=2, seed=16)
+    t0 = time.perf_counter()
+    offn.expert_ffn(tok[:cpu_tokens], ids[:cpu_tokens], wts[:cpu_tokens], {e: w.originals[3 * e] for e in range(8)},
+                    {e: w.originals[3 * e + 1] for e in range(8)}, {e: w.originals[3 * e + 2] for e in range(8)})
+    dt = time.perf_counter() - t0
+    out["cpu_oracle"] = {"tokens_per_s": cpu_tokens / dt, "sample": "%d tokens of the T=16 case, fp64 numpy" % cpu_tokens,
+                         "cores": os.cpu_count() or 1}
+    out["config"] = "8 experts 4096->14336->4096 bf16 (blocked layout, 256K-element chunks), top-2, Zipf(1.2)"
+    return out
+
+
 # ----------------------------------------------------------------------------- GPU leg
 def run_ours(args):
     import torch
@@ -276,6 +355,10 @@ def run_ours(args):
                          "kernel": "zipmoe_dev::decode_kernel", "launch_ms": per_launch_s * 1e3},
             "verified_bit_exact": verified,
         }
+        if world == 1 and not args.no_ffn:
+            del dplan, out, h_pay, h_sm, h_out
+            torch.cuda.empty_cache()
+            line["ffn"] = bench_ffn(dev)
         if world == 1:
             cores = os.cpu_count() or 1
             count = int(max(cores, 20.0 / oracle_seconds_per_tensor(w.blobs[0])))   # ~20 s of CPU work
@@ -305,6 +388,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="small_layer", choices=["small_layer", "large_layer", "single_matrix"])
+    ap.add_argument("--no-ffn", action="store_true", help="skip the fused expert-FFN section of the report")
     ap.add_argument("--max-code-len", type=int, default=0, help="longest Huffman code the encoder may use (8..12)")
     ap.add_argument("--experts", type=int, default=None,
                     help="fewer experts than the configuration names (profiling captures on a small case only)")

@@ -6,18 +6,26 @@
 // tcgen05 tensor-core MMAs, so decoded weights never reach global memory.
 //
 // One kernel, ffn_matmul_kernel, computes  Y[slot, row] = sum_k W[row, k] * X[slot, k]
-// for the token slots routed to one expert and a group of 16-row strips of one
-// compressed matrix W (blocked layout: tiles of 16 rows x 256 columns):
+// for the token slots routed to one expert, a group of 16-row strips of one
+// compressed matrix W (blocked layout: tiles of 16 rows x 256 columns) and a
+// range of K:
 //   * each decode warp owns one strip and walks its tiles along K.  A tile is
-//     decoded in two halves of 8 rows; a half is written as the B operand
-//     (N = 8, K-major, no swizzle) into the warp's own buffer and multiplied at
-//     once by 16 MMAs (M = 64 token rows, K = 16 each) issued by one lane; the
-//     accumulators of a strip are 16 fp32 columns of tensor memory;
-//   * one loader warp stages the activations of the current K step (64 x 256
-//     bf16, the A operand) in a two-stage ring shared by all decode warps;
-//   * at the end four warps read the accumulators back (tcgen05.ld) and store Y.
+//     decoded in two halves of 8 rows.  Four warps form a quad: their four
+//     half-tile buffers (8 rows x 256 columns each, K-major, no swizzle) are
+//     the first four 8-row groups of one A operand (M = 64; the upper 32 rows
+//     read whatever follows in shared memory and land in accumulator rows that
+//     nobody reads).  A half is decoded into registers first and stored once
+//     the MMAs that read the previous half are done, so decode and MMA overlap;
+//   * one MMA warp waits for a quad's half to be complete and issues its 16
+//     MMAs (K = 16 each; B = the activations, N = token rows); accumulators live
+//     in tensor memory, one [64 x N] fp32 block per quad and half;
+//   * one loader warp stages the activations of the current K step (token rows
+//     x 256 bf16) in a two-stage ring shared by all quads;
+//   * at the end two warps read the accumulators back (tcgen05.ld) and store Y.
 // The host wrapper runs it for W1 and W3 (gate, up), applies SiLU(g)*u, runs it
-// for W2 with K split four ways, and combines the experts of every token.
+// for W2, and combines the experts of every token; K is split over several
+// CTAs where few experts are active, the partial sums are added by the
+// elementwise kernels.
 // Every wait on a barrier is bounded; a wait that runs out is reported through
 // the status word and the kernel still runs to its end and frees tensor memory.
 #include <cuda_bf16.h>
@@ -31,15 +39,14 @@
 
 namespace zipmoe_dev {
 
-constexpr int kFfnMaxWarps = 20;                         // decode warps per CTA (plus one loader warp)
-constexpr int kFfnMaxThreads = (kFfnMaxWarps + 1) * 32;
+constexpr int kFfnMaxWarps = 16;                         // decode warps per CTA, a multiple of 4 (plus loader and MMA warps)
+constexpr int kFfnMaxThreads = (kFfnMaxWarps + 2) * 32;
 constexpr uint32_t kBLbo = 144;                          // bytes between the 8x8 cores of a half-tile along K: 128 + 16 of
                                                          // padding, so that the 32 lanes' 16-byte stores spread over all banks
 constexpr uint32_t kBBufBytes = 32 * kBLbo;              // one half-tile: 8 rows x 256 columns
 constexpr uint32_t kXGroupBytes = 4096;                  // 8 token rows x 256 columns of bf16, cores 128 bytes apart
-constexpr uint32_t kFfnWarpBytes = 2 * kPayStage + kBBufBytes;
-constexpr uint32_t kFfnBarsPerWarp = 3;                  // two record stages, one "MMAs of my buffer are done"
-constexpr uint32_t kDownSplits = 4;                      // K splits of the down projection
+constexpr uint32_t kFfnWarpBytes = 2 * kPayStage + kBBufBytes;   // two record stages, one half-tile buffer
+constexpr uint32_t kFfnShortTries = 1u << 10;            // wait limit once something has already gone wrong
 
 struct FfnArgs {
   LaunchArgs la;                       // descriptors, tables, payload and SM buffers of all expert tensors
@@ -49,14 +56,21 @@ struct FfnArgs {
   const uint16_t *x;                   // bf16 activations, row pitch K
   float *y;                            // [gridDim.z][S][rows]
   uint32_t rows, K;                    // the matrix is [rows, K]
-  uint32_t tensor_in_expert;           // 0 (then grid z adds 0 or 1: w1, w3) or 2 (w2, grid z is the K split)
-  uint32_t steps_per_split;            // K steps of 256 per CTA
-  uint32_t n_warps, groups, S;         // decode warps, 8-row groups of token rows held per stage, total slots
+  uint32_t tensor_base;                // tensor in expert = tensor_base + blockIdx.z / splits
+  uint32_t splits, steps_per_split;    // K split = blockIdx.z % splits, K steps of 256 per split
+  uint32_t n_warps, groups, S;         // decode warps, 8-row groups of token rows per stage, total slots
+  uint32_t smem_bytes;                 // dynamic shared memory of the launch
 };
 
+// shared-memory layout: [X stages][per-warp buffers][tables][table scratch][barriers][tmem slot]
+__host__ __device__ inline uint32_t ffn_bar_count(uint32_t n_warps) { return 2 * n_warps + 2 * (n_warps / 4) + 4; }
 __host__ __device__ inline uint32_t ffn_smem_bytes(uint32_t n_warps, uint32_t groups) {
-  return 2 * groups * kXGroupBytes + kLutBytes + kLutScratchBytes + n_warps * kFfnWarpBytes +
-         (n_warps * kFfnBarsPerWarp + 4) * 8 + 16;
+  uint32_t after_warps = kLutBytes + kLutScratchBytes + ffn_bar_count(n_warps) * 8 + 16;
+  // the A operand of the last quad reads 8 groups kFfnWarpBytes apart: 4 real ones and 4 more that must
+  // still lie inside the allocation
+  const uint32_t overrun = 4 * kFfnWarpBytes;
+  if (after_warps < overrun) after_warps = overrun;
+  return 2 * groups * kXGroupBytes + n_warps * kFfnWarpBytes + after_warps;
 }
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -91,43 +105,49 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
 
 __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const FfnArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  const uint32_t NW = a.n_warps, G = a.groups;
+  const uint32_t NW = a.n_warps, G = a.groups, Q = NW >> 2, NCOL = 8 * G;
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t e = blockIdx.y, z = blockIdx.z;
   const uint32_t off = __ldg(a.expert_offset + e);
   uint32_t Te = __ldg(a.expert_offset + e + 1) - off;
   if (Te == 0) return;   // nothing routed to this expert
-  if (Te > 8 * G) {      // more slots than the stage holds (a token listing the same expert twice)
+  if (Te > NCOL) {       // more slots than the stage holds (a token listing the same expert twice)
     report(a.la.status, kStatusBadDescriptor);
-    Te = 8 * G;
+    Te = NCOL;
   }
 
   uint8_t *x_raw = smem;                                   // [2][G][4096]
-  uint8_t *lut_raw = x_raw + 2 * G * kXGroupBytes;
+  uint8_t *warp_raw = x_raw + 2 * G * kXGroupBytes;        // [NW][2 record stages | half-tile buffer]
+  uint8_t *lut_raw = warp_raw + NW * kFfnWarpBytes;
   uint8_t *lut_scratch = lut_raw + kLutBytes;
-  uint8_t *warp_raw = lut_scratch + kLutScratchBytes;      // [NW][2 record stages | half-tile buffer]
-  uint64_t *bars = reinterpret_cast<uint64_t *>(warp_raw + NW * kFfnWarpBytes);
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NW * kFfnBarsPerWarp + 4);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(lut_scratch + kLutScratchBytes);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + ffn_bar_count(NW));
+  // barriers: [NW][2] record stages, [Q] quad half written, [Q] quad MMAs done, [2] X full, [2] X empty
   const uint32_t bar0 = smem_addr(bars);
-  const uint32_t x_full = bar0 + 8 * (NW * kFfnBarsPerWarp), x_empty = x_full + 16;   // two barriers each
+  const uint32_t quad_full = bar0 + 8 * (2 * NW), quad_done = quad_full + 8 * Q;
+  const uint32_t x_full = quad_done + 8 * Q, x_empty = x_full + 16;
   const uint32_t x_addr = smem_addr(x_raw), lut = smem_addr(lut_raw);
-  const bool is_loader = warp == NW;
+  const bool is_loader = warp == NW, is_mma = warp == NW + 1, is_decode = warp < NW;
 
   const uint32_t n_strips = a.rows >> 4, strip = blockIdx.x * NW + warp;
-  const bool has_strip = !is_loader && strip < n_strips;
-  const uint32_t tensor = e * 3 + a.tensor_in_expert + (a.tensor_in_expert == 2 ? 0 : z);
-  const uint32_t split = a.tensor_in_expert == 2 ? z : 0;
+  const bool has_strip = is_decode && strip < n_strips;
+  const uint32_t tensor = e * 3 + a.tensor_base + z / a.splits, split = z % a.splits;
   const uint32_t steps_total = a.K >> 8;
-  const uint32_t s0 = split * a.steps_per_split, s1 = min(s0 + a.steps_per_split, steps_total);
+  const uint32_t s0 = min(split * a.steps_per_split, steps_total), s1 = min(s0 + a.steps_per_split, steps_total);
+  const uint32_t n_steps = s1 - s0;
 
   uint32_t tmem_cols = 32;
-  while (tmem_cols < 16 * NW) tmem_cols <<= 1;
+  while (tmem_cols < 2 * Q * NCOL) tmem_cols <<= 1;
   if (tid == 0) {
-    for (uint32_t b = 0; b < NW * kFfnBarsPerWarp; ++b) mbar_init(bar0 + 8 * b, 1);
+    for (uint32_t b = 0; b < 2 * NW; ++b) mbar_init(bar0 + 8 * b, 1);
+    for (uint32_t q = 0; q < Q; ++q) {
+      mbar_init(quad_full + 8 * q, 4);
+      mbar_init(quad_done + 8 * q, 1);
+    }
     mbar_init(x_full, 1);
     mbar_init(x_full + 8, 1);
-    mbar_init(x_empty, NW);
-    mbar_init(x_empty + 8, NW);
+    mbar_init(x_empty, 1);
+    mbar_init(x_empty + 8, 1);
   }
   fence_barrier_init();
   if (warp == 0) {
@@ -143,7 +163,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
 
   // the tensor: blocked layout, 16 x 256 tiles, one Huffman table
   const uint32_t c0 = __ldg(a.tensor_first_chunk + tensor);
-  bool ok = c0 < a.la.n_chunks;
+  bool ok = c0 < a.la.n_chunks && 2 * Q * NCOL <= 512 && 4 * Q == NW;
   uint32_t table_id = 0, tpc = 1;
   if (ok) {
     const zipmoe_chunk_desc *d = a.la.chunks + c0;
@@ -161,40 +181,72 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
 
   if (ok && is_loader) {
     // ---- activations: one K step (8G token rows x 256 columns) per stage ----
-    for (uint32_t s = s0; s < s1; ++s) {
-      const uint32_t b = (s - s0) & 1, n = (s - s0) >> 1;
+    for (uint32_t s = 0; s < n_steps; ++s) {
+      const uint32_t b = s & 1, n = s >> 1;
       if (n > 0 && !mbar_wait_bounded(x_empty + 8 * b, (n - 1) & 1)) {
         report(a.la.status, kStatusWaitTimeout);
         break;
       }
       const uint32_t stage = x_addr + b * G * kXGroupBytes;
-      for (uint32_t idx = lane; idx < 8 * G * 32; idx += 32) {
-        const uint32_t rr = idx & 7, g = (idx >> 3) % G, k8 = idx / (8 * G), row = 8 * g + rr;
+      for (uint32_t row = lane; row < NCOL; row += 32) {
         const uint16_t *src = a.x;
         uint32_t src_bytes = 0;   // rows past the expert's last slot are filled with zeros
         if (row < Te) {
           const uint32_t xr = a.slot_token ? __ldg(a.slot_token + off + row) : off + row;
-          src = a.x + (size_t)xr * a.K + s * 256 + k8 * 8;
+          src = a.x + (size_t)xr * a.K + (size_t)(s0 + s) * 256;
           src_bytes = 16;
         }
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(stage + g * kXGroupBytes + k8 * 128 + rr * 16),
-                     "l"(src), "r"(src_bytes)
-                     : "memory");
+        const uint32_t dst = stage + (row >> 3) * kXGroupBytes + (row & 7) * 16;
+#pragma unroll 8
+        for (uint32_t k8 = 0; k8 < 32; ++k8)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + k8 * 128),
+                       "l"(src + (src_bytes ? k8 * 8 : 0)), "r"(src_bytes)
+                       : "memory");
       }
       asm volatile("cp.async.wait_all;" ::: "memory");
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(x_full + 8 * b);
     }
-  } else if (ok && !is_loader) {
-    // ---- one strip of 16 rows: decode tile after tile along K, multiply half-tile by half-tile ----
+  } else if (ok && is_mma) {
+    // ---- one lane issues, per half-tile and quad: D[64 x N] (+)= A[64 x 256] * X[N x 256]^T ----
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (G << 17) | (4u << 24);   // bf16 x bf16 -> fp32, N = 8G, M = 64
+    const uint32_t buf0 = smem_addr(warp_raw) + 2 * kPayStage;
+    bool alive = true;
+    for (uint32_t s = 0; s < n_steps && alive; ++s) {
+      const uint32_t xb = s & 1, xs = x_addr + xb * G * kXGroupBytes;
+      if (!mbar_wait_bounded(x_full + 8 * xb, (s >> 1) & 1)) alive = false;
+      for (uint32_t half = 0; half < 2 && alive; ++half) {
+        const uint32_t hn = 2 * s + half;
+        for (uint32_t q = 0; q < Q && alive; ++q) {
+          if (!mbar_wait_bounded(quad_full + 8 * q, hn & 1)) {
+            alive = false;
+            break;
+          }
+          if (lane == 0) {
+            tc_fence_after();
+            const uint32_t abuf = buf0 + 4 * q * kFfnWarpBytes;
+            const uint32_t d_tmem = tmem + (2 * q + half) * NCOL;
+#pragma unroll
+            for (uint32_t j = 0; j < 16; ++j)
+              mma_bf16(d_tmem, smem_desc(abuf + j * 2 * kBLbo, kBLbo, kFfnWarpBytes),
+                       smem_desc(xs + j * 256, 128, kXGroupBytes), idesc, (s > 0 || j > 0) ? 1u : 0u);
+            mma_commit(quad_done + 8 * q);
+          }
+          __syncwarp();
+        }
+      }
+      if (alive && lane == 0) mma_commit(x_empty + 8 * xb);   // every MMA that reads this X stage has been issued
+      __syncwarp();
+    }
+    if (!alive) report(a.la.status, kStatusWaitTimeout);
+  } else if (ok && is_decode) {
+    // ---- one strip of 16 rows: decode tile after tile along K, hand half-tiles to the quad's A operand ----
     const uint32_t my = smem_addr(warp_raw + warp * kFfnWarpBytes);
     const uint32_t buf = my + 2 * kPayStage;
-    const uint32_t rec_bar = bar0 + 8 * (warp * kFfnBarsPerWarp), mma_bar = rec_bar + 16;
-    const uint32_t d_tmem = tmem + 16 * warp;
-    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 17) | (4u << 24);   // bf16 x bf16 -> fp32, N=8, M=64
-    uint32_t rec_phase = 0, mma_phase = 0;
-    bool mma_pending = false, failed = !has_strip;
+    const uint32_t rec_bar = bar0 + 8 * (2 * warp), q = warp >> 2;
+    uint32_t rec_phase = 0, hn = 0;
+    bool failed = !has_strip;
     LaunchArgs la = a.la;
     la.out = nullptr;
     la.out_elems = ~0ull;
@@ -203,10 +255,10 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
     TileWork cur;
     cur.ok = false;
     uint2 smA[8], smB[8];
-    if (has_strip) {
-      const uint32_t q = strip * steps_total + s0;
-      tc = c0 + q / tpc;
-      tt = q % tpc;
+    if (has_strip && n_steps) {
+      const uint32_t tq = strip * steps_total + s0;
+      tc = c0 + tq / tpc;
+      tt = tq % tpc;
       cur = resolve_tile(la, tc, tt);
       if (!cur.ok || cur.valid != ZIPMOE_TILE_ELEMS_MAX) {
         report(a.la.status, kStatusBadDescriptor);
@@ -217,12 +269,23 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
         for (int k = 0; k < 8; ++k) smA[k] = __ldg(reinterpret_cast<const uint2 *>(cur.sm + k * 256) + lane);
       }
     }
+    // hand-over of one half in two moves: before the first store, wait until the MMAs of the previous half have
+    // read the buffer; after the last store, make the stores visible to the tensor core and tell the MMA warp
+    auto buffer_free = [&]() -> bool {
+      if (hn == 0) return true;
+      return mbar_wait_bounded(quad_done + 8 * q, (hn - 1) & 1, failed ? kFfnShortTries : (1u << 20));
+    };
+    auto publish = [&]() {
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(quad_full + 8 * q);
+      ++hn;
+    };
     uint32_t stage = 0;
-    for (uint32_t s = s0; s < s1; ++s) {
-      const uint32_t xb = (s - s0) & 1, xn = (s - s0) >> 1;
+    for (uint32_t s = 0; s < n_steps; ++s) {
       TileWork nxt;
       nxt.ok = false;
-      if (!failed && s + 1 < s1) {
+      if (!failed && s + 1 < n_steps) {
         if (++tt >= tpc) {
           tt = 0;
           ++tc;
@@ -248,92 +311,88 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
           LaneDecoder<decltype(staged_c)::value, decltype(fast_c)::value> dec;
           if (!dec.init(my + stage * kPayStage, cur.rec, cur.rec_bytes, lut, lane)) {
             report(a.la.status, kStatusBadBitCount);
+            buffer_free();
+            publish();   // keep the count of halves
+            buffer_free();
+            publish();
             return false;
           }
 #pragma unroll
           for (int k = 0; k < 8; ++k) smB[k] = __ldg(reinterpret_cast<const uint2 *>(cur.sm + (8 + k) * 256) + lane);
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
-            if (mma_pending) {   // the MMAs that read the buffer must be done before it is overwritten
-              if (!mbar_wait_bounded(mma_bar, mma_phase)) {
-                report(a.la.status, kStatusWaitTimeout);
-                return false;
-              }
-              mma_phase ^= 1;
-              mma_pending = false;
+            // the first four iterations are decoded into registers while the previous half's MMAs may still run
+            uint4 v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) v[k] = dec.group(half ? smB[k] : smA[k]);
+            if (!buffer_free()) {
+              report(a.la.status, kStatusWaitTimeout);
+              publish();
+              if (half == 0) publish();   // keep the count of halves
+              return false;
             }
 #pragma unroll
-            for (int k = 0; k < 8; ++k) sts_v4(buf + lane * kBLbo + k * 16, dec.group(half ? smB[k] : smA[k]));
+            for (int k = 0; k < 4; ++k) sts_v4(buf + lane * kBLbo + k * 16, v[k]);
+#pragma unroll
+            for (int k = 4; k < 8; ++k) sts_v4(buf + lane * kBLbo + k * 16, dec.group(half ? smB[k] : smA[k]));
             if (half == 0 && nxt.ok) {
 #pragma unroll
               for (int k = 0; k < 8; ++k) smA[k] = __ldg(reinterpret_cast<const uint2 *>(nxt.sm + k * 256) + lane);
             }
-            fence_async_smem();   // the stores above must be visible to the tensor core's reads
-            __syncwarp();
-            if (half == 0 && !mbar_wait_bounded(x_full + 8 * xb, xn & 1)) {
-              report(a.la.status, kStatusWaitTimeout);
-              return false;
-            }
-            if (lane == 0) {
-              tc_fence_after();
-              const uint32_t xs = x_addr + xb * G * kXGroupBytes;
-#pragma unroll
-              for (uint32_t j = 0; j < 16; ++j)
-                mma_bf16(d_tmem + 8 * half, smem_desc(xs + j * 256, 128, kXGroupBytes),
-                         smem_desc(buf + j * 2 * kBLbo, kBLbo, kBBufBytes), idesc, (s > s0 || j > 0) ? 1u : 0u);
-              mma_commit(mma_bar);
-              if (half == 1) mma_commit(x_empty + 8 * xb);
-            }
-            mma_pending = true;
-            __syncwarp();
+            publish();
           }
           return true;
         };
         if (good) {
           if (cur.staged) good = fast ? run(std::true_type{}, std::true_type{}) : run(std::true_type{}, std::false_type{});
           else good = fast ? run(std::false_type{}, std::true_type{}) : run(std::false_type{}, std::false_type{});
+          step_done = true;   // run() publishes both halves even when it fails
         }
-        if (good) step_done = true;
-        else failed = true;
-        if (!nxt.ok && s + 1 < s1) failed = true;
+        if (!good) failed = true;
+        if (!nxt.ok && s + 1 < n_steps) failed = true;
       }
-      if (!step_done) {
-        // keep the stage ring moving for the other warps: wait for the step, then release it
-        mbar_wait_bounded(x_full + 8 * xb, xn & 1);
-        if (lane == 0) mbar_arrive(x_empty + 8 * xb);
+      if (!step_done) {   // nothing to contribute: keep the quad's hand-over going with whatever the buffer holds
+        buffer_free();
+        publish();
+        buffer_free();
+        publish();
       }
       cur = nxt;
       stage ^= 1;
     }
-    if (mma_pending && !mbar_wait_bounded(mma_bar, mma_phase)) report(a.la.status, kStatusWaitTimeout);
+    // the accumulators are final once the MMAs of the last half are done
+    if (hn > 0 && !mbar_wait_bounded(quad_done + 8 * q, (hn - 1) & 1, failed ? kFfnShortTries : (1u << 20)))
+      report(a.la.status, kStatusWaitTimeout);
   }
 
   // ---- accumulators -> Y ----
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (ok && warp < 4) {
-    // a warp reads the 32 tensor-memory lanes of its quarter; with M = 64, D row 16q + i is lane 32q + i (i < 16)
-    const uint32_t row = 16 * warp + lane;
-    float *yrow = a.y + ((size_t)z * a.S + off + row) * a.rows;
-    for (uint32_t w = 0; w < NW; ++w) {
-      const uint32_t st = blockIdx.x * NW + w;
-      if (st >= n_strips) break;
-      uint32_t r[16];
-      const uint32_t taddr = tmem + ((32 * warp) << 16) + 16 * w;
-      asm volatile(
-          "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-          : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-            "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-          : "r"(taddr)
-          : "memory");
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      if (lane < 16 && row < Te) {
-        float4 *dst = reinterpret_cast<float4 *>(yrow + 16 * st);
+  if (ok && warp < 2 && n_steps) {
+    // With M = 64, D row 16j + i sits in tensor-memory lane 32j + i (i < 16): warp 0 reads rows 0..15 (the halves
+    // of the quad's warps 0 and 1), warp 1 rows 16..31 (warps 2 and 3); rows 32..63 are not used.
+    const uint32_t wq = 2 * warp + ((lane >> 3) & 1), r = lane & 7;
+    for (uint32_t q = 0; q < Q; ++q) {
+      const uint32_t st = blockIdx.x * NW + 4 * q + wq;
+      for (uint32_t half = 0; half < 2; ++half) {
+        const uint32_t row = 16 * st + 8 * half + r;
+        for (uint32_t c = 0; c < G; ++c) {
+          uint32_t v[8];
+          const uint32_t taddr = tmem + ((32 * warp) << 16) + (2 * q + half) * NCOL + 8 * c;
+          asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                       : "r"(taddr)
+                       : "memory");
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          if (lane < 16 && st < n_strips) {
 #pragma unroll
-        for (int v = 0; v < 4; ++v)
-          dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
-                               __uint_as_float(r[4 * v + 3]));
+            for (uint32_t n = 0; n < 8; ++n) {
+              const uint32_t tokrow = 8 * c + n;
+              if (tokrow < Te) a.y[((size_t)z * a.S + off + tokrow) * a.rows + row] = __uint_as_float(v[n]);
+            }
+          }
+        }
       }
     }
   }
@@ -379,11 +438,16 @@ __global__ void route_kernel(const int32_t *topk_ids, uint32_t S, uint32_t k, ui
   }
 }
 
-// h = bf16(SiLU(g) * u), g and u fp32 [S][I]
-__global__ void swiglu_kernel(const float *g, const float *u, uint16_t *h, uint64_t n) {
+// h = bf16(SiLU(g) * u); g = sum of the `splits` partial blocks gu[0 .. splits), u of gu[splits .. 2*splits),
+// each block fp32 [n]
+__global__ void swiglu_kernel(const float *gu, uint32_t splits, uint16_t *h, uint64_t n) {
   for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
-    const float gv = g[i];
-    const float hv = gv / (1.0f + __expf(-gv)) * u[i];
+    float gv = 0.f, uv = 0.f;
+    for (uint32_t sp = 0; sp < splits; ++sp) {
+      gv += gu[(uint64_t)sp * n + i];
+      uv += gu[(uint64_t)(splits + sp) * n + i];
+    }
+    const float hv = gv / (1.0f + __expf(-gv)) * uv;
     h[i] = __bfloat16_as_ushort(__float2bfloat16_rn(hv));
   }
 }
@@ -410,29 +474,40 @@ __global__ void combine_kernel(const float *y, const uint32_t *slot_of, const fl
 namespace {
 
 struct FfnPlan {
-  uint32_t S, groups, n_warps, smem;
+  uint32_t S, groups, n_warps, smem, splits_gu, splits_dn;
   uint64_t off_offsets, off_slot_token, off_slot_of, off_gu, off_h, off_y, total;
 };
+
+// K splits so that the CTAs of the busiest plausible case fill the GPU a few times over:
+// `ctas` CTAs exist without splitting, `steps` K steps are there to split
+uint32_t pick_splits(uint32_t ctas, uint32_t steps) {
+  const uint32_t target = 4 * 148;
+  uint32_t splits = 1;
+  while (splits * 2 <= 8 && ctas * splits < target && steps / (splits * 2) >= 2) splits *= 2;
+  return splits;
+}
 
 zipmoe_status make_plan(uint32_t T, uint32_t k, const zipmoe_compressed_experts *ex, FfnPlan *p) {
   if (!ex || T == 0 || k == 0 || T > 64 || k > 8 || ex->n_experts == 0 || ex->n_experts > 256) return ZIPMOE_ERR_UNSUPPORTED;
   if (ex->hidden == 0 || ex->inter == 0 || ex->hidden % 256 || ex->inter % 256) return ZIPMOE_ERR_UNSUPPORTED;
-  if ((ex->inter / 256) % zipmoe_dev::kDownSplits) return ZIPMOE_ERR_UNSUPPORTED;
   p->S = T * k;
   p->groups = (T + 7) / 8;
   uint32_t nw = zipmoe_dev::kFfnMaxWarps;
-  while (nw > 8 && zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) --nw;   // the table builder needs 256 threads
+  while (nw > 8 && zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) nw -= 4;   // the table builder needs 256 threads
   if (zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) return ZIPMOE_ERR_UNSUPPORTED;
   p->n_warps = nw;
   p->smem = zipmoe_dev::ffn_smem_bytes(nw, p->groups);
+  const uint32_t active = p->S < ex->n_experts ? p->S : ex->n_experts;   // at most this many experts get tokens
+  p->splits_gu = pick_splits(active * 2 * ((ex->inter / 16 + nw - 1) / nw), ex->hidden / 256);
+  p->splits_dn = pick_splits(active * ((ex->hidden / 16 + nw - 1) / nw), ex->inter / 256);
   auto up = [](uint64_t v) { return (v + 255) / 256 * 256; };
   uint64_t at = 0;
   p->off_offsets = at; at = up(at + 4ull * (ex->n_experts + 1));
   p->off_slot_token = at; at = up(at + 4ull * p->S);
   p->off_slot_of = at; at = up(at + 4ull * p->S);
-  p->off_gu = at; at = up(at + 2ull * p->S * ex->inter * 4);
+  p->off_gu = at; at = up(at + 2ull * p->splits_gu * p->S * ex->inter * 4);
   p->off_h = at; at = up(at + (uint64_t)p->S * ex->inter * 2);
-  p->off_y = at; at = up(at + (uint64_t)zipmoe_dev::kDownSplits * p->S * ex->hidden * 4);
+  p->off_y = at; at = up(at + (uint64_t)p->splits_dn * p->S * ex->hidden * 4);
   p->total = at;
   return ZIPMOE_OK;
 }
@@ -510,22 +585,24 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.n_warps = p.n_warps;
   a.groups = p.groups;
   a.S = S;
-  const uint32_t threads = (p.n_warps + 1) * 32;
+  a.smem_bytes = p.smem;
+  const uint32_t threads = (p.n_warps + 2) * 32;
 
-  // gate and up: Y[z] = W_{1,3} X over the full K = H
+  // gate and up: partial Y[matrix][split] = W_{1,3}[:, split] X[:, split]
   a.slot_token = slot_token;
   a.x = tokens;
   a.y = gu;
   a.rows = I;
   a.K = H;
-  a.tensor_in_expert = 0;
-  a.steps_per_split = H / 256;
-  dim3 grid_gu((I / 16 + p.n_warps - 1) / p.n_warps, E, 2);
+  a.tensor_base = 0;
+  a.splits = p.splits_gu;
+  a.steps_per_split = (H / 256 + p.splits_gu - 1) / p.splits_gu;
+  dim3 grid_gu((I / 16 + p.n_warps - 1) / p.n_warps, E, 2 * p.splits_gu);
   ffn_matmul_kernel<<<grid_gu, threads, p.smem, stream>>>(a);
 
   const uint64_t n_h = (uint64_t)S * I;
   const unsigned act_blocks = (unsigned)((n_h + 1023) / 1024 < 592 ? (n_h + 1023) / 1024 : 592);
-  swiglu_kernel<<<act_blocks, 256, 0, stream>>>(gu, gu + n_h, h, n_h);
+  swiglu_kernel<<<act_blocks, 256, 0, stream>>>(gu, p.splits_gu, h, n_h);
 
   // down: partial Y[split] = W_2[:, split] H[:, split]
   a.slot_token = nullptr;
@@ -533,11 +610,12 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.y = y;
   a.rows = H;
   a.K = I;
-  a.tensor_in_expert = 2;
-  a.steps_per_split = I / 256 / kDownSplits;
-  dim3 grid_dn((H / 16 + p.n_warps - 1) / p.n_warps, E, kDownSplits);
+  a.tensor_base = 2;
+  a.splits = p.splits_dn;
+  a.steps_per_split = (I / 256 + p.splits_dn - 1) / p.splits_dn;
+  dim3 grid_dn((H / 16 + p.n_warps - 1) / p.n_warps, E, p.splits_dn);
   ffn_matmul_kernel<<<grid_dn, threads, p.smem, stream>>>(a);
 
-  combine_kernel<<<dim3((H + 255) / 256, T), 256, 0, stream>>>(y, slot_of, topk_weights, T, k, S, H, kDownSplits, out);
+  combine_kernel<<<dim3((H + 255) / 256, T), 256, 0, stream>>>(y, slot_of, topk_weights, T, k, S, H, p.splits_dn, out);
   return cudaGetLastError() == cudaSuccess ? ZIPMOE_OK : ZIPMOE_ERR_CUDA;
 }
