@@ -160,7 +160,7 @@ class ClockSampler(threading.Thread):
 
 
 # ----------------------------------------------------------------------------- fused expert FFN
-def bench_ffn(dev, iters=20, cpu_tokens=2):
+def bench_ffn(dev, iters=20, cpu_tokens=2, token_counts=(1, 16, 64)):
     """Fused decode + expert SwiGLU FFN on 8 experts of 4096 -> 14336 -> 4096 (top-2 of 8, Zipf(1.2)
     popularity) for T = 1, 16, 64 tokens, against decode-then-GEMM: zipmoe_decode of the routed experts
     into bf16 followed by torch matmuls on the same stream.  Also times the CPU oracle's FFN on a few tokens."""
@@ -173,7 +173,7 @@ def bench_ffn(dev, iters=20, cpu_tokens=2):
     expert_bytes = [sum(i.payload_bytes + i.n_elems for i in p.plan.infos) for p in per_expert]
     stream = torch.cuda.current_stream(dev)
     out = {}
-    for T in (1, 16, 64):
+    for T in token_counts:
         tok = inputs.tokens(T, 4096, seed=100 + T)
         ids, wts = inputs.routing(T, n_experts=8, k=2, seed=T)
         d_tok = torch.from_numpy(tok.view(np.int16)).to(dev)
@@ -224,6 +224,9 @@ def bench_ffn(dev, iters=20, cpu_tokens=2):
                           "compressed_gbs": nbytes / us_f / 1e3, "decode_then_gemm_us": us_u,
                           "speedup_vs_decode_then_gemm": us_u / us_f, "max_abs_diff_vs_decode_then_gemm": diff,
                           "status": int(ex.dev.status.item())}
+    out["config"] = "8 experts 4096->14336->4096 bf16 (blocked layout, 256K-element chunks), top-2, Zipf(1.2)"
+    if not cpu_tokens:
+        return out
     # CPU oracle FFN on a few tokens of the T = 16 case (fp64 numpy)
     from oracle import ffn as offn
     tok = inputs.tokens(16, 4096, seed=116)
@@ -234,7 +237,6 @@ def bench_ffn(dev, iters=20, cpu_tokens=2):
     dt = time.perf_counter() - t0
     out["cpu_oracle"] = {"tokens_per_s": cpu_tokens / dt, "sample": "%d tokens of the T=16 case, fp64 numpy" % cpu_tokens,
                          "cores": os.cpu_count() or 1}
-    out["config"] = "8 experts 4096->14336->4096 bf16 (blocked layout, 256K-element chunks), top-2, Zipf(1.2)"
     return out
 
 
@@ -253,6 +255,10 @@ def run_ours(args):
 
     from paper_2601_21198_b200 import binding, build
     build.build()
+    if args.ffn_only:      # profiling captures of the fused kernels on one token count
+        res = bench_ffn(dev, iters=args.ffn_iters, cpu_tokens=0, token_counts=(args.ffn_only,))
+        print(json.dumps({"ffn": res}))
+        return
     w = build_workload(args.workload, keep_originals=False, experts=args.experts, max_code_len=args.max_code_len)
     plan = w.plan
     dplan = plan.to_device(dev)
@@ -388,6 +394,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="small_layer", choices=["small_layer", "large_layer", "single_matrix"])
+    ap.add_argument("--ffn-only", type=int, default=0, metavar="T",
+                    help="run only the fused expert-FFN section for T tokens (profiling captures)")
+    ap.add_argument("--ffn-iters", type=int, default=20)
     ap.add_argument("--no-ffn", action="store_true", help="skip the fused expert-FFN section of the report")
     ap.add_argument("--max-code-len", type=int, default=0, help="longest Huffman code the encoder may use (8..12)")
     ap.add_argument("--experts", type=int, default=None,
