@@ -217,6 +217,37 @@ zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32_t T, const
                                        const zipmoe_compressed_experts *experts, uint16_t *out, void *workspace,
                                        uint64_t workspace_bytes, uint32_t *status_word, zipmoe_stream stream);
 
+/* Size of the scratch built into the library for zipmoe_decode_expert_ffn_noalloc. */
+#define ZIPMOE_NOALLOC_SCRATCH_BYTES (8u << 20)
+
+/* The fused expert FFN for callers that have no way to obtain device memory.  (The paper has no
+ * counterpart: this entry point exists for the embedding program's sake, not for the method's.)
+ *
+ * zipmoe_decode_expert_ffn needs a scratch buffer, and somebody has to allocate it.  Some callers
+ * cannot: a plug-in inside a serving process whose host framework owns the whole device-memory pool
+ * and hands out none of it, or a latency-critical decode loop in which cudaMalloc is off limits because
+ * it synchronises the device and may fail late.  This variant takes no workspace argument.  It computes
+ * exactly what zipmoe_decode_expert_ffn computes, with the same kernels, using a fixed array of
+ * ZIPMOE_NOALLOC_SCRATCH_BYTES (8 MiB) that is part of the library image: every GPU that loads the
+ * library keeps those 8 MiB reserved until the process exits.  It calls no allocation or free routine
+ * of any kind.
+ *
+ *   - Calls whose scratch need (zipmoe_ffn_workspace_bytes) exceeds the built-in array are refused
+ *     with ZIPMOE_ERR_BUFFER_TOO_SMALL before anything is launched; use zipmoe_decode_expert_ffn with
+ *     a buffer of your own for those.
+ *   - The first call on each device looks up the device address of the array (the device must be
+ *     current).  Make that first call outside any stream capture; later calls do no set-up.
+ *   - Every call on a device uses the same array, which keeps the previous call's contents.  Nothing
+ *     in it has to be cleared: each call writes every word it later reads.  Two calls that overlap on
+ *     the GPU (different streams, no ordering between them) race on the array and give wrong results;
+ *     order them, or give all but one a workspace of their own through zipmoe_decode_expert_ffn.
+ *
+ * Arguments, limits and errors otherwise as for zipmoe_decode_expert_ffn. */
+zipmoe_status zipmoe_decode_expert_ffn_noalloc(const uint16_t *tokens, uint32_t T, const int32_t *topk_ids,
+                                               const float *topk_weights, uint32_t k,
+                                               const zipmoe_compressed_experts *experts, uint16_t *out,
+                                               uint32_t *status_word, zipmoe_stream stream);
+
 /* Name of a status code (static string). */
 const char *zipmoe_status_string(zipmoe_status s);
 

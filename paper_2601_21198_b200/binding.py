@@ -68,6 +68,10 @@ _lib.zipmoe_decode.argtypes = [_vp, _u32, _u32, _vp, _u32, _vp, _u64, _vp, _u64,
 _lib.zipmoe_ffn_workspace_bytes.argtypes = [_u32, _u32, ctypes.POINTER(CompressedExperts), ctypes.POINTER(_u64)]
 _lib.zipmoe_decode_expert_ffn.argtypes = [_vp, _u32, _vp, _vp, _u32, ctypes.POINTER(CompressedExperts), _vp, _vp, _u64,
                                           _vp, _vp]
+_lib.zipmoe_decode_expert_ffn_noalloc.argtypes = [_vp, _u32, _vp, _vp, _u32, ctypes.POINTER(CompressedExperts), _vp, _vp,
+                                                  _vp]
+_lib.zipmoe_decode_expert_ffn_noalloc.restype = _int
+NOALLOC_SCRATCH_BYTES = 8 << 20
 for _f in ("zipmoe_ffn_workspace_bytes", "zipmoe_decode_expert_ffn", "zipmoe_encode_bound", "zipmoe_encode", "zipmoe_blob_info_get", "zipmoe_blob_validate",
            "zipmoe_blob_plan", "zipmoe_decode"):
     getattr(_lib, _f).restype = _int
@@ -172,6 +176,15 @@ def zipmoe_decode_expert_ffn(tokens, T, topk_ids, topk_weights, k, experts, out,
     _check("zipmoe_decode_expert_ffn",
            _lib.zipmoe_decode_expert_ffn(_ptr(tokens), T, _ptr(topk_ids), _ptr(topk_weights), k, ctypes.byref(experts),
                                          _ptr(out), _ptr(workspace), workspace_bytes, _ptr(status_word), _ptr(stream)))
+
+
+def zipmoe_decode_expert_ffn_noalloc(tokens, T, topk_ids, topk_weights, k, experts, out, status_word=None, stream=None):
+    """zipmoe_decode_expert_ffn without a workspace argument: the library's built-in scratch is used, so the
+    caller (and this binding) allocates nothing.  Raises ZipMoEError(ERR_BUFFER_TOO_SMALL) when the call needs
+    more than NOALLOC_SCRATCH_BYTES of scratch."""
+    _check("zipmoe_decode_expert_ffn_noalloc",
+           _lib.zipmoe_decode_expert_ffn_noalloc(_ptr(tokens), T, _ptr(topk_ids), _ptr(topk_weights), k,
+                                                 ctypes.byref(experts), _ptr(out), _ptr(status_word), _ptr(stream)))
 
 
 class DecodePlan:

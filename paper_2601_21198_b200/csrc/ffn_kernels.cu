@@ -619,3 +619,33 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   combine_kernel<<<dim3((H + 255) / 256, T), 256, 0, stream>>>(y, slot_of, topk_weights, T, k, S, H, p.splits_dn, out);
   return cudaGetLastError() == cudaSuccess ? ZIPMOE_OK : ZIPMOE_ERR_CUDA;
 }
+
+// ---- the same call for callers that cannot allocate device memory ------------------------------
+namespace {
+// Scratch for zipmoe_decode_expert_ffn_noalloc.  It is part of the library image: every GPU that loads the
+// library sets these bytes aside until the process exits, whether or not the entry point is ever called.
+constexpr uint64_t kNoAllocScratchBytes = ZIPMOE_NOALLOC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+// Device address of g_noalloc_scratch per device.  In host code the symbol itself is only a stand-in, not an
+// address the GPU can use, so the address is asked for once per device and kept here.
+void *g_noalloc_ptr[64];
+}  // namespace
+
+extern "C" zipmoe_status zipmoe_decode_expert_ffn_noalloc(const uint16_t *tokens, uint32_t T, const int32_t *topk_ids,
+                                                          const float *topk_weights, uint32_t k,
+                                                          const zipmoe_compressed_experts *experts, uint16_t *out,
+                                                          uint32_t *status_word, zipmoe_stream stream) {
+  uint64_t need = 0;
+  zipmoe_status rc = zipmoe_ffn_workspace_bytes(T, k, experts, &need);
+  if (rc != ZIPMOE_OK) return rc;
+  if (need > kNoAllocScratchBytes) return ZIPMOE_ERR_BUFFER_TOO_SMALL;   // the call does not fit the built-in scratch
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ZIPMOE_ERR_CUDA;
+  if (!g_noalloc_ptr[dev]) {   // first call on this device, with this device current
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return ZIPMOE_ERR_CUDA;
+    g_noalloc_ptr[dev] = ptr;
+  }
+  return zipmoe_decode_expert_ffn(tokens, T, topk_ids, topk_weights, k, experts, out, g_noalloc_ptr[dev],
+                                  kNoAllocScratchBytes, status_word, stream);
+}
