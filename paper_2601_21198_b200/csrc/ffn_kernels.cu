@@ -246,28 +246,71 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
     const uint32_t buf = my + 2 * kPayStage;
     const uint32_t rec_bar = bar0 + 8 * (2 * warp), q = warp >> 2;
     uint32_t rec_phase = 0, hn = 0;
-    bool failed = !has_strip;
-    LaunchArgs la = a.la;
-    la.out = nullptr;
-    la.out_elems = ~0ull;
+    bool failed = !has_strip || n_steps == 0;
 
-    uint32_t tc = 0, tt = 0;
-    TileWork cur;
-    cur.ok = false;
-    uint2 smA[8], smB[8];
+    // Where the strip's tiles are: lane i (and i + 32) looks up record start and length of the i-th tile of
+    // the K range once, so that the loop below touches global memory only for the data itself.
+    uint32_t rec_at[2] = {0, 0}, rec_len[2] = {0, 0};   // in 16-byte units from the start of the payload buffer
+    const uint8_t *sm_strip = a.la.sm;                  // sign+mantissa bytes of the strip's first tile
     if (has_strip && n_steps) {
-      const uint32_t tq = strip * steps_total + s0;
-      tc = c0 + tq / tpc;
-      tt = tq % tpc;
-      cur = resolve_tile(la, tc, tt);
-      if (!cur.ok || cur.valid != ZIPMOE_TILE_ELEMS_MAX) {
+      const uint32_t tq0 = strip * steps_total + s0;
+      bool bad = n_steps > 64;
+      for (uint32_t r = 0; r < 2; ++r) {
+        const uint32_t i = lane + 32 * r;
+        if (i >= n_steps || bad) continue;
+        const uint32_t tq = tq0 + i, c = c0 + tq / tpc, t = tq % tpc;
+        if (c >= a.la.n_chunks) {
+          bad = true;
+          continue;
+        }
+        const zipmoe_chunk_desc *d = a.la.chunks + c;
+        const uint64_t pay_off = __ldg(&d->payload_off);
+        if (t >= __ldg(&d->n_tiles) || __ldg(&d->tile_elems) != ZIPMOE_TILE_ELEMS_MAX || (pay_off & 15) ||
+            __ldg(&d->table_id) != table_id || pay_off + 4ull * (t + 2) > a.la.payload_bytes ||
+            (t + 1 == __ldg(&d->n_tiles) && __ldg(&d->last_tile_elems) != ZIPMOE_TILE_ELEMS_MAX)) {
+          bad = true;
+          continue;
+        }
+        const uint32_t *tab = reinterpret_cast<const uint32_t *>(a.la.payload + pay_off);
+        const uint32_t o0 = __ldg(tab + t), o1 = __ldg(tab + t + 1);
+        if (o1 <= o0 || o1 - o0 < 4 || o1 - o0 > (64 + ZIPMOE_TILE_ELEMS_MAX / 8 * ZIPMOE_MAX_CODE_LEN) / 16 + 1 ||
+            pay_off + 16ull * o1 > a.la.payload_bytes) {
+          bad = true;
+          continue;
+        }
+        rec_at[r] = (uint32_t)(pay_off >> 4) + o0;
+        rec_len[r] = o1 - o0;
+      }
+      const uint64_t sm_first = __ldg(&a.la.chunks[c0].sm_off) + (uint64_t)tq0 * ZIPMOE_TILE_ELEMS_MAX;
+      if ((sm_first & 15) || sm_first + (uint64_t)n_steps * ZIPMOE_TILE_ELEMS_MAX > a.la.sm_bytes) bad = true;
+      sm_strip = a.la.sm + sm_first;
+      if (__any_sync(0xFFFFFFFFu, bad)) {
         report(a.la.status, kStatusBadDescriptor);
         failed = true;
-      } else {
-        if (cur.staged && lane == 0) bulk_load(my, cur.rec, cur.rec_bytes, rec_bar);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) smA[k] = __ldg(reinterpret_cast<const uint2 *>(cur.sm + k * 256) + lane);
       }
+    }
+    struct Tile {
+      const uint8_t *rec, *sm;
+      uint32_t rec_bytes;
+      bool staged;
+    };
+    auto tile = [&](uint32_t i) -> Tile {   // the i-th tile of the K range (all lanes call this)
+      const uint32_t at = __shfl_sync(0xFFFFFFFFu, i < 32 ? rec_at[0] : rec_at[1], i & 31);
+      const uint32_t len = __shfl_sync(0xFFFFFFFFu, i < 32 ? rec_len[0] : rec_len[1], i & 31);
+      Tile t;
+      t.rec = a.la.payload + (size_t)at * 16;
+      t.rec_bytes = len * 16;
+      t.sm = sm_strip + (size_t)i * ZIPMOE_TILE_ELEMS_MAX;
+      t.staged = t.rec_bytes <= (uint32_t)kPayBuf;
+      return t;
+    };
+    Tile cur = {a.la.payload, a.la.sm, 0, false};
+    uint2 smA[8], smB[8];
+    if (!failed) {
+      cur = tile(0);
+      if (cur.staged && lane == 0) bulk_load(my, cur.rec, cur.rec_bytes, rec_bar);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) smA[k] = __ldg(reinterpret_cast<const uint2 *>(cur.sm + k * 256) + lane);
     }
     // hand-over of one half in two moves: before the first store, wait until the MMAs of the previous half have
     // read the buffer; after the last store, make the stores visible to the tensor core and tell the MMA warp
@@ -283,20 +326,12 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
     };
     uint32_t stage = 0;
     for (uint32_t s = 0; s < n_steps; ++s) {
-      TileWork nxt;
-      nxt.ok = false;
-      if (!failed && s + 1 < n_steps) {
-        if (++tt >= tpc) {
-          tt = 0;
-          ++tc;
-        }
-        nxt = resolve_tile(la, tc, tt);
-        if (!nxt.ok || nxt.valid != ZIPMOE_TILE_ELEMS_MAX) {
-          report(a.la.status, kStatusBadDescriptor);
-          nxt.ok = false;
-        } else if (nxt.staged && lane == 0) {
+      Tile nxt = cur;
+      const bool have_next = !failed && s + 1 < n_steps;
+      if (have_next) {
+        nxt = tile(s + 1);
+        if (nxt.staged && lane == 0)
           bulk_load(my + (stage ^ 1) * kPayStage, nxt.rec, nxt.rec_bytes, rec_bar + 8 * (stage ^ 1));
-        }
       }
       bool step_done = false;
       if (!failed) {
@@ -335,7 +370,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
             for (int k = 0; k < 4; ++k) sts_v4(buf + lane * kBLbo + k * 16, v[k]);
 #pragma unroll
             for (int k = 4; k < 8; ++k) sts_v4(buf + lane * kBLbo + k * 16, dec.group(half ? smB[k] : smA[k]));
-            if (half == 0 && nxt.ok) {
+            if (half == 0 && have_next) {
 #pragma unroll
               for (int k = 0; k < 8; ++k) smA[k] = __ldg(reinterpret_cast<const uint2 *>(nxt.sm + k * 256) + lane);
             }
@@ -349,7 +384,6 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
           step_done = true;   // run() publishes both halves even when it fails
         }
         if (!good) failed = true;
-        if (!nxt.ok && s + 1 < n_steps) failed = true;
       }
       if (!step_done) {   // nothing to contribute: keep the quad's hand-over going with whatever the buffer holds
         buffer_free();
