@@ -52,6 +52,8 @@ def build_workload(name, keep_originals, experts=None, max_code_len=0):
         return workloads.large_layer(n_experts=experts or 8, keep_originals=keep_originals, max_code_len=max_code_len)
     if name == "single_matrix":
         return workloads.single_matrix(keep_originals=keep_originals, max_code_len=max_code_len)
+    if name.startswith("stress"):      # stress1024 / stress16384 / stress262144: the stress-set tensors of one chunk size
+        return workloads.stress_set(chunk_elems=int(name[6:]), keep_originals=keep_originals)[0]
     raise SystemExit("unknown workload %s" % name)
 
 
@@ -393,7 +395,7 @@ def main():
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="small_layer", choices=["small_layer", "large_layer", "single_matrix"])
+    ap.add_argument("--workload", default="small_layer", choices=["small_layer", "large_layer", "single_matrix", "stress1024", "stress16384", "stress262144"])
     ap.add_argument("--ffn-only", type=int, default=0, metavar="T",
                     help="run only the fused expert-FFN section for T tokens (profiling captures)")
     ap.add_argument("--ffn-iters", type=int, default=20)

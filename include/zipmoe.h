@@ -181,7 +181,7 @@ zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t n_chunks, 
  * out_off is not used), `tensor_first_chunk[3e+j]` the index of each tensor's
  * first descriptor, `tables` the code lengths its table_id refers to. */
 typedef struct {
-  uint32_t n_experts, hidden, inter, n_chunks;   /* hidden, inter: multiples of 256; inter/256 a multiple of 4 */
+  uint32_t n_experts, hidden, inter, n_chunks;   /* hidden, inter: multiples of 256                           */
   const zipmoe_chunk_desc *chunks;               /* device [n_chunks]                                          */
   const uint32_t *tensor_first_chunk;            /* device [3 * n_experts]                                     */
   const zipmoe_table *tables;                    /* device [n_tables]                                          */

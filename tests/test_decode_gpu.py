@@ -212,3 +212,27 @@ def test_large_expert_layer_config_full(zb):
 def test_large_expert_layer_blocked_layout(zb):
     from paper_2601_21198_b200 import workloads
     _check_full_workload(zb, workloads.large_layer(n_experts=1, layout=1), 6)
+
+
+def test_codec_stress_set_full(zb):
+    """All 4096 tensors of the stress set (sizes 1K-4M, four value families, chunk sizes 1K / 16K / 256K): one
+    launch per chunk size, whole output against the originals, sampled tensors against the oracle's decode."""
+    import torch
+    from paper_2601_21198_b200 import workloads
+    rng = np.random.default_rng(5)
+    seen = 0
+    for w in workloads.stress_set():
+        dev = w.plan.to_device()
+        out = dev.new_output()
+        dev.decode(out)
+        torch.cuda.synchronize()
+        assert int(dev.status.item()) == 0, w.label
+        host = out.cpu().numpy().view(np.uint16)
+        for i, x in enumerate(w.originals):
+            assert np.array_equal(w.plan.tensor_slice(host, i), x), (w.label, w.names[i])
+        small = [i for i, x in enumerate(w.originals) if x.size < 200000]
+        for i in rng.choice(small, 6, replace=False):
+            assert np.array_equal(w.plan.tensor_slice(host, int(i)), codec.decode(w.blobs[int(i)]))
+        seen += len(w.blobs)
+        del dev, out, host
+    assert seen == 4096
