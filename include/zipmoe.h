@@ -171,6 +171,14 @@ zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t n_chunks, 
                             uint64_t payload_bytes, const uint8_t *sm, uint64_t sm_bytes, uint16_t *out_bf16,
                             uint64_t out_elems, uint32_t *status_word, zipmoe_stream stream);
 
+/* The recovery step alone (Section 3.3, "Memory-Coalesced Tensor Recovery Kernel"): exponent bytes that
+ * are already decompressed and sign+mantissa bytes, both in element order, are merged into bf16:
+ *     out[i] = (sm[i] & 0x80) << 8 | exp[i] << 7 | (sm[i] & 0x7F).
+ * One launch on `stream`, asynchronous, 2 bytes read and 2 written per element.
+ * device in : exp[n_elems], sm[n_elems];  device out: out_bf16[n_elems]; all three 16-byte aligned. */
+zipmoe_status zipmoe_recover(const uint8_t *exp, const uint8_t *sm, uint64_t n_elems, uint16_t *out_bf16,
+                             zipmoe_stream stream);
+
 /* ---- fused decode + routed expert FFN (device) ----------------------------- */
 
 /* The compressed experts of one MoE layer.  A HOST struct holding DEVICE

@@ -65,6 +65,8 @@ _lib.zipmoe_blob_info_get.argtypes = [_vp, _u64, ctypes.POINTER(BlobInfo)]
 _lib.zipmoe_blob_validate.argtypes = [_vp, _u64]
 _lib.zipmoe_blob_plan.argtypes = [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _u32, _vp, _vp]
 _lib.zipmoe_decode.argtypes = [_vp, _u32, _u32, _vp, _u32, _vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp]
+_lib.zipmoe_recover.argtypes = [_vp, _vp, _u64, _vp, _vp]
+_lib.zipmoe_recover.restype = _int
 _lib.zipmoe_ffn_workspace_bytes.argtypes = [_u32, _u32, ctypes.POINTER(CompressedExperts), ctypes.POINTER(_u64)]
 _lib.zipmoe_decode_expert_ffn.argtypes = [_vp, _u32, _vp, _vp, _u32, ctypes.POINTER(CompressedExperts), _vp, _vp, _u64,
                                           _vp, _vp]
@@ -162,6 +164,11 @@ def zipmoe_decode(chunks, n_chunks, n_tiles, tables, n_tables, payload, payload_
     _check("zipmoe_decode", _lib.zipmoe_decode(_ptr(chunks), n_chunks, n_tiles, _ptr(tables), n_tables, _ptr(payload),
                                                 payload_bytes, _ptr(sm), sm_bytes, _ptr(out_bf16), out_elems,
                                                 _ptr(status_word), _ptr(stream)))
+
+
+def zipmoe_recover(exp, sm, n_elems, out_bf16, stream=None):
+    """Merge decompressed exponent bytes and sign+mantissa bytes (device tensors) into bf16."""
+    _check("zipmoe_recover", _lib.zipmoe_recover(_ptr(exp), _ptr(sm), n_elems, _ptr(out_bf16), _ptr(stream)))
 
 
 def zipmoe_ffn_workspace_bytes(T, k, experts):

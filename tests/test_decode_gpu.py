@@ -236,3 +236,20 @@ def test_codec_stress_set_full(zb):
         seen += len(w.blobs)
         del dev, out, host
     assert seen == 4096
+
+
+@pytest.mark.parametrize("n", [1, 15, 16, 17, 4097, 1 << 20, (1 << 22) + 5])
+def test_recovery_kernel_matches_oracle_merge(zb, n):
+    """zipmoe_recover against the oracle's bit-field merge (pinned on the CPU by the value formula)."""
+    import torch
+    rng = np.random.default_rng(n)
+    e = rng.integers(0, 256, n, dtype=np.uint8)
+    s = rng.integers(0, 256, n, dtype=np.uint8)
+    pad = (-n) % 16
+    de = torch.from_numpy(np.concatenate([e, np.zeros(pad, np.uint8)])).cuda()
+    ds = torch.from_numpy(np.concatenate([s, np.zeros(pad, np.uint8)])).cuda()
+    out = torch.full((n + pad,), 0x5555, dtype=torch.int16, device="cuda")
+    zb.zipmoe_recover(de, ds, n, out, torch.cuda.current_stream().cuda_stream)
+    got = out.cpu().numpy().view(np.uint16)
+    assert np.array_equal(got[:n], codec.merge(e, s))
+    assert (got[n:] == 0x5555).all()
