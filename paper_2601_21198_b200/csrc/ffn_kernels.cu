@@ -52,6 +52,7 @@ struct FfnArgs {
   LaunchArgs la;                       // descriptors, tables, payload and SM buffers of all expert tensors
   const uint32_t *tensor_first_chunk;  // [3E] first descriptor of tensor e*3 + {0 w1, 1 w3, 2 w2}
   const uint32_t *expert_offset;       // [E+1] first slot of each expert
+  const uint32_t *active;              // [0] number of experts with tokens, [1..] their ids; blockIdx.y indexes this list
   const uint32_t *slot_token;          // [S] token of each slot, or null when X rows are the slots themselves
   const uint16_t *x;                   // bf16 activations, row pitch K
   float *y;                            // [gridDim.z][S][rows]
@@ -107,7 +108,8 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   extern __shared__ __align__(128) uint8_t smem[];
   const uint32_t NW = a.n_warps, G = a.groups, Q = NW >> 2, NCOL = 8 * G;
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t e = blockIdx.y, z = blockIdx.z;
+  if (blockIdx.y >= __ldg(a.active)) return;   // fewer experts have tokens than the grid allows for
+  const uint32_t e = __ldg(a.active + 1 + blockIdx.y), z = blockIdx.z;
   const uint32_t off = __ldg(a.expert_offset + e);
   uint32_t Te = __ldg(a.expert_offset + e + 1) - off;
   if (Te == 0) return;   // nothing routed to this expert
@@ -440,28 +442,33 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
 // slot_of[t*k + j] = slot of the j-th choice of token t (0xFFFFFFFF for an id out of range);
 // slots of an expert are consecutive, in token order.
 __global__ void route_kernel(const int32_t *topk_ids, uint32_t S, uint32_t k, uint32_t E, uint32_t max_per_expert,
-                             uint32_t *expert_offset, uint32_t *slot_token, uint32_t *slot_of, uint32_t *status) {
-  extern __shared__ uint32_t cnt[];   // [E] counts, then [E] cursors
-  uint32_t *cursor = cnt + E;
-  for (uint32_t i = threadIdx.x; i < 2 * E; i += blockDim.x) cnt[i] = 0;
+                             uint32_t *expert_offset, uint32_t *active, uint32_t *slot_token, uint32_t *slot_of,
+                             uint32_t *status) {
+  extern __shared__ uint32_t sh[];   // [E] counts, [E] cursors, [S] ids
+  uint32_t *cnt = sh, *cursor = sh + E;
+  int32_t *ids = reinterpret_cast<int32_t *>(sh + 2 * E);
+  for (uint32_t i = threadIdx.x; i < 2 * E; i += blockDim.x) sh[i] = 0;
   __syncthreads();
   for (uint32_t i = threadIdx.x; i < S; i += blockDim.x) {
     const int32_t ex = topk_ids[i];
+    ids[i] = ex;
     if (ex >= 0 && (uint32_t)ex < E) atomicAdd(&cnt[ex], 1u);
     else report(status, kStatusBadDescriptor);
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    uint32_t run = 0;
+    uint32_t run = 0, n_active = 0;
     for (uint32_t x = 0; x < E; ++x) {
       expert_offset[x] = run;
       cursor[x] = run;
       if (cnt[x] > max_per_expert) report(status, kStatusBadDescriptor);
+      if (cnt[x]) active[1 + n_active++] = x;
       run += cnt[x];
     }
     expert_offset[E] = run;
-    for (uint32_t i = 0; i < S; ++i) {
-      const int32_t ex = topk_ids[i];
+    active[0] = n_active;
+    for (uint32_t i = 0; i < S; ++i) {   // slots of an expert in token order
+      const int32_t ex = ids[i];
       uint32_t slot = 0xFFFFFFFFu;
       if (ex >= 0 && (uint32_t)ex < E) {
         slot = cursor[ex]++;
@@ -509,7 +516,8 @@ namespace {
 
 struct FfnPlan {
   uint32_t S, groups, n_warps, smem, splits_gu, splits_dn;
-  uint64_t off_offsets, off_slot_token, off_slot_of, off_gu, off_h, off_y, total;
+  uint64_t off_offsets, off_active, off_slot_token, off_slot_of, off_gu, off_h, off_y, total;
+  uint32_t max_active;
 };
 
 // K splits so that the CTAs of the busiest plausible case fill the GPU a few times over:
@@ -537,6 +545,8 @@ zipmoe_status make_plan(uint32_t T, uint32_t k, const zipmoe_compressed_experts 
   auto up = [](uint64_t v) { return (v + 255) / 256 * 256; };
   uint64_t at = 0;
   p->off_offsets = at; at = up(at + 4ull * (ex->n_experts + 1));
+  p->off_active = at; at = up(at + 4ull * (ex->n_experts + 1));
+  p->max_active = active;
   p->off_slot_token = at; at = up(at + 4ull * p->S);
   p->off_slot_of = at; at = up(at + 4ull * p->S);
   p->off_gu = at; at = up(at + 2ull * p->splits_gu * p->S * ex->inter * 4);
@@ -590,6 +600,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   uint8_t *ws = static_cast<uint8_t *>(workspace);
   uint32_t *expert_offset = reinterpret_cast<uint32_t *>(ws + p.off_offsets);
+  uint32_t *active = reinterpret_cast<uint32_t *>(ws + p.off_active);
   uint32_t *slot_token = reinterpret_cast<uint32_t *>(ws + p.off_slot_token);
   uint32_t *slot_of = reinterpret_cast<uint32_t *>(ws + p.off_slot_of);
   float *gu = reinterpret_cast<float *>(ws + p.off_gu);
@@ -597,8 +608,8 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   float *y = reinterpret_cast<float *>(ws + p.off_y);
   const uint32_t E = ex->n_experts, H = ex->hidden, I = ex->inter, S = p.S;
 
-  route_kernel<<<1, 256, 2 * E * sizeof(uint32_t), stream>>>(topk_ids, S, k, E, 8 * p.groups, expert_offset, slot_token,
-                                                             slot_of, status_word);
+  route_kernel<<<1, 256, (2 * E + S) * sizeof(uint32_t), stream>>>(topk_ids, S, k, E, 8 * p.groups, expert_offset, active,
+                                                                   slot_token, slot_of, status_word);
 
   FfnArgs a;
   a.la.chunks = ex->chunks;
@@ -616,6 +627,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.la.tiles_per_cta = 0;
   a.tensor_first_chunk = ex->tensor_first_chunk;
   a.expert_offset = expert_offset;
+  a.active = active;
   a.n_warps = p.n_warps;
   a.groups = p.groups;
   a.S = S;
@@ -631,7 +643,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.tensor_base = 0;
   a.splits = p.splits_gu;
   a.steps_per_split = (H / 256 + p.splits_gu - 1) / p.splits_gu;
-  dim3 grid_gu((I / 16 + p.n_warps - 1) / p.n_warps, E, 2 * p.splits_gu);
+  dim3 grid_gu((I / 16 + p.n_warps - 1) / p.n_warps, p.max_active, 2 * p.splits_gu);
   ffn_matmul_kernel<<<grid_gu, threads, p.smem, stream>>>(a);
 
   const uint64_t n_h = (uint64_t)S * I;
@@ -647,7 +659,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.tensor_base = 2;
   a.splits = p.splits_dn;
   a.steps_per_split = (I / 256 + p.splits_dn - 1) / p.splits_dn;
-  dim3 grid_dn((H / 16 + p.n_warps - 1) / p.n_warps, E, p.splits_dn);
+  dim3 grid_dn((H / 16 + p.n_warps - 1) / p.n_warps, p.max_active, p.splits_dn);
   ffn_matmul_kernel<<<grid_dn, threads, p.smem, stream>>>(a);
 
   combine_kernel<<<dim3((H + 255) / 256, T), 256, 0, stream>>>(y, slot_of, topk_weights, T, k, S, H, p.splits_dn, out);
