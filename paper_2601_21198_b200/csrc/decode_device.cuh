@@ -114,9 +114,10 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
 // Returns the longest code length (0 for an invalid table).  An incomplete or
 // over-full code is reported and leaves zero entries in the holes: decoding
 // then yields garbage but stays in bounds.
-// lut_raw holds the lane table when the result is <= 8, the wide table otherwise.
+// lut_raw holds the lane table (u32 entries, or u16 entries when lane16) when the result is <= 8, the wide
+// table otherwise.
 __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint8_t *code_len, uint8_t *lut_raw,
-                                              uint8_t *scratch, uint32_t *status) {
+                                              uint8_t *scratch, uint32_t *status, const bool lane16 = false) {
   uint8_t *s_len = scratch;                                           // [256]
   uint32_t *s_first = reinterpret_cast<uint32_t *>(scratch + 256);    // [16] left-aligned 12-bit start of each length
   uint32_t *s_wcnt = s_first + 16;                                    // [8][16] per-warp symbol counts by length
@@ -188,8 +189,14 @@ __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint
   }
   __syncthreads();
   // replicate the 8-bit table once per lane
-  if (longest <= (uint32_t)kLaneLutBits)
-    for (uint32_t k = tid; k < (1u << kLaneLutBits) * 32; k += THREADS) lane_lut[k] = s_short[k >> 5];
+  if (longest <= (uint32_t)kLaneLutBits) {
+    if (lane16) {
+      uint16_t *lane_lut16 = reinterpret_cast<uint16_t *>(lut_raw);
+      for (uint32_t k = tid; k < (1u << kLaneLutBits) * 32; k += THREADS) lane_lut16[k] = (uint16_t)s_short[k >> 5];
+    } else {
+      for (uint32_t k = tid; k < (1u << kLaneLutBits) * 32; k += THREADS) lane_lut[k] = s_short[k >> 5];
+    }
+  }
   __syncthreads();
   return longest;
 }
@@ -337,8 +344,13 @@ __device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) 
 // bits 4..6 are zero, so the low 7 bits of pos stay exact and the rest is
 // ignored (the funnel shifts take the shift amount mod 32).  When bit 5 of pos
 // is set a whole word has been consumed and the next one is shifted in.
-template <bool STAGED, bool FAST>
+// KIND: kLutWide (12-bit shared table), kLutLane32 (8-bit table, one u32 copy per lane: no bank conflicts, 32 KB) or
+// kLutLane16 (8-bit table, one u16 copy per lane: two lanes share a bank, 16 KB).
+constexpr int kLutWide = 0, kLutLane32 = 1, kLutLane16 = 2;
+
+template <bool STAGED, int KIND>
 struct LaneDecoder {
+  static constexpr bool FAST = KIND != kLutWide;
   WordSource<STAGED> src;
   uint32_t pos, b_hi, b_lo, lut, my_lut;
 
@@ -366,11 +378,12 @@ struct LaneDecoder {
     b_hi = src.pop();
     b_lo = src.pop();
     lut = lut_addr;
-    my_lut = lut_addr + 4 * lane;
+    my_lut = lut_addr + (KIND == kLutLane16 ? 2 : 4) * lane;
     return true;
   }
   __device__ __forceinline__ uint32_t lookup(uint32_t w) const {   // (symbol << 7) | length of the code at the top of w
-    if (FAST) return lds_u32(mad_u32(w >> (32 - kLaneLutBits), 128u, my_lut));
+    if (KIND == kLutLane32) return lds_u32(mad_u32(w >> (32 - kLaneLutBits), 128u, my_lut));
+    if (KIND == kLutLane16) return lds_u16(mad_u32(w >> (32 - kLaneLutBits), 64u, my_lut));
     return lds_u16(mad_u32(w >> (32 - kWideLutBits), 2u, lut));
   }
   __device__ __forceinline__ void pair(uint32_t &ea, uint32_t &eb) {   // two codes from the 32 bits at pos
@@ -436,7 +449,7 @@ template <bool STAGED, bool FAST, class Feed, class Sink>
 __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *rec_g, uint32_t rec_bytes,
                                                 uint32_t lut, uint32_t valid, uint32_t iters,
                                                 uint32_t lane, Feed &feed, Sink &sink) {
-  LaneDecoder<STAGED, FAST> dec;
+  LaneDecoder<STAGED, FAST ? kLutLane32 : kLutWide> dec;
   if (!dec.init(rec_s, rec_g, rec_bytes, lut, lane)) return kStatusBadBitCount;
   auto group = [&](uint32_t sm_at) -> uint4 { return dec.group(lds_v2(sm_at)); };
   auto single = [&]() -> uint32_t { return dec.single(); };

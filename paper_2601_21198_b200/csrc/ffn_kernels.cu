@@ -39,13 +39,19 @@
 
 namespace zipmoe_dev {
 
-constexpr int kFfnMaxWarps = 16;                         // decode warps per CTA, a multiple of 4 (plus loader and MMA warps)
-constexpr int kFfnMaxThreads = (kFfnMaxWarps + 2) * 32;
+#ifndef ZIPMOE_FFN_WARPS
+#define ZIPMOE_FFN_WARPS 16
+#endif
+constexpr int kFfnMaxWarps = ZIPMOE_FFN_WARPS;                         // decode warps per CTA, a multiple of 4 (plus loader and MMA warps)
+constexpr int kGroupWarps = 8;                           // decode warps whose half-tiles form one M = 64 operand
+constexpr int kFfnMaxThreads = (kFfnMaxWarps + kFfnMaxWarps / kGroupWarps + 1) * 32;   // decode, one MMA warp per group, loader
 constexpr uint32_t kBLbo = 144;                          // bytes between the 8x8 cores of a half-tile along K: 128 + 16 of
                                                          // padding, so that the 32 lanes' 16-byte stores spread over all banks
 constexpr uint32_t kBBufBytes = 32 * kBLbo;              // one half-tile: 8 rows x 256 columns
 constexpr uint32_t kXGroupBytes = 4096;                  // 8 token rows x 256 columns of bf16, cores 128 bytes apart
 constexpr uint32_t kFfnWarpBytes = 2 * kPayStage + kBBufBytes;   // two record stages, one half-tile buffer
+constexpr uint32_t kFfnLutBytes = kLaneLutBytes / 2;     // u16 lane table (two lanes per bank): the fused kernel spends its
+                                                         // shared memory on decode warps rather than on the table
 constexpr uint32_t kFfnShortTries = 1u << 10;            // wait limit once something has already gone wrong
 
 struct FfnArgs {
@@ -64,13 +70,11 @@ struct FfnArgs {
 };
 
 // shared-memory layout: [X stages][per-warp buffers][tables][table scratch][barriers][tmem slot]
-__host__ __device__ inline uint32_t ffn_bar_count(uint32_t n_warps) { return 2 * n_warps + 2 * (n_warps / 4) + 4; }
+__host__ __device__ inline uint32_t ffn_bar_count(uint32_t n_warps) {
+  return 2 * n_warps + 2 * (n_warps / kGroupWarps) + 4;
+}
 __host__ __device__ inline uint32_t ffn_smem_bytes(uint32_t n_warps, uint32_t groups) {
-  uint32_t after_warps = kLutBytes + kLutScratchBytes + ffn_bar_count(n_warps) * 8 + 16;
-  // the A operand of the last quad reads 8 groups kFfnWarpBytes apart: 4 real ones and 4 more that must
-  // still lie inside the allocation
-  const uint32_t overrun = 4 * kFfnWarpBytes;
-  if (after_warps < overrun) after_warps = overrun;
+  const uint32_t after_warps = kFfnLutBytes + kLutScratchBytes + ffn_bar_count(n_warps) * 8 + 16;
   return 2 * groups * kXGroupBytes + n_warps * kFfnWarpBytes + after_warps;
 }
 
@@ -106,7 +110,7 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
 
 __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const FfnArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  const uint32_t NW = a.n_warps, G = a.groups, Q = NW >> 2, NCOL = 8 * G;
+  const uint32_t NW = a.n_warps, G = a.groups, Q = NW / kGroupWarps, NCOL = 8 * G;
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (blockIdx.y >= __ldg(a.active)) return;   // fewer experts have tokens than the grid allows for
   const uint32_t e = __ldg(a.active + 1 + blockIdx.y), z = blockIdx.z;
@@ -121,7 +125,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   uint8_t *x_raw = smem;                                   // [2][G][4096]
   uint8_t *warp_raw = x_raw + 2 * G * kXGroupBytes;        // [NW][2 record stages | half-tile buffer]
   uint8_t *lut_raw = warp_raw + NW * kFfnWarpBytes;
-  uint8_t *lut_scratch = lut_raw + kLutBytes;
+  uint8_t *lut_scratch = lut_raw + kFfnLutBytes;
   uint64_t *bars = reinterpret_cast<uint64_t *>(lut_scratch + kLutScratchBytes);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + ffn_bar_count(NW));
   // barriers: [NW][2] record stages, [Q] quad half written, [Q] quad MMAs done, [2] X full, [2] X empty
@@ -129,7 +133,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   const uint32_t quad_full = bar0 + 8 * (2 * NW), quad_done = quad_full + 8 * Q;
   const uint32_t x_full = quad_done + 8 * Q, x_empty = x_full + 16;
   const uint32_t x_addr = smem_addr(x_raw), lut = smem_addr(lut_raw);
-  const bool is_loader = warp == NW, is_mma = warp == NW + 1, is_decode = warp < NW;
+  const bool is_decode = warp < NW, is_mma = warp >= NW && warp < NW + Q, is_loader = warp == NW + Q;
 
   const uint32_t n_strips = a.rows >> 4, strip = blockIdx.x * NW + warp;
   const bool has_strip = is_decode && strip < n_strips;
@@ -143,13 +147,13 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   if (tid == 0) {
     for (uint32_t b = 0; b < 2 * NW; ++b) mbar_init(bar0 + 8 * b, 1);
     for (uint32_t q = 0; q < Q; ++q) {
-      mbar_init(quad_full + 8 * q, 4);
+      mbar_init(quad_full + 8 * q, kGroupWarps);
       mbar_init(quad_done + 8 * q, 1);
     }
     mbar_init(x_full, 1);
     mbar_init(x_full + 8, 1);
-    mbar_init(x_empty, 1);
-    mbar_init(x_empty + 8, 1);
+    mbar_init(x_empty, Q);
+    mbar_init(x_empty + 8, Q);
   }
   fence_barrier_init();
   if (warp == 0) {
@@ -165,7 +169,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
 
   // the tensor: blocked layout, 16 x 256 tiles, one Huffman table
   const uint32_t c0 = __ldg(a.tensor_first_chunk + tensor);
-  bool ok = c0 < a.la.n_chunks && 2 * Q * NCOL <= 512 && 4 * Q == NW;
+  bool ok = c0 < a.la.n_chunks && 2 * Q * NCOL <= 512 && kGroupWarps * Q == NW;
   uint32_t table_id = 0, tpc = 1;
   if (ok) {
     const zipmoe_chunk_desc *d = a.la.chunks + c0;
@@ -177,7 +181,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   }
   if (!ok) report(a.la.status, kStatusBadDescriptor);
   bool fast = true;
-  if (ok) fast = build_lut(blockDim.x, a.la.tables[table_id].code_len, lut_raw, lut_scratch, a.la.status) <=
+  if (ok) fast = build_lut(blockDim.x, a.la.tables[table_id].code_len, lut_raw, lut_scratch, a.la.status, true) <=
                  (uint32_t)kLaneLutBits;
   // (build_lut ends with a CTA barrier)
 
@@ -211,42 +215,41 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
       if (lane == 0) mbar_arrive(x_full + 8 * b);
     }
   } else if (ok && is_mma) {
-    // ---- one lane issues, per half-tile and quad: D[64 x N] (+)= A[64 x 256] * X[N x 256]^T ----
+    // ---- one MMA warp per quad; one lane issues, per half-tile: D[64 x N] (+)= A[64 x 256] * X[N x 256]^T ----
     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (G << 17) | (4u << 24);   // bf16 x bf16 -> fp32, N = 8G, M = 64
-    const uint32_t buf0 = smem_addr(warp_raw) + 2 * kPayStage;
+    const uint32_t q = warp - NW;
+    const uint32_t abuf = smem_addr(warp_raw) + 2 * kPayStage + kGroupWarps * q * kFfnWarpBytes;
+    const uint64_t a_desc0 = smem_desc(abuf, kBLbo, kFfnWarpBytes);
     bool alive = true;
     for (uint32_t s = 0; s < n_steps && alive; ++s) {
-      const uint32_t xb = s & 1, xs = x_addr + xb * G * kXGroupBytes;
+      const uint32_t xb = s & 1;
+      const uint64_t b_desc0 = smem_desc(x_addr + xb * G * kXGroupBytes, 128, kXGroupBytes);
       if (!mbar_wait_bounded(x_full + 8 * xb, (s >> 1) & 1)) alive = false;
       for (uint32_t half = 0; half < 2 && alive; ++half) {
         const uint32_t hn = 2 * s + half;
-        for (uint32_t q = 0; q < Q && alive; ++q) {
-          if (!mbar_wait_bounded(quad_full + 8 * q, hn & 1)) {
-            alive = false;
-            break;
-          }
-          if (lane == 0) {
-            tc_fence_after();
-            const uint32_t abuf = buf0 + 4 * q * kFfnWarpBytes;
-            const uint32_t d_tmem = tmem + (2 * q + half) * NCOL;
-#pragma unroll
-            for (uint32_t j = 0; j < 16; ++j)
-              mma_bf16(d_tmem, smem_desc(abuf + j * 2 * kBLbo, kBLbo, kFfnWarpBytes),
-                       smem_desc(xs + j * 256, 128, kXGroupBytes), idesc, (s > 0 || j > 0) ? 1u : 0u);
-            mma_commit(quad_done + 8 * q);
-          }
-          __syncwarp();
+        if (!mbar_wait_bounded(quad_full + 8 * q, hn & 1)) {
+          alive = false;
+          break;
         }
+        if (lane == 0) {
+          tc_fence_after();
+          const uint32_t d_tmem = tmem + (2 * q + half) * NCOL;
+          // the K slice j of an operand starts 2 cores further: the start-address field counts 16-byte units
+#pragma unroll
+          for (uint32_t j = 0; j < 16; ++j)
+            mma_bf16(d_tmem, a_desc0 + j * (2 * kBLbo / 16), b_desc0 + j * (256 / 16), idesc, (s > 0 || j > 0) ? 1u : 0u);
+          mma_commit(quad_done + 8 * q);
+          if (half == 1) mma_commit(x_empty + 8 * xb);   // this quad is done with the X stage
+        }
+        __syncwarp();
       }
-      if (alive && lane == 0) mma_commit(x_empty + 8 * xb);   // every MMA that reads this X stage has been issued
-      __syncwarp();
     }
     if (!alive) report(a.la.status, kStatusWaitTimeout);
   } else if (ok && is_decode) {
     // ---- one strip of 16 rows: decode tile after tile along K, hand half-tiles to the quad's A operand ----
     const uint32_t my = smem_addr(warp_raw + warp * kFfnWarpBytes);
     const uint32_t buf = my + 2 * kPayStage;
-    const uint32_t rec_bar = bar0 + 8 * (2 * warp), q = warp >> 2;
+    const uint32_t rec_bar = bar0 + 8 * (2 * warp), q = warp / kGroupWarps;
     uint32_t rec_phase = 0, hn = 0;
     bool failed = !has_strip || n_steps == 0;
 
@@ -345,7 +348,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
         }
         // both halves of the tile, for every combination of record location and table kind
         auto run = [&](auto staged_c, auto fast_c) -> bool {
-          LaneDecoder<decltype(staged_c)::value, decltype(fast_c)::value> dec;
+          LaneDecoder<decltype(staged_c)::value, decltype(fast_c)::value ? kLutLane16 : kLutWide> dec;
           if (!dec.init(my + stage * kPayStage, cur.rec, cur.rec_bytes, lut, lane)) {
             report(a.la.status, kStatusBadBitCount);
             buffer_free();
@@ -405,12 +408,12 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (ok && warp < 2 && n_steps) {
-    // With M = 64, D row 16j + i sits in tensor-memory lane 32j + i (i < 16): warp 0 reads rows 0..15 (the halves
-    // of the quad's warps 0 and 1), warp 1 rows 16..31 (warps 2 and 3); rows 32..63 are not used.
-    const uint32_t wq = 2 * warp + ((lane >> 3) & 1), r = lane & 7;
+  if (ok && warp < 4 && n_steps) {
+    // With M = 64, D row 16j + i sits in tensor-memory lane 32j + i (i < 16): warp j reads rows 16j..16j+15,
+    // the halves of the group's warps 2j and 2j + 1.
+    const uint32_t wg = 2 * warp + ((lane >> 3) & 1), r = lane & 7;
     for (uint32_t q = 0; q < Q; ++q) {
-      const uint32_t st = blockIdx.x * NW + 4 * q + wq;
+      const uint32_t st = blockIdx.x * NW + kGroupWarps * q + wg;
       for (uint32_t half = 0; half < 2; ++half) {
         const uint32_t row = 16 * st + 8 * half + r;
         for (uint32_t c = 0; c < G; ++c) {
@@ -535,7 +538,7 @@ zipmoe_status make_plan(uint32_t T, uint32_t k, const zipmoe_compressed_experts 
   p->S = T * k;
   p->groups = (T + 7) / 8;
   uint32_t nw = zipmoe_dev::kFfnMaxWarps;
-  while (nw > 8 && zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) nw -= 4;   // the table builder needs 256 threads
+  while (nw > 8 && zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) nw -= zipmoe_dev::kGroupWarps;
   if (zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) return ZIPMOE_ERR_UNSUPPORTED;
   p->n_warps = nw;
   p->smem = zipmoe_dev::ffn_smem_bytes(nw, p->groups);
@@ -632,7 +635,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.groups = p.groups;
   a.S = S;
   a.smem_bytes = p.smem;
-  const uint32_t threads = (p.n_warps + 2) * 32;
+  const uint32_t threads = (p.n_warps + p.n_warps / zipmoe_dev::kGroupWarps + 1) * 32;
 
   // gate and up: partial Y[matrix][split] = W_{1,3}[:, split] X[:, split]
   a.slot_token = slot_token;
