@@ -43,7 +43,11 @@ namespace zipmoe_dev {
 #define ZIPMOE_FFN_WARPS 16
 #endif
 constexpr int kFfnMaxWarps = ZIPMOE_FFN_WARPS;                         // decode warps per CTA, a multiple of 4 (plus loader and MMA warps)
-constexpr int kGroupWarps = 8;                           // decode warps whose half-tiles form one M = 64 operand
+#ifndef ZIPMOE_FFN_GROUP
+#define ZIPMOE_FFN_GROUP 8
+#endif
+constexpr int kGroupWarps = ZIPMOE_FFN_GROUP;            // decode warps whose half-tiles form one operand of M = 8 * kGroupWarps (64 or 128)
+static_assert(kGroupWarps == 8 || kGroupWarps == 16, "M is 64 or 128");
 constexpr int kFfnMaxThreads = (kFfnMaxWarps + kFfnMaxWarps / kGroupWarps + 1) * 32;   // decode, one MMA warp per group, loader
 constexpr uint32_t kBLbo = 144;                          // bytes between the 8x8 cores of a half-tile along K: 128 + 16 of
                                                          // padding, so that the 32 lanes' 16-byte stores spread over all banks
@@ -216,7 +220,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
     }
   } else if (ok && is_mma) {
     // ---- one MMA warp per quad; one lane issues, per half-tile: D[64 x N] (+)= A[64 x 256] * X[N x 256]^T ----
-    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (G << 17) | (4u << 24);   // bf16 x bf16 -> fp32, N = 8G, M = 64
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (G << 17) | ((uint32_t)(kGroupWarps / 2) << 24);   // bf16 x bf16 -> fp32, N = 8G, M = 8 * kGroupWarps
     const uint32_t q = warp - NW;
     const uint32_t abuf = smem_addr(warp_raw) + 2 * kPayStage + kGroupWarps * q * kFfnWarpBytes;
     const uint64_t a_desc0 = smem_desc(abuf, kBLbo, kFfnWarpBytes);
@@ -411,7 +415,9 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   if (ok && warp < 4 && n_steps) {
     // With M = 64, D row 16j + i sits in tensor-memory lane 32j + i (i < 16): warp j reads rows 16j..16j+15,
     // the halves of the group's warps 2j and 2j + 1.
-    const uint32_t wg = 2 * warp + ((lane >> 3) & 1), r = lane & 7;
+    // With M = 128, D row r sits in lane r: warp j reads rows 32j..32j+31, the halves of warps 4j..4j+3.
+    const uint32_t wg = kGroupWarps == 8 ? 2 * warp + ((lane >> 3) & 1) : 4 * warp + (lane >> 3), r = lane & 7;
+    const uint32_t live_lanes = kGroupWarps == 8 ? 16 : 32;
     for (uint32_t q = 0; q < Q; ++q) {
       const uint32_t st = blockIdx.x * NW + kGroupWarps * q + wg;
       for (uint32_t half = 0; half < 2; ++half) {
@@ -424,7 +430,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
                        : "r"(taddr)
                        : "memory");
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-          if (lane < 16 && st < n_strips) {
+          if (lane < live_lanes && st < n_strips) {
 #pragma unroll
             for (uint32_t n = 0; n < 8; ++n) {
               const uint32_t tokrow = 8 * c + n;
@@ -538,7 +544,8 @@ zipmoe_status make_plan(uint32_t T, uint32_t k, const zipmoe_compressed_experts 
   p->S = T * k;
   p->groups = (T + 7) / 8;
   uint32_t nw = zipmoe_dev::kFfnMaxWarps;
-  while (nw > 8 && zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) nw -= zipmoe_dev::kGroupWarps;
+  while (nw > (uint32_t)zipmoe_dev::kGroupWarps && zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u)
+    nw -= zipmoe_dev::kGroupWarps;
   if (zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) return ZIPMOE_ERR_UNSUPPORTED;
   p->n_warps = nw;
   p->smem = zipmoe_dev::ffn_smem_bytes(nw, p->groups);
