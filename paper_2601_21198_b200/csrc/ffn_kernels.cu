@@ -77,8 +77,8 @@ struct FfnArgs {
 __host__ __device__ inline uint32_t ffn_bar_count(uint32_t n_warps) {
   return 2 * n_warps + 2 * (n_warps / kGroupWarps) + 4;
 }
-__host__ __device__ inline uint32_t ffn_smem_bytes(uint32_t n_warps, uint32_t groups) {
-  const uint32_t after_warps = kFfnLutBytes + kLutScratchBytes + ffn_bar_count(n_warps) * 8 + 16;
+__host__ __device__ inline uint32_t ffn_smem_bytes(uint32_t n_warps, uint32_t groups, bool lane16) {
+  const uint32_t after_warps = (lane16 ? kFfnLutBytes : (uint32_t)kLutBytes) + kLutScratchBytes + ffn_bar_count(n_warps) * 8 + 16;
   return 2 * groups * kXGroupBytes + n_warps * kFfnWarpBytes + after_warps;
 }
 
@@ -87,6 +87,12 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 __device__ __forceinline__ void sts_v4(uint32_t addr, const uint4 &v) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+// ordered with the other volatile asm of the decoder, so the load is issued where it is written: early
+__device__ __forceinline__ uint2 ldg_v2_early(const uint8_t *p) {
+  uint2 v;
+  asm volatile("ld.global.nc.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+  return v;
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -112,7 +118,9 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+template <bool LANE16>
 __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const FfnArgs a) {
+  constexpr uint32_t kMyLutBytes = LANE16 ? kFfnLutBytes : kLutBytes;
   extern __shared__ __align__(128) uint8_t smem[];
   const uint32_t NW = a.n_warps, G = a.groups, Q = NW / kGroupWarps, NCOL = 8 * G;
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -129,7 +137,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   uint8_t *x_raw = smem;                                   // [2][G][4096]
   uint8_t *warp_raw = x_raw + 2 * G * kXGroupBytes;        // [NW][2 record stages | half-tile buffer]
   uint8_t *lut_raw = warp_raw + NW * kFfnWarpBytes;
-  uint8_t *lut_scratch = lut_raw + kFfnLutBytes;
+  uint8_t *lut_scratch = lut_raw + kMyLutBytes;
   uint64_t *bars = reinterpret_cast<uint64_t *>(lut_scratch + kLutScratchBytes);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + ffn_bar_count(NW));
   // barriers: [NW][2] record stages, [Q] quad half written, [Q] quad MMAs done, [2] X full, [2] X empty
@@ -185,7 +193,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   }
   if (!ok) report(a.la.status, kStatusBadDescriptor);
   bool fast = true;
-  if (ok) fast = build_lut(blockDim.x, a.la.tables[table_id].code_len, lut_raw, lut_scratch, a.la.status, true) <=
+  if (ok) fast = build_lut(blockDim.x, a.la.tables[table_id].code_len, lut_raw, lut_scratch, a.la.status, LANE16) <=
                  (uint32_t)kLaneLutBits;
   // (build_lut ends with a CTA barrier)
 
@@ -319,7 +327,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
       cur = tile(0);
       if (cur.staged && lane == 0) bulk_load(my, cur.rec, cur.rec_bytes, rec_bar);
 #pragma unroll
-      for (int k = 0; k < 8; ++k) smA[k] = __ldg(reinterpret_cast<const uint2 *>(cur.sm + k * 256) + lane);
+      for (int k = 0; k < 8; ++k) smA[k] = ldg_v2_early(cur.sm + k * 256 + lane * 8);
     }
     // hand-over of one half in two moves: before the first store, wait until the MMAs of the previous half have
     // read the buffer; after the last store, make the stores visible to the tensor core and tell the MMA warp
@@ -352,7 +360,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
         }
         // both halves of the tile, for every combination of record location and table kind
         auto run = [&](auto staged_c, auto fast_c) -> bool {
-          LaneDecoder<decltype(staged_c)::value, decltype(fast_c)::value ? kLutLane16 : kLutWide> dec;
+          LaneDecoder<decltype(staged_c)::value, !decltype(fast_c)::value ? kLutWide : LANE16 ? kLutLane16 : kLutLane32> dec;
           if (!dec.init(my + stage * kPayStage, cur.rec, cur.rec_bytes, lut, lane)) {
             report(a.la.status, kStatusBadBitCount);
             buffer_free();
@@ -362,7 +370,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
             return false;
           }
 #pragma unroll
-          for (int k = 0; k < 8; ++k) smB[k] = __ldg(reinterpret_cast<const uint2 *>(cur.sm + (8 + k) * 256) + lane);
+          for (int k = 0; k < 8; ++k) smB[k] = ldg_v2_early(cur.sm + (8 + k) * 256 + lane * 8);
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             // the first four iterations are decoded into registers while the previous half's MMAs may still run
@@ -381,7 +389,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
             for (int k = 4; k < 8; ++k) sts_v4(buf + lane * kBLbo + k * 16, dec.group(half ? smB[k] : smA[k]));
             if (half == 0 && have_next) {
 #pragma unroll
-              for (int k = 0; k < 8; ++k) smA[k] = __ldg(reinterpret_cast<const uint2 *>(nxt.sm + k * 256) + lane);
+              for (int k = 0; k < 8; ++k) smA[k] = ldg_v2_early(nxt.sm + k * 256 + lane * 8);
             }
             publish();
           }
@@ -525,6 +533,7 @@ namespace {
 
 struct FfnPlan {
   uint32_t S, groups, n_warps, smem, splits_gu, splits_dn;
+  bool lane16;
   uint64_t off_offsets, off_active, off_slot_token, off_slot_of, off_gu, off_h, off_y, total;
   uint32_t max_active;
 };
@@ -543,12 +552,14 @@ zipmoe_status make_plan(uint32_t T, uint32_t k, const zipmoe_compressed_experts 
   if (ex->hidden == 0 || ex->inter == 0 || ex->hidden % 256 || ex->inter % 256) return ZIPMOE_ERR_UNSUPPORTED;
   p->S = T * k;
   p->groups = (T + 7) / 8;
+  // as many decode warps as fit; the 32 KB conflict-free table if it still fits beside them, else the 16 KB one
   uint32_t nw = zipmoe_dev::kFfnMaxWarps;
-  while (nw > (uint32_t)zipmoe_dev::kGroupWarps && zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u)
+  p->lane16 = zipmoe_dev::ffn_smem_bytes(nw, p->groups, false) > 227u * 1024u;
+  while (nw > (uint32_t)zipmoe_dev::kGroupWarps && zipmoe_dev::ffn_smem_bytes(nw, p->groups, p->lane16) > 227u * 1024u)
     nw -= zipmoe_dev::kGroupWarps;
-  if (zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) return ZIPMOE_ERR_UNSUPPORTED;
+  if (zipmoe_dev::ffn_smem_bytes(nw, p->groups, p->lane16) > 227u * 1024u) return ZIPMOE_ERR_UNSUPPORTED;
   p->n_warps = nw;
-  p->smem = zipmoe_dev::ffn_smem_bytes(nw, p->groups);
+  p->smem = zipmoe_dev::ffn_smem_bytes(nw, p->groups, p->lane16);
   const uint32_t active = p->S < ex->n_experts ? p->S : ex->n_experts;   // at most this many experts get tokens
   p->splits_gu = pick_splits(active * 2 * ((ex->inter / 16 + nw - 1) / nw), ex->hidden / 256);
   p->splits_dn = pick_splits(active * ((ex->hidden / 16 + nw - 1) / nw), ex->inter / 256);
@@ -603,7 +614,10 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
     int major = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ZIPMOE_ERR_CUDA;
     if (major != 10) return ZIPMOE_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(ffn_matmul_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(ffn_matmul_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(ffn_matmul_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaSuccess)
       return ZIPMOE_ERR_CUDA;
     g_ffn_ready[dev] = true;
   }
@@ -654,7 +668,8 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.splits = p.splits_gu;
   a.steps_per_split = (H / 256 + p.splits_gu - 1) / p.splits_gu;
   dim3 grid_gu((I / 16 + p.n_warps - 1) / p.n_warps, p.max_active, 2 * p.splits_gu);
-  ffn_matmul_kernel<<<grid_gu, threads, p.smem, stream>>>(a);
+  if (p.lane16) ffn_matmul_kernel<true><<<grid_gu, threads, p.smem, stream>>>(a);
+  else ffn_matmul_kernel<false><<<grid_gu, threads, p.smem, stream>>>(a);
 
   const uint64_t n_h = (uint64_t)S * I;
   const unsigned act_blocks = (unsigned)((n_h + 1023) / 1024 < 592 ? (n_h + 1023) / 1024 : 592);
@@ -670,7 +685,8 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.splits = p.splits_dn;
   a.steps_per_split = (I / 256 + p.splits_dn - 1) / p.splits_dn;
   dim3 grid_dn((H / 16 + p.n_warps - 1) / p.n_warps, p.max_active, p.splits_dn);
-  ffn_matmul_kernel<<<grid_dn, threads, p.smem, stream>>>(a);
+  if (p.lane16) ffn_matmul_kernel<true><<<grid_dn, threads, p.smem, stream>>>(a);
+  else ffn_matmul_kernel<false><<<grid_dn, threads, p.smem, stream>>>(a);
 
   combine_kernel<<<dim3((H + 255) / 256, T), 256, 0, stream>>>(y, slot_of, topk_weights, T, k, S, H, p.splits_dn, out);
   return cudaGetLastError() == cudaSuccess ? ZIPMOE_OK : ZIPMOE_ERR_CUDA;
