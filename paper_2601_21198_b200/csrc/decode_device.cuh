@@ -208,6 +208,7 @@ struct TileWork {
   uint16_t *out;        // global address of the tile's first element
   uint32_t rec_bytes, pitch, valid, iters, pieces;
   bool ok, staged;
+  bool wide;            // staged across both record stages (a record of up to 2 * kPayStage - kPaySlack bytes)
 };
 
 struct LaunchArgs {
@@ -244,6 +245,7 @@ __device__ inline TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_
   TileWork w;
   w.ok = false;
   w.staged = false;
+  w.wide = false;
   if (c >= a.n_chunks) return w;
   const uint4 *d = reinterpret_cast<const uint4 *>(a.chunks + c);
   const uint4 d0 = __ldg(d), d1 = __ldg(d + 1), d2 = __ldg(d + 2), d3 = __ldg(d + 3);
@@ -278,7 +280,8 @@ __device__ inline TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_
   w.sm = a.sm + sm_tile;
   w.out = a.out + origin;
   w.pitch = pitch;
-  w.staged = w.rec_bytes <= kPayBuf;
+  w.wide = w.rec_bytes > (uint32_t)kPayBuf && w.rec_bytes <= (uint32_t)(2 * kPayStage - kPaySlack);
+  w.staged = w.rec_bytes <= (uint32_t)kPayBuf || w.wide;
   w.ok = true;
   return w;
 }

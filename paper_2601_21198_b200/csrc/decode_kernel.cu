@@ -52,8 +52,11 @@ struct WarpPipe {
     return true;
   }
   // all lanes call these; one lane starts the copy
+  // a record of ordinary size goes into `stage`; a wide one (8-bit codes everywhere: 4160 bytes) spans both
+  // stages and uses the first stage's barrier, so no other record can be in flight beside it
   __device__ __forceinline__ void load_record(const TileWork &t, uint32_t stage) {
     if (!t.staged) return;
+    if (t.wide) stage = 0;
     if (lane == 0) bulk_load(pay_addr + stage * kPayStage, t.rec, t.rec_bytes, bar(stage));
     pending |= 1u << stage;
   }
@@ -170,13 +173,16 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
         step();
         nxt = resolve_tile(a, tc, tt);
         if (!nxt.ok) report(a.status, kStatusBadDescriptor);
-        else pipe.load_record(nxt, stage ^ 1);   // that stage was released by the __syncwarp below
       }
+      // the next record is fetched while this one is decoded, unless one of the two needs both stages
+      const bool prefetch = nxt.ok && !nxt.wide && !(cur.ok && cur.wide);
+      if (prefetch) pipe.load_record(nxt, stage ^ 1);   // that stage was released by the __syncwarp below
       if (cur.ok) {
         uint32_t rc = 0;
-        if (cur.staged && !pipe.wait(stage)) rc = kStatusWaitTimeout;
+        const uint32_t rec_stage = cur.wide ? 0 : stage;
+        if (cur.staged && !pipe.wait(rec_stage)) rc = kStatusWaitTimeout;
         if (rc == 0) {
-          const uint32_t rec_s = pipe.pay_addr + stage * kPayStage;
+          const uint32_t rec_s = pipe.pay_addr + rec_stage * kPayStage;
           SmFeed feed{pipe, nxt, nxt_issued};
           GlobalSink sink{cur.out, cur.pitch};
           if (cur.staged) {
@@ -210,6 +216,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
         }
       }
       __syncwarp();   // every lane is done with the current record stage and SM slots
+      if (nxt.ok && !prefetch) pipe.load_record(nxt, stage ^ 1);
       if (nxt.ok)
         for (; nxt_issued < nxt.pieces; ++nxt_issued) pipe.load_sm_piece(nxt, nxt_issued);
       cur = nxt;
