@@ -131,7 +131,9 @@ typedef struct {
   uint32_t run_first_tile;  /* tile_prefix of that descriptor                                      */
   uint32_t run_end_tile;    /* tile_prefix + n_tiles of the run's last descriptor                  */
   uint32_t tiles_per_chunk; /* tiles in every chunk of the run but possibly the last               */
-  uint32_t reserved[2];     /* zero; pads the descriptor to 80 bytes (five 16-byte loads)          */
+  uint32_t max_record_bytes;/* largest tile record of the run, in bytes (0 = unknown); a hint that lets the
+                               kernel skip its wide-record handling for tensors that never need it  */
+  uint32_t reserved;        /* zero; pads the descriptor to 80 bytes (five 16-byte loads)          */
 } zipmoe_chunk_desc;
 
 typedef struct {

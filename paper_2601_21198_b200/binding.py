@@ -46,7 +46,7 @@ CHUNK_DESC_DTYPE = np.dtype([
     ("payload_off", "<u8"), ("sm_off", "<u8"), ("out_off", "<u8"), ("row_pitch", "<u4"), ("tiles_per_rowblk", "<u4"),
     ("tile0", "<u4"), ("n_tiles", "<u4"), ("tile_elems", "<u4"), ("last_tile_elems", "<u4"), ("table_id", "<u4"),
     ("tile_prefix", "<u4"), ("run_first_chunk", "<u4"), ("run_first_tile", "<u4"), ("run_end_tile", "<u4"),
-    ("tiles_per_chunk", "<u4"), ("reserved", "<u4", (2,))], align=True)
+    ("tiles_per_chunk", "<u4"), ("max_record_bytes", "<u4"), ("reserved", "<u4")], align=True)
 assert CHUNK_DESC_DTYPE.itemsize == 80
 TABLE_BYTES = 256
 

@@ -241,7 +241,7 @@ static_assert(sizeof(zipmoe_chunk_desc) == 80, "descriptor is read as five 16-by
 
 // Everything the decoder needs about tile t of descriptor c, with every offset
 // checked against the sizes of the buffers the launch was given.
-__device__ inline TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_t t) {
+__device__ inline TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_t t, const bool allow_wide = false) {
   TileWork w;
   w.ok = false;
   w.staged = false;
@@ -280,7 +280,7 @@ __device__ inline TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_
   w.sm = a.sm + sm_tile;
   w.out = a.out + origin;
   w.pitch = pitch;
-  w.wide = w.rec_bytes > (uint32_t)kPayBuf && w.rec_bytes <= (uint32_t)(2 * kPayStage - kPaySlack);
+  w.wide = allow_wide && w.rec_bytes > (uint32_t)kPayBuf && w.rec_bytes <= (uint32_t)(2 * kPayStage - kPaySlack);
   w.staged = w.rec_bytes <= (uint32_t)kPayBuf || w.wide;
   w.ok = true;
   return w;

@@ -17,6 +17,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <type_traits>
 
 #include "zipmoe.h"
 #include "decode_device.cuh"
@@ -143,6 +144,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
     const bool fast = build_lut(kThreads, a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <=
                       (uint32_t)kLaneLutBits;
 
+    // Tensors whose largest record fits one record stage (all but near-incompressible ones) never take the
+    // wide-record branches below.
+#ifndef ZIPMOE_WIDE_STAGING
+#define ZIPMOE_WIDE_STAGING 1
+#endif
+    const bool wide_seg = ZIPMOE_WIDE_STAGING && __ldg(&d->max_record_bytes) > (uint32_t)kPayBuf;
     uint32_t g = g0 + warp;
     uint32_t stage = 0;
     // descriptor and tile-in-chunk of this warp's next tile, stepped without divisions
@@ -157,7 +164,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
     TileWork cur;
     cur.ok = false;
     if (g < seg_end && !dead) {
-      cur = resolve_tile(a, tc, tt);
+      cur = resolve_tile(a, tc, tt, wide_seg);
       if (!cur.ok) report(a.status, kStatusBadDescriptor);
       else {
         pipe.load_record(cur, stage);
@@ -171,15 +178,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
       const uint32_t g2 = g + kWarps;
       if (g2 < seg_end) {
         step();
-        nxt = resolve_tile(a, tc, tt);
+        nxt = resolve_tile(a, tc, tt, wide_seg);
         if (!nxt.ok) report(a.status, kStatusBadDescriptor);
       }
       // the next record is fetched while this one is decoded, unless one of the two needs both stages
-      const bool prefetch = nxt.ok && !nxt.wide && !(cur.ok && cur.wide);
+      const bool prefetch = nxt.ok && (!wide_seg || (!nxt.wide && !(cur.ok && cur.wide)));
       if (prefetch) pipe.load_record(nxt, stage ^ 1);   // that stage was released by the __syncwarp below
       if (cur.ok) {
         uint32_t rc = 0;
-        const uint32_t rec_stage = cur.wide ? 0 : stage;
+        const uint32_t rec_stage = (wide_seg && cur.wide) ? 0 : stage;
         if (cur.staged && !pipe.wait(rec_stage)) rc = kStatusWaitTimeout;
         if (rc == 0) {
           const uint32_t rec_s = pipe.pay_addr + rec_stage * kPayStage;

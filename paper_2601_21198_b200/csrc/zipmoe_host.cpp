@@ -443,6 +443,18 @@ zipmoe_status zipmoe_blob_plan(const void *blob_v, uint64_t bytes, uint64_t payl
   Geometry g;
   make_geometry(info.rows, info.cols, info.layout, info.chunk_elems, &g);
   std::memcpy(table->code_len, blob + kTableOff, 256);
+  // largest tile record of the tensor, from the chunks' tile tables
+  uint32_t max_record = 0;
+  for (uint32_t k = 0; k < g.n_chunks; ++k) {
+    const uint64_t at = info.payload_off + load_le<uint64_t>(blob + kChunkOffOff + 8ull * k) / 8;
+    const uint32_t m = g.chunk_tiles(k);
+    if (at + 4ull * (m + 1) > info.payload_off + info.payload_bytes) return ZIPMOE_ERR_BAD_FORMAT;
+    for (uint32_t t = 0; t < m; ++t) {
+      const uint32_t o0 = load_le<uint32_t>(blob + at + 4ull * t), o1 = load_le<uint32_t>(blob + at + 4ull * (t + 1));
+      if (o1 < o0) return ZIPMOE_ERR_BAD_FORMAT;
+      max_record = std::max(max_record, (o1 - o0) * 16u);
+    }
+  }
   for (uint32_t k = 0; k < g.n_chunks; ++k) {
     zipmoe_chunk_desc &d = descs[k];
     uint32_t q0 = k * g.tiles_per_chunk, m = g.chunk_tiles(k);
@@ -461,7 +473,8 @@ zipmoe_status zipmoe_blob_plan(const void *blob_v, uint64_t bytes, uint64_t payl
     d.run_first_tile = tile_base;
     d.run_end_tile = tile_base + g.n_tiles;
     d.tiles_per_chunk = g.tiles_per_chunk;
-    d.reserved[0] = d.reserved[1] = 0;
+    d.max_record_bytes = max_record;
+    d.reserved = 0;
   }
   return ZIPMOE_OK;
 }
