@@ -10,18 +10,17 @@
 // compressed matrix W (blocked layout: tiles of 16 rows x 256 columns) and a
 // range of K:
 //   * each decode warp owns one strip and walks its tiles along K.  A tile is
-//     decoded in two halves of 8 rows.  Four warps form a quad: their four
+//     decoded in two halves of 8 rows.  Eight warps form a group: their eight
 //     half-tile buffers (8 rows x 256 columns each, K-major, no swizzle) are
-//     the first four 8-row groups of one A operand (M = 64; the upper 32 rows
-//     read whatever follows in shared memory and land in accumulator rows that
-//     nobody reads).  A half is decoded into registers first and stored once
-//     the MMAs that read the previous half are done, so decode and MMA overlap;
-//   * one MMA warp waits for a quad's half to be complete and issues its 16
-//     MMAs (K = 16 each; B = the activations, N = token rows); accumulators live
-//     in tensor memory, one [64 x N] fp32 block per quad and half;
+//     the eight 8-row groups of one A operand of M = 64.  A half is decoded
+//     into registers first and stored once the MMAs that read the previous
+//     half are done, so decode and MMA overlap;
+//   * one MMA warp per group waits for the group's half to be complete and
+//     issues its 16 MMAs (K = 16 each; B = the activations, N = token rows);
+//     accumulators live in tensor memory, one [64 x N] fp32 block per group and half;
 //   * one loader warp stages the activations of the current K step (token rows
-//     x 256 bf16) in a two-stage ring shared by all quads;
-//   * at the end two warps read the accumulators back (tcgen05.ld) and store Y.
+//     x 256 bf16) in a two-stage ring shared by all groups;
+//   * at the end four warps read the accumulators back (tcgen05.ld) and store Y.
 // The host wrapper runs it for W1 and W3 (gate, up), applies SiLU(g)*u, runs it
 // for W2, and combines the experts of every token; K is split over several
 // CTAs where few experts are active, the partial sums are added by the
@@ -42,7 +41,7 @@ namespace zipmoe_dev {
 #ifndef ZIPMOE_FFN_WARPS
 #define ZIPMOE_FFN_WARPS 16
 #endif
-constexpr int kFfnMaxWarps = ZIPMOE_FFN_WARPS;                         // decode warps per CTA, a multiple of 4 (plus loader and MMA warps)
+constexpr int kFfnMaxWarps = ZIPMOE_FFN_WARPS;            // decode warps per CTA, a multiple of the group size
 #ifndef ZIPMOE_FFN_GROUP
 #define ZIPMOE_FFN_GROUP 8
 #endif
@@ -140,7 +139,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   uint8_t *lut_scratch = lut_raw + kMyLutBytes;
   uint64_t *bars = reinterpret_cast<uint64_t *>(lut_scratch + kLutScratchBytes);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + ffn_bar_count(NW));
-  // barriers: [NW][2] record stages, [Q] quad half written, [Q] quad MMAs done, [2] X full, [2] X empty
+  // barriers: [NW][2] record stages, [Q] group's half written, [Q] group's MMAs done, [2] X full, [2] X empty
   const uint32_t bar0 = smem_addr(bars);
   const uint32_t quad_full = bar0 + 8 * (2 * NW), quad_done = quad_full + 8 * Q;
   const uint32_t x_full = quad_done + 8 * Q, x_empty = x_full + 16;
@@ -192,6 +191,76 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
          __ldg(&d->tile0) == 0;
   }
   if (!ok) report(a.la.status, kStatusBadDescriptor);
+  // ---- decode warps: where the strip's tiles are, and the first fetches, while the table is being built ----
+  bool failed = !has_strip || n_steps == 0 || !ok;
+  const uint32_t my = smem_addr(warp_raw + (is_decode ? warp : 0) * kFfnWarpBytes);
+  const uint32_t rec_bar = bar0 + 8 * (2 * (is_decode ? warp : 0));
+
+  // Where the strip's tiles are: lane i (and i + 32) looks up record start and length of the i-th tile of
+  // the K range once, so that the loop below touches global memory only for the data itself.
+  uint32_t rec_at[2] = {0, 0}, rec_len[2] = {0, 0};   // in 16-byte units from the start of the payload buffer
+  const uint8_t *sm_strip = a.la.sm;                  // sign+mantissa bytes of the strip's first tile
+  if (!failed) {
+    const uint32_t tq0 = strip * steps_total + s0;
+    bool bad = n_steps > 64;
+    for (uint32_t r = 0; r < 2; ++r) {
+      const uint32_t i = lane + 32 * r;
+      if (i >= n_steps || bad) continue;
+      const uint32_t tq = tq0 + i, c = c0 + tq / tpc, t = tq % tpc;
+      if (c >= a.la.n_chunks) {
+        bad = true;
+        continue;
+      }
+      const zipmoe_chunk_desc *d = a.la.chunks + c;
+      const uint64_t pay_off = __ldg(&d->payload_off);
+      if (t >= __ldg(&d->n_tiles) || __ldg(&d->tile_elems) != ZIPMOE_TILE_ELEMS_MAX || (pay_off & 15) ||
+          __ldg(&d->table_id) != table_id || pay_off + 4ull * (t + 2) > a.la.payload_bytes ||
+          (t + 1 == __ldg(&d->n_tiles) && __ldg(&d->last_tile_elems) != ZIPMOE_TILE_ELEMS_MAX)) {
+        bad = true;
+        continue;
+      }
+      const uint32_t *tab = reinterpret_cast<const uint32_t *>(a.la.payload + pay_off);
+      const uint32_t o0 = __ldg(tab + t), o1 = __ldg(tab + t + 1);
+      if (o1 <= o0 || o1 - o0 < 4 || o1 - o0 > (64 + ZIPMOE_TILE_ELEMS_MAX / 8 * ZIPMOE_MAX_CODE_LEN) / 16 + 1 ||
+          pay_off + 16ull * o1 > a.la.payload_bytes) {
+        bad = true;
+        continue;
+      }
+      rec_at[r] = (uint32_t)(pay_off >> 4) + o0;
+      rec_len[r] = o1 - o0;
+    }
+    const uint64_t sm_first = __ldg(&a.la.chunks[c0].sm_off) + (uint64_t)tq0 * ZIPMOE_TILE_ELEMS_MAX;
+    if ((sm_first & 15) || sm_first + (uint64_t)n_steps * ZIPMOE_TILE_ELEMS_MAX > a.la.sm_bytes) bad = true;
+    sm_strip = a.la.sm + sm_first;
+    if (__any_sync(0xFFFFFFFFu, bad)) {
+      report(a.la.status, kStatusBadDescriptor);
+      failed = true;
+    }
+  }
+  struct Tile {
+    const uint8_t *rec, *sm;
+    uint32_t rec_bytes;
+    bool staged;
+  };
+  auto tile = [&](uint32_t i) -> Tile {   // the i-th tile of the K range (all lanes call this)
+    const uint32_t at = __shfl_sync(0xFFFFFFFFu, i < 32 ? rec_at[0] : rec_at[1], i & 31);
+    const uint32_t len = __shfl_sync(0xFFFFFFFFu, i < 32 ? rec_len[0] : rec_len[1], i & 31);
+    Tile t;
+    t.rec = a.la.payload + (size_t)at * 16;
+    t.rec_bytes = len * 16;
+    t.sm = sm_strip + (size_t)i * ZIPMOE_TILE_ELEMS_MAX;
+    t.staged = t.rec_bytes <= (uint32_t)kPayBuf;
+    return t;
+  };
+  Tile cur = {a.la.payload, a.la.sm, 0, false};
+  uint2 smA[8], smB[8];
+  if (!failed) {
+    cur = tile(0);
+    if (cur.staged && lane == 0) bulk_load(my, cur.rec, cur.rec_bytes, rec_bar);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) smA[k] = ldg_v2_early(cur.sm + k * 256 + lane * 8);
+  }
+
   bool fast = true;
   if (ok) fast = build_lut(blockDim.x, a.la.tables[table_id].code_len, lut_raw, lut_scratch, a.la.status, LANE16) <=
                  (uint32_t)kLaneLutBits;
@@ -227,7 +296,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
       if (lane == 0) mbar_arrive(x_full + 8 * b);
     }
   } else if (ok && is_mma) {
-    // ---- one MMA warp per quad; one lane issues, per half-tile: D[64 x N] (+)= A[64 x 256] * X[N x 256]^T ----
+    // ---- one MMA warp per group; one lane issues, per half-tile: D[64 x N] (+)= A[64 x 256] * X[N x 256]^T ----
     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (G << 17) | ((uint32_t)(kGroupWarps / 2) << 24);   // bf16 x bf16 -> fp32, N = 8G, M = 8 * kGroupWarps
     const uint32_t q = warp - NW;
     const uint32_t abuf = smem_addr(warp_raw) + 2 * kPayStage + kGroupWarps * q * kFfnWarpBytes;
@@ -251,84 +320,17 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
           for (uint32_t j = 0; j < 16; ++j)
             mma_bf16(d_tmem, a_desc0 + j * (2 * kBLbo / 16), b_desc0 + j * (256 / 16), idesc, (s > 0 || j > 0) ? 1u : 0u);
           mma_commit(quad_done + 8 * q);
-          if (half == 1) mma_commit(x_empty + 8 * xb);   // this quad is done with the X stage
+          if (half == 1) mma_commit(x_empty + 8 * xb);   // this group is done with the X stage
         }
         __syncwarp();
       }
     }
     if (!alive) report(a.la.status, kStatusWaitTimeout);
   } else if (ok && is_decode) {
-    // ---- one strip of 16 rows: decode tile after tile along K, hand half-tiles to the quad's A operand ----
-    const uint32_t my = smem_addr(warp_raw + warp * kFfnWarpBytes);
+    // ---- one strip of 16 rows: decode tile after tile along K, hand half-tiles to the group's A operand ----
     const uint32_t buf = my + 2 * kPayStage;
-    const uint32_t rec_bar = bar0 + 8 * (2 * warp), q = warp / kGroupWarps;
+    const uint32_t q = warp / kGroupWarps;
     uint32_t rec_phase = 0, hn = 0;
-    bool failed = !has_strip || n_steps == 0;
-
-    // Where the strip's tiles are: lane i (and i + 32) looks up record start and length of the i-th tile of
-    // the K range once, so that the loop below touches global memory only for the data itself.
-    uint32_t rec_at[2] = {0, 0}, rec_len[2] = {0, 0};   // in 16-byte units from the start of the payload buffer
-    const uint8_t *sm_strip = a.la.sm;                  // sign+mantissa bytes of the strip's first tile
-    if (has_strip && n_steps) {
-      const uint32_t tq0 = strip * steps_total + s0;
-      bool bad = n_steps > 64;
-      for (uint32_t r = 0; r < 2; ++r) {
-        const uint32_t i = lane + 32 * r;
-        if (i >= n_steps || bad) continue;
-        const uint32_t tq = tq0 + i, c = c0 + tq / tpc, t = tq % tpc;
-        if (c >= a.la.n_chunks) {
-          bad = true;
-          continue;
-        }
-        const zipmoe_chunk_desc *d = a.la.chunks + c;
-        const uint64_t pay_off = __ldg(&d->payload_off);
-        if (t >= __ldg(&d->n_tiles) || __ldg(&d->tile_elems) != ZIPMOE_TILE_ELEMS_MAX || (pay_off & 15) ||
-            __ldg(&d->table_id) != table_id || pay_off + 4ull * (t + 2) > a.la.payload_bytes ||
-            (t + 1 == __ldg(&d->n_tiles) && __ldg(&d->last_tile_elems) != ZIPMOE_TILE_ELEMS_MAX)) {
-          bad = true;
-          continue;
-        }
-        const uint32_t *tab = reinterpret_cast<const uint32_t *>(a.la.payload + pay_off);
-        const uint32_t o0 = __ldg(tab + t), o1 = __ldg(tab + t + 1);
-        if (o1 <= o0 || o1 - o0 < 4 || o1 - o0 > (64 + ZIPMOE_TILE_ELEMS_MAX / 8 * ZIPMOE_MAX_CODE_LEN) / 16 + 1 ||
-            pay_off + 16ull * o1 > a.la.payload_bytes) {
-          bad = true;
-          continue;
-        }
-        rec_at[r] = (uint32_t)(pay_off >> 4) + o0;
-        rec_len[r] = o1 - o0;
-      }
-      const uint64_t sm_first = __ldg(&a.la.chunks[c0].sm_off) + (uint64_t)tq0 * ZIPMOE_TILE_ELEMS_MAX;
-      if ((sm_first & 15) || sm_first + (uint64_t)n_steps * ZIPMOE_TILE_ELEMS_MAX > a.la.sm_bytes) bad = true;
-      sm_strip = a.la.sm + sm_first;
-      if (__any_sync(0xFFFFFFFFu, bad)) {
-        report(a.la.status, kStatusBadDescriptor);
-        failed = true;
-      }
-    }
-    struct Tile {
-      const uint8_t *rec, *sm;
-      uint32_t rec_bytes;
-      bool staged;
-    };
-    auto tile = [&](uint32_t i) -> Tile {   // the i-th tile of the K range (all lanes call this)
-      const uint32_t at = __shfl_sync(0xFFFFFFFFu, i < 32 ? rec_at[0] : rec_at[1], i & 31);
-      const uint32_t len = __shfl_sync(0xFFFFFFFFu, i < 32 ? rec_len[0] : rec_len[1], i & 31);
-      Tile t;
-      t.rec = a.la.payload + (size_t)at * 16;
-      t.rec_bytes = len * 16;
-      t.sm = sm_strip + (size_t)i * ZIPMOE_TILE_ELEMS_MAX;
-      t.staged = t.rec_bytes <= (uint32_t)kPayBuf;
-      return t;
-    };
-    Tile cur = {a.la.payload, a.la.sm, 0, false};
-    uint2 smA[8], smB[8];
-    if (!failed) {
-      cur = tile(0);
-      if (cur.staged && lane == 0) bulk_load(my, cur.rec, cur.rec_bytes, rec_bar);
-#pragma unroll
-      for (int k = 0; k < 8; ++k) smA[k] = ldg_v2_early(cur.sm + k * 256 + lane * 8);
-    }
     // hand-over of one half in two moves: before the first store, wait until the MMAs of the previous half have
     // read the buffer; after the last store, make the stores visible to the tensor core and tell the MMA warp
     auto buffer_free = [&]() -> bool {
@@ -402,7 +404,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
         }
         if (!good) failed = true;
       }
-      if (!step_done) {   // nothing to contribute: keep the quad's hand-over going with whatever the buffer holds
+      if (!step_done) {   // nothing to contribute: keep the group's hand-over going with whatever the buffer holds
         buffer_free();
         publish();
         buffer_free();
