@@ -64,7 +64,7 @@ _lib.zipmoe_encode.argtypes = [_vp, _u64, _u64, ctypes.POINTER(EncodeOpts), _vp,
 _lib.zipmoe_blob_info_get.argtypes = [_vp, _u64, ctypes.POINTER(BlobInfo)]
 _lib.zipmoe_blob_validate.argtypes = [_vp, _u64]
 _lib.zipmoe_blob_plan.argtypes = [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _u32, _vp, _vp]
-_lib.zipmoe_decode.argtypes = [_vp, _u32, _u32, _vp, _u32, _vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp]
+_lib.zipmoe_decode.argtypes = [_vp, _u32, _u32, _vp, _u32, _vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp, _u32]
 _lib.zipmoe_recover.argtypes = [_vp, _vp, _u64, _vp, _vp]
 _lib.zipmoe_recover.restype = _int
 _lib.zipmoe_ffn_workspace_bytes.argtypes = [_u32, _u32, ctypes.POINTER(CompressedExperts), ctypes.POINTER(_u64)]
@@ -159,11 +159,11 @@ def zipmoe_blob_plan(blob, payload_base, sm_base, out_base, table_id, chunk_base
 
 
 def zipmoe_decode(chunks, n_chunks, n_tiles, tables, n_tables, payload, payload_bytes, sm, sm_bytes, out_bf16,
-                  out_elems, status_word=None, stream=None):
+                  out_elems, status_word=None, stream=None, max_record_bytes=0):
     """All pointer arguments are device tensors (or raw device addresses)."""
     _check("zipmoe_decode", _lib.zipmoe_decode(_ptr(chunks), n_chunks, n_tiles, _ptr(tables), n_tables, _ptr(payload),
                                                 payload_bytes, _ptr(sm), sm_bytes, _ptr(out_bf16), out_elems,
-                                                _ptr(status_word), _ptr(stream)))
+                                                _ptr(status_word), _ptr(stream), int(max_record_bytes)))
 
 
 def zipmoe_recover(exp, sm, n_elems, out_bf16, stream=None):
@@ -229,6 +229,7 @@ class DecodePlan:
         self.descs = np.concatenate(descs) if descs else np.zeros(0, CHUNK_DESC_DTYPE)
         self.tables = np.concatenate(tables) if tables else np.zeros(0, np.uint8)
         self.n_chunks, self.n_tiles, self.n_tables = chunk_base, tile_base, len(blobs)
+        self.max_record_bytes = int(self.descs["max_record_bytes"].max()) if self.n_chunks else 0
 
     def algorithmic_bytes(self):
         """Bytes one decode must move: E-chunk section + SM bytes read, bf16 written."""
@@ -267,7 +268,7 @@ class DevicePlan:
         p = self.plan
         s = torch.cuda.current_stream(self.device) if stream is None else stream
         zipmoe_decode(self.descs, p.n_chunks, p.n_tiles, self.tables, p.n_tables, self.payload, p.payload_bytes,
-                      self.sm, p.sm_bytes, out, p.out_elems, self.status, s.cuda_stream)
+                      self.sm, p.sm_bytes, out, p.out_elems, self.status, s.cuda_stream, p.max_record_bytes)
 
 
 class DeviceExperts:

@@ -207,8 +207,8 @@ struct TileWork {
   const uint8_t *sm;    // global address of the tile's sign+mantissa bytes
   uint16_t *out;        // global address of the tile's first element
   uint32_t rec_bytes, pitch, valid, iters, pieces;
-  bool ok, staged;
-  bool wide;            // staged across both record stages (a record of up to 2 * kPayStage - kPaySlack bytes)
+  uint32_t ok, staged;  // flags (whole registers: the struct is copied once per tile)
+  uint32_t wide;        // staged across both record stages (a record of up to 2 * kPayStage - kPaySlack bytes)
 };
 
 struct LaunchArgs {

@@ -57,7 +57,7 @@ struct WarpPipe {
   // stages and uses the first stage's barrier, so no other record can be in flight beside it
   __device__ __forceinline__ void load_record(const TileWork &t, uint32_t stage) {
     if (!t.staged) return;
-    if (t.wide) stage = 0;
+    if (t.wide) stage = 0;   // never set in the instantiation without wide records
     if (lane == 0) bulk_load(pay_addr + stage * kPayStage, t.rec, t.rec_bytes, bar(stage));
     pending |= 1u << stage;
   }
@@ -102,6 +102,9 @@ struct GlobalSink {
   }
 };
 
+// WIDE: records longer than one record stage may be staged across both (near-incompressible tensors); the
+// host picks the instantiation without it when it knows that no record of the launch is that long.
+template <bool WIDE>
 __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t *lut_raw = smem;
@@ -144,12 +147,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
     const bool fast = build_lut(kThreads, a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <=
                       (uint32_t)kLaneLutBits;
 
-    // Tensors whose largest record fits one record stage (all but near-incompressible ones) never take the
-    // wide-record branches below.
-#ifndef ZIPMOE_WIDE_STAGING
-#define ZIPMOE_WIDE_STAGING 1
-#endif
-    const bool wide_seg = ZIPMOE_WIDE_STAGING && __ldg(&d->max_record_bytes) > (uint32_t)kPayBuf;
     uint32_t g = g0 + warp;
     uint32_t stage = 0;
     // descriptor and tile-in-chunk of this warp's next tile, stepped without divisions
@@ -164,7 +161,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
     TileWork cur;
     cur.ok = false;
     if (g < seg_end && !dead) {
-      cur = resolve_tile(a, tc, tt, wide_seg);
+      cur = resolve_tile(a, tc, tt, WIDE);
       if (!cur.ok) report(a.status, kStatusBadDescriptor);
       else {
         pipe.load_record(cur, stage);
@@ -178,15 +175,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
       const uint32_t g2 = g + kWarps;
       if (g2 < seg_end) {
         step();
-        nxt = resolve_tile(a, tc, tt, wide_seg);
+        nxt = resolve_tile(a, tc, tt, WIDE);
         if (!nxt.ok) report(a.status, kStatusBadDescriptor);
       }
       // the next record is fetched while this one is decoded, unless one of the two needs both stages
-      const bool prefetch = nxt.ok && (!wide_seg || (!nxt.wide && !(cur.ok && cur.wide)));
+      const bool prefetch = nxt.ok && (!WIDE || (!nxt.wide && !(cur.ok && cur.wide)));
       if (prefetch) pipe.load_record(nxt, stage ^ 1);   // that stage was released by the __syncwarp below
       if (cur.ok) {
         uint32_t rc = 0;
-        const uint32_t rec_stage = (wide_seg && cur.wide) ? 0 : stage;
+        const uint32_t rec_stage = (WIDE && cur.wide) ? 0 : stage;
         if (cur.staged && !pipe.wait(rec_stage)) rc = kStatusWaitTimeout;
         if (rc == 0) {
           const uint32_t rec_s = pipe.pay_addr + rec_stage * kPayStage;
@@ -223,7 +220,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
         }
       }
       __syncwarp();   // every lane is done with the current record stage and SM slots
-      if (nxt.ok && !prefetch) pipe.load_record(nxt, stage ^ 1);
+      if (WIDE && nxt.ok && !prefetch) pipe.load_record(nxt, stage ^ 1);
       if (nxt.ok)
         for (; nxt_issued < nxt.pieces; ++nxt_issued) pipe.load_sm_piece(nxt, nxt_issued);
       cur = nxt;
@@ -255,7 +252,9 @@ zipmoe_status prepare_device(int *sm_count) {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ZIPMOE_ERR_CUDA;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ZIPMOE_ERR_CUDA;
     if (major != 10) return ZIPMOE_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(zipmoe_dev::decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(zipmoe_dev::decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             zipmoe_dev::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(zipmoe_dev::decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              zipmoe_dev::kSmemBytes) != cudaSuccess)
       return ZIPMOE_ERR_CUDA;
     g_dev[dev].sm_count = sms;
@@ -270,7 +269,7 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
                                        const zipmoe_table *tables, uint32_t n_tables, const uint8_t *payload,
                                        uint64_t payload_bytes, const uint8_t *sm, uint64_t sm_bytes,
                                        uint16_t *out_bf16, uint64_t out_elems, uint32_t *status_word,
-                                       zipmoe_stream stream) {
+                                       zipmoe_stream stream, uint32_t max_record_bytes) {
   if (n_chunks == 0 || n_tiles == 0) return (n_chunks == 0 && n_tiles == 0) ? ZIPMOE_OK : ZIPMOE_ERR_INVALID_ARG;
   if (!chunks || !tables || n_tables == 0 || !payload || !sm || !out_bf16) return ZIPMOE_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(payload) | reinterpret_cast<uintptr_t>(sm) | reinterpret_cast<uintptr_t>(out_bf16) |
@@ -299,7 +298,10 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
   if (n_tiles < ctas) ctas = n_tiles;
   a.tiles_per_cta = (n_tiles + ctas - 1) / ctas;
   ctas = (n_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
-  zipmoe_dev::decode_kernel<<<ctas, zipmoe_dev::kThreads, zipmoe_dev::kSmemBytes,
-                              reinterpret_cast<cudaStream_t>(stream)>>>(a);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (max_record_bytes != 0 && max_record_bytes <= (uint32_t)zipmoe_dev::kPayBuf)
+    zipmoe_dev::decode_kernel<false><<<ctas, zipmoe_dev::kThreads, zipmoe_dev::kSmemBytes, st>>>(a);
+  else
+    zipmoe_dev::decode_kernel<true><<<ctas, zipmoe_dev::kThreads, zipmoe_dev::kSmemBytes, st>>>(a);
   return cudaGetLastError() == cudaSuccess ? ZIPMOE_OK : ZIPMOE_ERR_CUDA;
 }
