@@ -207,8 +207,8 @@ struct TileWork {
   const uint8_t *sm;    // global address of the tile's sign+mantissa bytes
   uint16_t *out;        // global address of the tile's first element
   uint32_t rec_bytes, pitch, valid, iters, pieces;
-  uint32_t ok, staged;  // flags (whole registers: the struct is copied once per tile)
-  uint32_t wide;        // staged across both record stages (a record of up to 2 * kPayStage - kPaySlack bytes)
+  bool ok, staged;
+  bool wide;            // staged across both record stages (a record of up to 2 * kPayStage - kPaySlack bytes)
 };
 
 struct LaunchArgs {
@@ -241,7 +241,7 @@ static_assert(sizeof(zipmoe_chunk_desc) == 80, "descriptor is read as five 16-by
 
 // Everything the decoder needs about tile t of descriptor c, with every offset
 // checked against the sizes of the buffers the launch was given.
-__device__ inline TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_t t, const bool allow_wide = false) {
+__device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_t t, const bool allow_wide = false) {
   TileWork w;
   w.ok = false;
   w.staged = false;

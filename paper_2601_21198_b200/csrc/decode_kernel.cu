@@ -55,9 +55,10 @@ struct WarpPipe {
   // all lanes call these; one lane starts the copy
   // a record of ordinary size goes into `stage`; a wide one (8-bit codes everywhere: 4160 bytes) spans both
   // stages and uses the first stage's barrier, so no other record can be in flight beside it
+  template <bool WIDE>
   __device__ __forceinline__ void load_record(const TileWork &t, uint32_t stage) {
     if (!t.staged) return;
-    if (t.wide) stage = 0;   // never set in the instantiation without wide records
+    if (WIDE && t.wide) stage = 0;
     if (lane == 0) bulk_load(pay_addr + stage * kPayStage, t.rec, t.rec_bytes, bar(stage));
     pending |= 1u << stage;
   }
@@ -164,7 +165,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
       cur = resolve_tile(a, tc, tt, WIDE);
       if (!cur.ok) report(a.status, kStatusBadDescriptor);
       else {
-        pipe.load_record(cur, stage);
+        pipe.template load_record<WIDE>(cur, stage);
         for (uint32_t p = 0; p < cur.pieces; ++p) pipe.load_sm_piece(cur, p);
       }
     }
@@ -180,7 +181,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
       }
       // the next record is fetched while this one is decoded, unless one of the two needs both stages
       const bool prefetch = nxt.ok && (!WIDE || (!nxt.wide && !(cur.ok && cur.wide)));
-      if (prefetch) pipe.load_record(nxt, stage ^ 1);   // that stage was released by the __syncwarp below
+      if (prefetch) pipe.template load_record<WIDE>(nxt, stage ^ 1);   // that stage was released by the __syncwarp below
       if (cur.ok) {
         uint32_t rc = 0;
         const uint32_t rec_stage = (WIDE && cur.wide) ? 0 : stage;
@@ -220,7 +221,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
         }
       }
       __syncwarp();   // every lane is done with the current record stage and SM slots
-      if (WIDE && nxt.ok && !prefetch) pipe.load_record(nxt, stage ^ 1);
+      if (WIDE && nxt.ok && !prefetch) pipe.template load_record<WIDE>(nxt, stage ^ 1);
       if (nxt.ok)
         for (; nxt_issued < nxt.pieces; ++nxt_issued) pipe.load_sm_piece(nxt, nxt_issued);
       cur = nxt;
