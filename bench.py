@@ -392,6 +392,25 @@ def run_ours(args):
                                       "frac_of_peak": 4 * n / rms / 1e6 / peaks["hbm_gbs"], "ms": rms,
                                       "note": "exponent bytes already decompressed: 2 B read + 2 B written per element"}
             del d_e, d_s
+        if world == 1:
+            # compression states: one stream stays in pinned host memory and is read in place over PCIe
+            states = {}
+            d_pay, d_sm = dplan.payload, dplan.sm
+            for name, (pay, smb, moved) in {"sm_chunks_on_host": (d_pay, h_sm, int(h_sm.numel())),
+                                            "e_chunks_on_host": (h_pay, d_sm, int(h_pay.numel()))}.items():
+                dplan.payload, dplan.sm = pay, smb
+                c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                dplan.decode(out)
+                c0.record(stream)
+                for _ in range(3):
+                    dplan.decode(out)
+                c1.record(stream)
+                torch.cuda.synchronize(dev)
+                cms = c0.elapsed_time(c1) / 3
+                states[name] = {"decoded_bf16_gbs": bf16_bytes / cms / 1e6, "ms": cms,
+                                "host_bytes_read_per_step": moved, "host_link_gbs": moved / cms / 1e6}
+            dplan.payload, dplan.sm = d_pay, d_sm
+            line["compression_states"] = states
         if world == 1 and not args.no_ffn:
             del dplan, out, h_pay, h_sm, h_out
             torch.cuda.empty_cache()

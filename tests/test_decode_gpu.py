@@ -253,3 +253,22 @@ def test_recovery_kernel_matches_oracle_merge(zb, n):
     got = out.cpu().numpy().view(np.uint16)
     assert np.array_equal(got[:n], codec.merge(e, s))
     assert (got[n:] == 0x5555).all()
+
+
+@pytest.mark.parametrize("on_host", ["sm", "payload", "both"])
+def test_streams_in_pinned_host_memory(zb, on_host):
+    """Compression states: the E-chunks and the SM-chunks of a tensor may live in different memories.  Either
+    stream (or both) stays in pinned host memory, which the device reads in place during the decode."""
+    import torch
+    x = inputs.gaussian((700, 1031), 0.02, 77)
+    plan = zb.DecodePlan([zb.zipmoe_encode(x, chunk_elems=65536)])
+    dev = plan.to_device()
+    if on_host in ("sm", "both"):
+        dev.sm = torch.from_numpy(plan.sm).pin_memory()
+    if on_host in ("payload", "both"):
+        dev.payload = torch.from_numpy(plan.payload).pin_memory()
+    out = dev.new_output()
+    dev.decode(out)
+    torch.cuda.synchronize()
+    assert int(dev.status.item()) == 0
+    assert np.array_equal(out.cpu().numpy().view(np.uint16)[: x.size], x.ravel())
