@@ -7,10 +7,12 @@
 // decompressed exponents never reach global memory.
 //
 // Data movement per tile (256*I elements):
-//   global -> shared : the tile record (sub-stream bit counts + code bits) and
-//                      the tile's sign+mantissa bytes, each by one bulk
-//                      asynchronous copy (cp.async.bulk, completion on an
-//                      mbarrier), issued one tile ahead of the decode;
+//   global -> shared : the tile record (sub-stream bit counts + code bits) by
+//                      one bulk asynchronous copy (cp.async.bulk, completion
+//                      on an mbarrier), one tile ahead of the decode; the
+//                      tile's sign+mantissa bytes as two 2 KB pieces through
+//                      two slots, each refilled for the next tile as soon as
+//                      the current tile is done with it;
 //   shared -> regs   : 8 SM bytes per lane per iteration, code words on demand;
 //   regs   -> global : one 16-byte store per lane per iteration; a warp writes
 //                      512 contiguous bytes per iteration.

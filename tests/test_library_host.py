@@ -138,3 +138,29 @@ def test_plan_descriptors(zb):
     assert (d["payload_off"] % 16 == 0).all() and d["payload_off"][2] == plan.payload_base[1]
     assert plan.payload.size == plan.payload_bytes + zb.DEVICE_PAD_BYTES
     assert plan.algorithmic_bytes() == plan.payload_bytes + 3 * (a.size + b.size)
+
+
+def test_ffn_planning_on_the_host(zb):
+    """zipmoe_ffn_workspace_bytes needs no GPU: limits and sizes of the fused call."""
+    ok = zb.CompressedExperts(8, 4096, 14336, 1, 16, 16, 16, 1, 0, 16, 0, 16, 0)
+    sizes = [zb.zipmoe_ffn_workspace_bytes(T, 2, ok) for T in (1, 8, 16, 64)]
+    assert sizes == sorted(sizes) and sizes[0] > 0
+    # fp32 gate/up partials dominate: at least 2 * S * inter * 4 bytes
+    assert sizes[-1] >= 2 * 128 * 14336 * 4
+    for bad in (dict(T=0), dict(T=65), dict(k=0), dict(k=9), dict(hidden=1000), dict(inter=100), dict(n_experts=0),
+                dict(n_experts=257)):
+        ex = zb.CompressedExperts(bad.get("n_experts", 8), bad.get("hidden", 4096), bad.get("inter", 14336), 1, 16, 16,
+                                  16, 1, 0, 16, 0, 16, 0)
+        with pytest.raises(zb.ZipMoEError) as err:
+            zb.zipmoe_ffn_workspace_bytes(bad.get("T", 4), bad.get("k", 2), ex)
+        assert err.value.status == zb.ERR_UNSUPPORTED, bad
+    assert ctypes.sizeof(zb.CompressedExperts) == 80
+
+
+def test_plan_reports_the_largest_tile_record(zb):
+    x = inputs.gaussian((64, 1408), 0.02, 5)
+    plan = zb.DecodePlan([zb.zipmoe_encode(x, chunk_elems=4096)])
+    assert 1300 < plan.max_record_bytes < 1700
+    u = np.random.default_rng(0).integers(0, 1 << 16, 20000, dtype=np.uint16)
+    plan = zb.DecodePlan([zb.zipmoe_encode(u, chunk_elems=4096)])
+    assert plan.max_record_bytes == 64 + 4096         # 8-bit codes everywhere
