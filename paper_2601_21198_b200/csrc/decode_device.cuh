@@ -36,7 +36,7 @@ constexpr uint32_t kSmPieceBytes = kPieceIters * 256;
 constexpr uint32_t kSmPieces = 16 / kPieceIters;   // pieces of a full tile = sign+mantissa slots of a warp
 
 constexpr int kPayBuf = 2048;        // record bytes staged in shared memory; longer records are read from global
-constexpr int kPaySlack = 64;        // readable bytes after a staged record (a lane looks two words ahead)
+constexpr int kPaySlack = 64;        // readable bytes after a staged record (a lane looks three words ahead)
 constexpr int kPayStage = kPayBuf + kPaySlack;
 
 __device__ __forceinline__ void report(uint32_t *status, uint32_t code) {
@@ -299,29 +299,32 @@ struct WordSource {
     }
     return __ldg(at_g++);
   }
-  // If bit 5 of pos is set (a whole word has been consumed): b_hi <- b_lo,
-  // b_lo <- next word, clear the bit.  Predicated, no branch.
-  __device__ __forceinline__ void advance(uint32_t &pos, uint32_t &b_hi, uint32_t &b_lo) {
+  // If bit 5 of pos is set (a whole word has been consumed): b_hi <- b_lo, b_lo <- b_next, b_next <- the
+  // following word, clear the bit.  b_next is loaded one word early so that its latency is off the decode chain.
+  // Predicated, no branch.
+  __device__ __forceinline__ void advance(uint32_t &pos, uint32_t &b_hi, uint32_t &b_lo, uint32_t &b_next) {
     if (STAGED) {
       asm volatile(
           "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
           "and.b32 t, %0, 32;\n\t"
           "setp.ne.u32 p, t, 0;\n\t"
           "@p mov.b32 %1, %2;\n\t"
-          "@p ld.shared.u32 %2, [%3];\n\t"
-          "@p add.u32 %3, %3, 4;\n\t"
+          "@p mov.b32 %2, %3;\n\t"
+          "@p ld.shared.u32 %3, [%4];\n\t"
+          "@p add.u32 %4, %4, 4;\n\t"
           "@p xor.b32 %0, %0, 32;\n\t}"
-          : "+r"(pos), "+r"(b_hi), "+r"(b_lo), "+r"(at_s));
+          : "+r"(pos), "+r"(b_hi), "+r"(b_lo), "+r"(b_next), "+r"(at_s));
     } else {
       asm volatile(
           "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
           "and.b32 t, %0, 32;\n\t"
           "setp.ne.u32 p, t, 0;\n\t"
           "@p mov.b32 %1, %2;\n\t"
-          "@p ld.global.nc.u32 %2, [%3];\n\t"
-          "@p add.u64 %3, %3, 4;\n\t"
+          "@p mov.b32 %2, %3;\n\t"
+          "@p ld.global.nc.u32 %3, [%4];\n\t"
+          "@p add.u64 %4, %4, 4;\n\t"
           "@p xor.b32 %0, %0, 32;\n\t}"
-          : "+r"(pos), "+r"(b_hi), "+r"(b_lo), "+l"(at_g));
+          : "+r"(pos), "+r"(b_hi), "+r"(b_lo), "+r"(b_next), "+l"(at_g));
     }
   }
 };
@@ -355,7 +358,7 @@ template <bool STAGED, int KIND>
 struct LaneDecoder {
   static constexpr bool FAST = KIND != kLutWide;
   WordSource<STAGED> src;
-  uint32_t pos, b_hi, b_lo, lut, my_lut;
+  uint32_t pos, b_hi, b_lo, b_next, lut, my_lut;
 
   // record in shared memory at rec_s (STAGED) or in global memory at rec_g; lut =
   // shared address of the lane table (FAST) or the wide table (!FAST).  Turns the
@@ -380,6 +383,7 @@ struct LaneDecoder {
     pos = start & 31;
     b_hi = src.pop();
     b_lo = src.pop();
+    b_next = src.pop();
     lut = lut_addr;
     my_lut = lut_addr + (KIND == kLutLane16 ? 2 : 4) * lane;
     return true;
@@ -395,7 +399,7 @@ struct LaneDecoder {
     w = __funnelshift_l(0u, w, ea);
     eb = lookup(w);
     pos += ea + eb;
-    src.advance(pos, b_hi, b_lo);
+    src.advance(pos, b_hi, b_lo, b_next);
   }
   __device__ __forceinline__ void quad(uint32_t &ea, uint32_t &eb, uint32_t &ec, uint32_t &ed) {   // four codes <= 8 bits
     uint32_t w = __funnelshift_l(b_lo, b_hi, pos);
@@ -407,12 +411,12 @@ struct LaneDecoder {
     w = __funnelshift_l(0u, w, ec);
     ed = lookup(w);
     pos += (ea + eb) + (ec + ed);
-    src.advance(pos, b_hi, b_lo);
+    src.advance(pos, b_hi, b_lo, b_next);
   }
   __device__ __forceinline__ uint32_t single() {
     const uint32_t e = lookup(__funnelshift_l(b_lo, b_hi, pos));
     pos += e;
-    src.advance(pos, b_hi, b_lo);
+    src.advance(pos, b_hi, b_lo, b_next);
     return e;
   }
   // the next 8 elements of this lane merged with their sign+mantissa bytes: 8 bf16
