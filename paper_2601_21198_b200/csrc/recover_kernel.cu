@@ -25,8 +25,8 @@ __global__ void __launch_bounds__(256) recover_kernel(const uint8_t *__restrict_
   const uint64_t n16 = n / 16;
   const uint4 *e4 = reinterpret_cast<const uint4 *>(exp), *s4 = reinterpret_cast<const uint4 *>(sm);
   uint4 *o4 = reinterpret_cast<uint4 *>(out);
-  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (uint64_t)gridDim.x * blockDim.x) {
-    const uint4 e = __ldcs(e4 + i), s = __ldcs(s4 + i);
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  auto merge16 = [&](const uint4 &e, const uint4 &s, uint64_t i) {
     const uint32_t ew[4] = {e.x, e.y, e.z, e.w}, sw[4] = {s.x, s.y, s.z, s.w};
     uint32_t o[8];
 #pragma unroll
@@ -36,7 +36,20 @@ __global__ void __launch_bounds__(256) recover_kernel(const uint8_t *__restrict_
     }
     __stcs(o4 + 2 * i, make_uint4(o[0], o[1], o[2], o[3]));
     __stcs(o4 + 2 * i + 1, make_uint4(o[4], o[5], o[6], o[7]));
+  };
+  uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  // four independent 16-element groups per thread and trip: 128 bytes of loads in flight per thread
+  for (; i + 3 * stride < n16; i += 4 * stride) {
+    uint4 e[4], s[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      e[u] = __ldcs(e4 + i + u * stride);
+      s[u] = __ldcs(s4 + i + u * stride);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) merge16(e[u], s[u], i + u * stride);
   }
+  for (; i < n16; i += stride) merge16(__ldcs(e4 + i), __ldcs(s4 + i), i);
   // the last n % 16 elements, one per thread of the first block
   const uint64_t tail = n16 * 16 + threadIdx.x;
   if (blockIdx.x == 0 && threadIdx.x < 16 && tail < n) {
@@ -58,7 +71,7 @@ extern "C" zipmoe_status zipmoe_recover(const uint8_t *exp, const uint8_t *sm, u
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return ZIPMOE_ERR_CUDA;
   uint64_t blocks = (n_elems / 16 + 255) / 256;
-  const uint64_t cap = (uint64_t)sms * 16;
+  const uint64_t cap = (uint64_t)sms * 8;
   if (blocks > cap) blocks = cap;
   if (blocks == 0) blocks = 1;
   zipmoe_dev::recover_kernel<<<(unsigned)blocks, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(exp, sm, n_elems,
