@@ -146,10 +146,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
       report(a.status, kStatusBadDescriptor);
       break;
     }
-    __syncthreads();  // every warp is done with the previous table
-    const bool fast = build_lut(kThreads, a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <=
-                      (uint32_t)kLaneLutBits;
-
     uint32_t g = g0 + warp;
     uint32_t stage = 0;
     // descriptor and tile-in-chunk of this warp's next tile, stepped without divisions
@@ -161,6 +157,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
         ++tc;
       }
     };
+    // the warp's first tile of the segment is fetched while the table is being built (its own stages and
+    // slots are free: it has finished its tiles of the previous segment)
     TileWork cur;
     cur.ok = false;
     if (g < seg_end && !dead) {
@@ -171,6 +169,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
         for (uint32_t p = 0; p < cur.pieces; ++p) pipe.load_sm_piece(cur, p);
       }
     }
+    __syncthreads();  // every warp is done with the previous table
+    const bool fast = build_lut(kThreads, a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <=
+                      (uint32_t)kLaneLutBits;
+
     for (; g < seg_end && !dead; g += kWarps) {
       TileWork nxt;
       nxt.ok = false;
