@@ -21,7 +21,7 @@
  *     canonical Huffman code over exponent bytes, the quantity the paper's
  *     own entropy analysis measures (Fig. 2, Fig. 3).
  *
- * The container layout ("ZMOE v1") is this project's own; it is written out
+ * The container layout ("ZMOE v2") is this project's own; it is written out
  * in full below because the decoder is defined by it.  Every function that
  * has an independent pin (closed form, brute force, textbook special case)
  * is pinned in tests/test_oracle_*.py.  The one part that cannot be pinned
@@ -30,9 +30,9 @@
  * unpinned" for blob bytes; only decodability and size bounds bind.
  *
  * ---------------------------------------------------------------------------
- * ZMOE v1 container (all integers little-endian)
+ * ZMOE v2 container (all integers little-endian)
  *
- *   offset  0  u32 magic 0x454F4D5A      4  u32 version (1)
+ *   offset  0  u32 magic 0x454F4D5A      4  u32 version (2)
  *           8  u64 n_elems              16  u32 rows     20 u32 cols
  *          24  u32 layout (0 linear, 1 blocked)          28 u32 chunk_elems
  *          32  u32 tile_elems           36  u32 max_code_len
@@ -60,11 +60,16 @@
  *                           this table, tile_off[m] the size of the chunk;
  *     zero padding to 16 bytes, then m tile records.
  *   Tile record:
- *     u16 sub_bits[32]      number of code bits of each lane's sub-stream;
- *     the 32 sub-streams, lane 0 first, concatenated bit by bit with no
- *     padding between them, stored as u32 words whose bits are consumed from
- *     bit 31 down to bit 0; zero padding to a 16-byte boundary.
- *   Lane `lane` codes its existing elements in order i = 0..I-1, j = 0..7.
+ *     u16 sub_bits[64]      number of code bits of each sub-stream; every lane
+ *                           has two, entry 2*lane + h for h = 0, 1;
+ *     the 64 sub-streams in that order (lane 0 h 0, lane 0 h 1, lane 1 h 0, ...),
+ *     concatenated bit by bit with no padding between them, stored as u32
+ *     words whose bits are consumed from bit 31 down to bit 0; zero padding to
+ *     a 16-byte boundary.
+ *   Sub-stream (lane, h) codes the lane's existing elements of the iterations
+ *   i = h, h+2, h+4, ... < I in that order, j = 0..7 inside each.  (Two
+ *   independent streams per lane let a decoder work on two codes at a time; the
+ *   paper leaves the order of elements inside a shard open.)
  *
  *   Sign+mantissa section: byte q*tile_elems + pos holds
  *     (sign << 7) | mantissa  of the element at (q, pos); zero padded to 16.
@@ -89,6 +94,8 @@
 #define ZO_TABLE_OFF 64u
 #define ZO_CHUNKOFF_OFF 320u
 #define ZO_MAX_CODE_LEN 12
+#define ZO_VERSION 2u
+#define ZO_REC_HEAD 128u /* u16 sub_bits[64] */
 
 /* ---- little-endian field access ---------------------------------------- */
 static uint32_t rd32(const uint8_t *p) {
@@ -294,7 +301,7 @@ static uint64_t elem_of(const zo_header *h, uint64_t q, uint32_t pos) {
 uint64_t zo_encode_bound(uint64_t rows, uint64_t cols, uint32_t layout, uint32_t chunk_elems) {
   zo_header h;
   if (geometry(rows, cols, layout, chunk_elems, &h) != ZO_OK) return 0;
-  uint64_t per_tile = 64 + (uint64_t)h.tile_elems * ZO_MAX_CODE_LEN / 8 + 16;
+  uint64_t per_tile = ZO_REC_HEAD + (uint64_t)h.tile_elems * ZO_MAX_CODE_LEN / 8 + 16;
   uint64_t tpc = h.chunk_elems / h.tile_elems;
   uint64_t per_chunk = round_up(4 * (tpc + 1), 16);
   return h.payload_off + h.n_tiles * per_tile + h.n_chunks * per_chunk + h.sm_bytes + 64;
@@ -354,21 +361,22 @@ int zo_encode(const uint16_t *x, uint64_t rows, uint64_t cols, uint32_t layout, 
       uint64_t q = (uint64_t)q0 + t;
       wr32(chunk + 4ull * t, (uint32_t)(rel / 16));
       uint8_t *rec = chunk + rel;
-      uint64_t rec_max = 64 + (uint64_t)h.tile_elems * ZO_MAX_CODE_LEN / 8 + 16;
+      uint64_t rec_max = ZO_REC_HEAD + (uint64_t)h.tile_elems * ZO_MAX_CODE_LEN / 8 + 16;
       memset(rec, 0, rec_max);
       uint64_t p = 0; /* bit position in the record's bit area */
-      for (uint32_t lane = 0; lane < 32; ++lane) {
-        uint64_t p_start = p;
-        for (uint32_t i = 0; i < I; ++i)
-          for (uint32_t j = 0; j < 8; ++j) {
-            uint64_t f = elem_of(&h, q, (i * 32 + lane) * 8 + j);
-            if (f == UINT64_MAX) continue;
-            uint32_t s = exp[f];
-            for (int b = len[s] - 1; b >= 0; --b) put_bit(rec + 64, p++, (code[s] >> b) & 1u);
-          }
-        wr16(rec + 2 * lane, (uint32_t)(p - p_start));
-      }
-      rel += round_up(64 + (p + 7) / 8, 16);
+      for (uint32_t lane = 0; lane < 32; ++lane)
+        for (uint32_t hh = 0; hh < 2; ++hh) {
+          uint64_t p_start = p;
+          for (uint32_t i = hh; i < I; i += 2)
+            for (uint32_t j = 0; j < 8; ++j) {
+              uint64_t f = elem_of(&h, q, (i * 32 + lane) * 8 + j);
+              if (f == UINT64_MAX) continue;
+              uint32_t s = exp[f];
+              for (int b = len[s] - 1; b >= 0; --b) put_bit(rec + ZO_REC_HEAD, p++, (code[s] >> b) & 1u);
+            }
+          wr16(rec + 2 * (2 * lane + hh), (uint32_t)(p - p_start));
+        }
+      rel += round_up(ZO_REC_HEAD + (p + 7) / 8, 16);
     }
     wr32(chunk + 4ull * m, (uint32_t)(rel / 16));
     at += rel;
@@ -387,7 +395,7 @@ int zo_encode(const uint16_t *x, uint64_t rows, uint64_t cols, uint32_t layout, 
     }
 
   wr32(blob + 0, ZO_MAGIC);
-  wr32(blob + 4, 1);
+  wr32(blob + 4, ZO_VERSION);
   wr64(blob + 8, h.n_elems);
   wr32(blob + 16, h.rows);
   wr32(blob + 20, h.cols);
@@ -408,7 +416,7 @@ int zo_encode(const uint16_t *x, uint64_t rows, uint64_t cols, uint32_t layout, 
 
 static int parse_header(const uint8_t *blob, uint64_t bytes, zo_header *h) {
   if (bytes < ZO_CHUNKOFF_OFF + 8) return ZO_ERR_FORMAT;
-  if (rd32(blob) != ZO_MAGIC || rd32(blob + 4) != 1) return ZO_ERR_FORMAT;
+  if (rd32(blob) != ZO_MAGIC || rd32(blob + 4) != ZO_VERSION) return ZO_ERR_FORMAT;
   zo_header g;
   uint64_t n = rd64(blob + 8);
   uint32_t rows = rd32(blob + 16), cols = rd32(blob + 20);
@@ -474,14 +482,15 @@ int zo_decode_chunk(const uint8_t *blob, uint64_t bytes, uint32_t k, uint16_t *o
   for (uint32_t t = 0; t < m; ++t) {
     uint64_t q = (uint64_t)q0 + t;
     uint64_t r0 = (uint64_t)rd32(chunk + 4ull * t) * 16, r1 = (uint64_t)rd32(chunk + 4ull * (t + 1)) * 16;
-    if (r1 < r0 + 64 || r1 > chunk_bytes) return ZO_ERR_CORRUPT;
+    if (r1 < r0 + ZO_REC_HEAD || r1 > chunk_bytes) return ZO_ERR_CORRUPT;
     const uint8_t *rec = chunk + r0;
-    uint64_t area_bits = (r1 - r0 - 64) * 8;
+    uint64_t area_bits = (r1 - r0 - ZO_REC_HEAD) * 8;
     uint64_t p = 0;
-    for (uint32_t lane = 0; lane < 32; ++lane) {
-      uint64_t p_end = p + rd16(rec + 2 * lane);
+    for (uint32_t sub = 0; sub < 64; ++sub) {
+      uint32_t lane = sub / 2, hh = sub % 2;
+      uint64_t p_end = p + rd16(rec + 2 * sub);
       if (p_end > area_bits) return ZO_ERR_CORRUPT;
-      for (uint32_t i = 0; i < I; ++i)
+      for (uint32_t i = hh; i < I; i += 2)
         for (uint32_t j = 0; j < 8; ++j) {
           uint32_t pos = (i * 32 + lane) * 8 + j;
           uint64_t f = elem_of(&h, q, pos);
@@ -490,7 +499,7 @@ int zo_decode_chunk(const uint8_t *blob, uint64_t bytes, uint32_t k, uint16_t *o
           int L = 0, found = 0;
           while (L < (int)h.max_code_len) {
             if (p >= p_end) return ZO_ERR_CORRUPT;
-            c = (c << 1) | get_bit(rec + 64, p++);
+            c = (c << 1) | get_bit(rec + ZO_REC_HEAD, p++);
             ++L;
             if (c >= first[L] && c - first[L] < count[L]) { found = 1; break; }
           }
