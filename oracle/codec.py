@@ -108,7 +108,7 @@ def canonical_codes(lengths):
 
 
 def encode(x, rows=None, cols=None, layout=0, chunk_elems=4096, max_code_len=12):
-    """bf16 bit patterns (uint16) -> ZMOE v1 blob (uint8 array)."""
+    """bf16 bit patterns (uint16) -> ZMOE v2 blob (uint8 array)."""
     x = np.ascontiguousarray(x, dtype=np.uint16)
     if rows is None:
         rows, cols = (x.shape if x.ndim == 2 else (1, x.size))
@@ -136,7 +136,7 @@ def info(blob):
 
 
 def decode(blob):
-    """ZMOE v1 blob -> bf16 bit patterns (uint16, flat, row-major)."""
+    """ZMOE v2 blob -> bf16 bit patterns (uint16, flat, row-major)."""
     blob = np.ascontiguousarray(blob, dtype=np.uint8)
     n = info(blob)["n_elems"]
     out = np.zeros(n, np.uint16)

@@ -60,16 +60,20 @@
  *                           this table, tile_off[m] the size of the chunk;
  *     zero padding to 16 bytes, then m tile records.
  *   Tile record:
- *     u16 sub_bits[64]      number of code bits of each sub-stream; every lane
- *                           has two, entry 2*lane + h for h = 0, 1;
- *     the 64 sub-streams in that order (lane 0 h 0, lane 0 h 1, lane 1 h 0, ...),
- *     concatenated bit by bit with no padding between them, stored as u32
- *     words whose bits are consumed from bit 31 down to bit 0; zero padding to
- *     a 16-byte boundary.
- *   Sub-stream (lane, h) codes the lane's existing elements of the iterations
- *   i = h, h+2, h+4, ... < I in that order, j = 0..7 inside each.  (Two
- *   independent streams per lane let a decoder work on two codes at a time; the
- *   paper leaves the order of elements inside a shard open.)
+ *     u16 sub_bits[32]      number of code bits of each lane (both of its
+ *                           sub-streams together);
+ *     the 32 lanes' bit ranges, lane 0 first, concatenated with no padding
+ *     between them, stored as u32 words whose bits are consumed from bit 31
+ *     down to bit 0; zero padding to a 16-byte boundary.
+ *   A lane has two sub-streams inside its bit range [S, E):
+ *     sub-stream 0 codes the lane's existing elements of the even iterations
+ *       i = 0, 2, 4, ... < I (j = 0..7 inside each) and runs forwards from S:
+ *       its k-th bit is bit S + k;
+ *     sub-stream 1 codes those of the odd iterations i = 1, 3, 5, ... < I and
+ *       runs backwards from E: its k-th bit is bit E - 1 - k.
+ *   The two meet without a gap.  (Two independent streams per lane let a decoder
+ *   work on two codes at a time at no cost in size; the paper leaves the order
+ *   of elements inside a shard open.)
  *
  *   Sign+mantissa section: byte q*tile_elems + pos holds
  *     (sign << 7) | mantissa  of the element at (q, pos); zero padded to 16.
@@ -95,7 +99,7 @@
 #define ZO_CHUNKOFF_OFF 320u
 #define ZO_MAX_CODE_LEN 12
 #define ZO_VERSION 2u
-#define ZO_REC_HEAD 128u /* u16 sub_bits[64] */
+#define ZO_REC_HEAD 64u /* u16 sub_bits[32] */
 
 /* ---- little-endian field access ---------------------------------------- */
 static uint32_t rd32(const uint8_t *p) {
@@ -364,18 +368,29 @@ int zo_encode(const uint16_t *x, uint64_t rows, uint64_t cols, uint32_t layout, 
       uint64_t rec_max = ZO_REC_HEAD + (uint64_t)h.tile_elems * ZO_MAX_CODE_LEN / 8 + 16;
       memset(rec, 0, rec_max);
       uint64_t p = 0; /* bit position in the record's bit area */
-      for (uint32_t lane = 0; lane < 32; ++lane)
-        for (uint32_t hh = 0; hh < 2; ++hh) {
-          uint64_t p_start = p;
-          for (uint32_t i = hh; i < I; i += 2)
-            for (uint32_t j = 0; j < 8; ++j) {
-              uint64_t f = elem_of(&h, q, (i * 32 + lane) * 8 + j);
-              if (f == UINT64_MAX) continue;
-              uint32_t s = exp[f];
-              for (int b = len[s] - 1; b >= 0; --b) put_bit(rec + ZO_REC_HEAD, p++, (code[s] >> b) & 1u);
+      for (uint32_t lane = 0; lane < 32; ++lane) {
+        /* size of the lane's bit range first, then both sub-streams into it */
+        uint64_t lane_bits = 0;
+        for (uint32_t i = 0; i < I; ++i)
+          for (uint32_t j = 0; j < 8; ++j) {
+            uint64_t f = elem_of(&h, q, (i * 32 + lane) * 8 + j);
+            if (f != UINT64_MAX) lane_bits += len[exp[f]];
+          }
+        uint64_t fwd = p, bwd = p + lane_bits; /* next bit of sub-stream 0; one past the next bit of sub-stream 1 */
+        for (uint32_t i = 0; i < I; ++i)
+          for (uint32_t j = 0; j < 8; ++j) {
+            uint64_t f = elem_of(&h, q, (i * 32 + lane) * 8 + j);
+            if (f == UINT64_MAX) continue;
+            uint32_t s = exp[f];
+            for (int b = len[s] - 1; b >= 0; --b) {
+              if (i % 2 == 0) put_bit(rec + ZO_REC_HEAD, fwd++, (code[s] >> b) & 1u);
+              else put_bit(rec + ZO_REC_HEAD, --bwd, (code[s] >> b) & 1u);
             }
-          wr16(rec + 2 * (2 * lane + hh), (uint32_t)(p - p_start));
-        }
+          }
+        /* fwd == bwd here: the sub-streams meet */
+        wr16(rec + 2 * lane, (uint32_t)lane_bits);
+        p += lane_bits;
+      }
       rel += round_up(ZO_REC_HEAD + (p + 7) / 8, 16);
     }
     wr32(chunk + 4ull * m, (uint32_t)(rel / 16));
@@ -486,11 +501,11 @@ int zo_decode_chunk(const uint8_t *blob, uint64_t bytes, uint32_t k, uint16_t *o
     const uint8_t *rec = chunk + r0;
     uint64_t area_bits = (r1 - r0 - ZO_REC_HEAD) * 8;
     uint64_t p = 0;
-    for (uint32_t sub = 0; sub < 64; ++sub) {
-      uint32_t lane = sub / 2, hh = sub % 2;
-      uint64_t p_end = p + rd16(rec + 2 * sub);
+    for (uint32_t lane = 0; lane < 32; ++lane) {
+      uint64_t p_end = p + rd16(rec + 2 * lane);
       if (p_end > area_bits) return ZO_ERR_CORRUPT;
-      for (uint32_t i = hh; i < I; i += 2)
+      uint64_t fwd = p, bwd = p_end;
+      for (uint32_t i = 0; i < I; ++i)
         for (uint32_t j = 0; j < 8; ++j) {
           uint32_t pos = (i * 32 + lane) * 8 + j;
           uint64_t f = elem_of(&h, q, pos);
@@ -498,8 +513,9 @@ int zo_decode_chunk(const uint8_t *blob, uint64_t bytes, uint32_t k, uint16_t *o
           uint32_t c = 0;
           int L = 0, found = 0;
           while (L < (int)h.max_code_len) {
-            if (p >= p_end) return ZO_ERR_CORRUPT;
-            c = (c << 1) | get_bit(rec + ZO_REC_HEAD, p++);
+            if (fwd >= bwd) return ZO_ERR_CORRUPT; /* the lane's bits are used up */
+            uint32_t bit = (i % 2 == 0) ? get_bit(rec + ZO_REC_HEAD, fwd++) : get_bit(rec + ZO_REC_HEAD, --bwd);
+            c = (c << 1) | bit;
             ++L;
             if (c >= first[L] && c - first[L] < count[L]) { found = 1; break; }
           }
@@ -508,7 +524,8 @@ int zo_decode_chunk(const uint8_t *blob, uint64_t bytes, uint32_t k, uint16_t *o
           uint8_t s = smsec[q * h.tile_elems + pos];
           zo_merge(&e, &s, 1, &out[f]);
         }
-      if (p != p_end) return ZO_ERR_CORRUPT;
+      if (fwd != bwd) return ZO_ERR_CORRUPT; /* the sub-streams must meet exactly */
+      p = p_end;
     }
   }
   return ZO_OK;

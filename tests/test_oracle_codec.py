@@ -195,11 +195,23 @@ def test_canonical_codes_are_ordered_and_prefix_free():
 
 # ---------------------------------------------------------------- container
 
+def _bits_of_bytes(values):
+    """MSB-first bits of a list of 8-bit codes."""
+    return [(v >> b) & 1 for v in values for b in range(7, -1, -1)]
+
+
+def _pack_words(bits):
+    """Bits -> bytes of a u32 word stream consumed from bit 31 down, little-endian in memory."""
+    bits = list(bits) + [0] * (-len(bits) % 32)
+    by = np.packbits(np.array(bits, dtype=np.uint8)).reshape(-1, 4)[:, ::-1]
+    return by.ravel()
+
+
 def test_uniform_exponents_store_the_raw_exponent_bytes():
-    """All 256 exponents equally frequent -> every code is the 8-bit symbol
-    itself, so a tile's bit area is the exponent bytes in sub-stream order (lane,
-    then even iterations before odd ones, then i, then j), packed four to a word
-    with the first byte in bits 31..24.  Needs no Huffman."""
+    """All 256 exponents equally frequent -> every code is the 8-bit symbol itself, so a
+    lane's bit range is: the exponent bytes of its even iterations, forwards, then those
+    of its odd iterations written backwards from the end of the range (the last byte of
+    the range is the bit-reversed first odd-iteration exponent).  Needs no Huffman."""
     rng = np.random.default_rng(11)
     e = np.tile(np.arange(256, dtype=np.uint16), 32)
     rng.shuffle(e)
@@ -211,17 +223,20 @@ def test_uniform_exponents_store_the_raw_exponent_bytes():
     assert hdr["n_chunks"] == 2 and hdr["n_tiles"] == 2 and hdr["tile_elems"] == 4096
     pay = hdr["payload_off"]
     offs = blob[320:320 + 8 * 3].view(np.uint64)
-    rec_bytes = 128 + 4096
+    rec_bytes = 64 + 4096
     assert offs.tolist() == [0, (16 + rec_bytes) * 8, 2 * (16 + rec_bytes) * 8]
     for q in range(2):
         chunk = blob[pay + q * (16 + rec_bytes): pay + (q + 1) * (16 + rec_bytes)]
         assert chunk[:8].view(np.uint32).tolist() == [1, 1 + rec_bytes // 16]
         rec = chunk[16:]
-        assert (rec[:128].view(np.uint16) == 64 * 8).all()                      # 64 sub-streams of 64 codes
-        tile = e[q * 4096:(q + 1) * 4096].astype(np.uint8).reshape(8, 2, 32, 8)  # [i // 2, i % 2, lane, j]
-        stream = tile.transpose(2, 1, 0, 3).ravel()                             # lane, parity of i, i // 2, j
-        expect = stream.reshape(-1, 4)[:, ::-1].ravel()                         # big-endian words in LE memory
-        assert np.array_equal(rec[128:], expect)
+        assert (rec[:64].view(np.uint16) == 128 * 8).all()
+        tile = e[q * 4096:(q + 1) * 4096].astype(np.uint8).reshape(16, 32, 8)   # [i, lane, j]
+        bits = []
+        for lane in range(32):
+            even = tile[0::2, lane, :].ravel().tolist()
+            odd = tile[1::2, lane, :].ravel().tolist()
+            bits += _bits_of_bytes(even) + _bits_of_bytes(odd)[::-1]
+        assert np.array_equal(rec[64:], _pack_words(bits))
     # sign+mantissa section: raw bytes in element order for the linear layout
     smsec = blob[pay + hdr["payload_bytes"]:]
     assert np.array_equal(smsec, ((x >> 8) & 0x80 | x & 0x7F).astype(np.uint8))
@@ -230,8 +245,8 @@ def test_uniform_exponents_store_the_raw_exponent_bytes():
 
 def test_uniform_exponents_odd_iteration_count_and_ragged_tail():
     """Three iterations per tile (chunk of 768 elements) and a tensor that ends in the
-    middle of a lane's group: sub-stream (lane, 0) holds iterations 0 and 2,
-    (lane, 1) holds iteration 1, and elements past the end are not coded."""
+    middle of a lane's group: sub-stream 0 holds iterations 0 and 2, sub-stream 1
+    iteration 1, and elements past the end are not coded."""
     n = 256 * 5 + 13
     rng = np.random.default_rng(5)
     e = np.concatenate([np.tile(np.arange(256, dtype=np.uint16), 5), np.arange(13, dtype=np.uint16)])
@@ -247,17 +262,16 @@ def test_uniform_exponents_odd_iteration_count_and_ragged_tail():
         chunk = blob[pay + offs[q]: pay + offs[q + 1]]
         first, end = chunk[:8].view(np.uint32).tolist()
         rec = chunk[16 * first: 16 * end]
-        counts, stream = [], []
+        counts, bits = [], []
         for lane in range(32):
-            for h in range(2):
-                mine = [int(e[f]) for i in range(h, 3, 2) for j in range(8)
-                        for f in [q * 768 + (i * 32 + lane) * 8 + j] if f < n]
-                counts.append(8 * len(mine))
-                stream += mine
-        assert rec[:128].view(np.uint16).tolist() == counts
-        body = np.array(stream + [0] * (-len(stream) % 4), dtype=np.uint8).reshape(-1, 4)[:, ::-1].ravel()
-        assert np.array_equal(rec[128:128 + body.size], body)
-        assert not rec[128 + body.size:].any() and rec.size == -(-(128 + len(stream)) // 16) * 16
+            sub = [[int(e[f]) for i in range(h, 3, 2) for j in range(8)
+                    for f in [q * 768 + (i * 32 + lane) * 8 + j] if f < n] for h in range(2)]
+            counts.append(8 * (len(sub[0]) + len(sub[1])))
+            bits += _bits_of_bytes(sub[0]) + _bits_of_bytes(sub[1])[::-1]
+        assert rec[:64].view(np.uint16).tolist() == counts
+        body = _pack_words(bits)
+        assert np.array_equal(rec[64:64 + body.size], body)
+        assert not rec[64 + body.size:].any() and rec.size == -(-(64 + len(bits) // 8) // 16) * 16
     assert np.array_equal(codec.decode(blob), x)
 
 
@@ -305,7 +319,7 @@ def test_empty_and_single_symbol_tensors():
     blob = codec.encode(x, chunk_elems=1024)
     assert np.array_equal(codec.decode(blob), x)
     rec = blob[codec.info(blob)["payload_off"] + 16:]
-    assert int(rec[:128].view(np.uint16).sum()) == 1000    # one bit per element
+    assert int(rec[:64].view(np.uint16).sum()) == 1000     # one bit per element
 
 
 def test_chunks_decode_independently_and_in_any_order():
