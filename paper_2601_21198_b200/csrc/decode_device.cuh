@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <type_traits>
 
 #include "zipmoe.h"
 
@@ -287,48 +288,6 @@ __device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c
 }
 
 // ---- tile decoder -------------------------------------------------------------
-template <bool STAGED>
-struct WordSource {
-  uint32_t at_s;             // shared address of the next unread word (STAGED)
-  const uint32_t *at_g;      // global address of the next unread word (!STAGED)
-  __device__ __forceinline__ uint32_t pop() {
-    if (STAGED) {
-      const uint32_t v = lds_u32(at_s);
-      at_s += 4;
-      return v;
-    }
-    return __ldg(at_g++);
-  }
-  // If bit 5 of pos is set (a whole word has been consumed): b_hi <- b_lo, b_lo <- b_next, b_next <- the
-  // following word, clear the bit.  b_next is loaded one word early so that its latency is off the decode chain.
-  // Predicated, no branch.
-  __device__ __forceinline__ void advance(uint32_t &pos, uint32_t &b_hi, uint32_t &b_lo, uint32_t &b_next) {
-    if (STAGED) {
-      asm volatile(
-          "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
-          "and.b32 t, %0, 32;\n\t"
-          "setp.ne.u32 p, t, 0;\n\t"
-          "@p mov.b32 %1, %2;\n\t"
-          "@p mov.b32 %2, %3;\n\t"
-          "@p ld.shared.u32 %3, [%4];\n\t"
-          "@p add.u32 %4, %4, 4;\n\t"
-          "@p xor.b32 %0, %0, 32;\n\t}"
-          : "+r"(pos), "+r"(b_hi), "+r"(b_lo), "+r"(b_next), "+r"(at_s));
-    } else {
-      asm volatile(
-          "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
-          "and.b32 t, %0, 32;\n\t"
-          "setp.ne.u32 p, t, 0;\n\t"
-          "@p mov.b32 %1, %2;\n\t"
-          "@p mov.b32 %2, %3;\n\t"
-          "@p ld.global.nc.u32 %3, [%4];\n\t"
-          "@p add.u64 %4, %4, 4;\n\t"
-          "@p xor.b32 %0, %0, 32;\n\t}"
-          : "+r"(pos), "+r"(b_hi), "+r"(b_lo), "+r"(b_next), "+l"(at_g));
-    }
-  }
-};
-
 // a*b + c on the multiply-add pipe (keeps pure integer adds and shifts-by-constant
 // off the ALU pipe, which the variable shifts and logic ops of the decoder fill)
 __device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) {
@@ -337,19 +296,101 @@ __device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) 
   return d;
 }
 
-// One lane's view of a tile record: its sub-stream of code bits and the table.
-// The code bits of a lane form a stream of u32 words consumed from bit 31 down.
-// The lane keeps two consecutive words of it (b_hi:b_lo) and the bit position
-// `pos` of the next code inside them (pos mod 64 < 32 between batches).  A batch
-// takes the 32 bits at pos into one register and decodes from its top:
+// One sub-stream of a lane: a stream of u32 words of which the lane keeps two in
+// registers (`cur` holds the next code bit, `nxt` the bits after it) plus a third,
+// loaded one word early so that its latency is off the decode chain, and the
+// number `pos` of bits of `cur` already consumed (pos mod 64 < 32 between batches).
+//   DIR = +1 (forward sub-stream): words in ascending address order, each consumed
+//         from bit 31 down;
+//   DIR = -1 (backward sub-stream): words in descending address order, each consumed
+//         from bit 0 up.
+// window() returns the next 32 code bits with the first one in bit 31.
+template <bool STAGED, int DIR>
+struct SubStream {
+  uint32_t pos, cur, nxt, ahead;
+  uint32_t at_s;             // shared address of the next word to load (STAGED)
+  const uint32_t *at_g;      // global address of the next word to load (!STAGED)
+  const uint32_t *floor_g;   // the record's first word: a backward stream of a corrupt record stops here (!STAGED)
+
+  __device__ __forceinline__ uint32_t pop() {
+    if (STAGED) {
+      const uint32_t v = lds_u32(at_s);
+      at_s += (uint32_t)(4 * DIR);
+      return v;
+    }
+    const uint32_t v = __ldg(at_g);
+    at_g += DIR;
+    if (DIR < 0 && at_g < floor_g) at_g = floor_g;
+    return v;
+  }
+  // word = index of the word that holds the next code bit, counted from `words_s` / `words_g`
+  // (may be -1 for an empty backward stream at the very start of the bit area: the word before it exists)
+  __device__ __forceinline__ void start(uint32_t words_s, const uint32_t *words_g, const uint32_t *floor, int32_t word,
+                                        uint32_t consumed) {
+    at_s = words_s + 4 * word;
+    at_g = words_g + word;
+    floor_g = floor;
+    if (!STAGED && DIR < 0 && at_g < floor_g) at_g = floor_g;
+    pos = consumed;
+    cur = pop();
+    nxt = pop();
+    ahead = pop();
+  }
+  __device__ __forceinline__ uint32_t window() const {
+    if (DIR > 0) return __funnelshift_l(nxt, cur, pos);
+    return __brev(__funnelshift_r(cur, nxt, pos));
+  }
+  // If bit 5 of pos is set (a whole word has been consumed): cur <- nxt, nxt <- ahead, ahead <- the
+  // following word, clear the bit.  Predicated, no branch.
+  __device__ __forceinline__ void advance() {
+    if (STAGED) {
+      if (DIR > 0)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
+            "and.b32 t, %0, 32;\n\t"
+            "setp.ne.u32 p, t, 0;\n\t"
+            "@p mov.b32 %1, %2;\n\t"
+            "@p mov.b32 %2, %3;\n\t"
+            "@p ld.shared.u32 %3, [%4];\n\t"
+            "@p add.u32 %4, %4, 4;\n\t"
+            "@p xor.b32 %0, %0, 32;\n\t}"
+            : "+r"(pos), "+r"(cur), "+r"(nxt), "+r"(ahead), "+r"(at_s));
+      else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
+            "and.b32 t, %0, 32;\n\t"
+            "setp.ne.u32 p, t, 0;\n\t"
+            "@p mov.b32 %1, %2;\n\t"
+            "@p mov.b32 %2, %3;\n\t"
+            "@p ld.shared.u32 %3, [%4];\n\t"
+            "@p add.u32 %4, %4, -4;\n\t"
+            "@p xor.b32 %0, %0, 32;\n\t}"
+            : "+r"(pos), "+r"(cur), "+r"(nxt), "+r"(ahead), "+r"(at_s));
+    } else if (pos & 32u) {
+      cur = nxt;
+      nxt = ahead;
+      ahead = pop();
+      pos ^= 32u;
+    }
+  }
+};
+
+// One lane's view of a tile record: its two sub-streams of code bits and the
+// lookup table.  The record's bit area is a stream of u32 words; bit y of it is
+// bit 31 - (y mod 32) of word y / 32.  The lane's codes occupy the bit range
+// [S, E) (S = sum of the bit counts of the lanes before, E = S + the lane's own):
+//   sub-stream 0 (the lane's elements of even iterations) runs forwards from S,
+//   sub-stream 1 (odd iterations) runs backwards from E: its k-th bit is bit E-1-k.
+// The two are independent, so the lane decodes one code of each at a time and the
+// two lookup chains overlap.  A batch takes a stream's next 32 bits into one
+// register and decodes from its top:
 //   FAST  (no code longer than 8 bits): four codes per batch, looked up in the
 //         lane table with the top 8 bits;
 //   !FAST (codes up to 12 bits): two codes per batch, looked up in the wide
 //         table with the top 12 bits.
-// Whole table entries are added to pos: their low 4 bits are the code length and
-// bits 4..6 are zero, so the low 7 bits of pos stay exact and the rest is
-// ignored (the funnel shifts take the shift amount mod 32).  When bit 5 of pos
-// is set a whole word has been consumed and the next one is shifted in.
+// Whole table entries, (symbol << 7) | length, are added to a stream's pos: their
+// low 4 bits are the code length and bits 4..6 are zero, so the low 7 bits of pos
+// stay exact and the rest is ignored (the funnel shifts take the amount mod 32).
 // KIND: kLutWide (12-bit shared table), kLutLane32 (8-bit table, one u32 copy per lane: no bank conflicts, 32 KB) or
 // kLutLane16 (8-bit table, one u16 copy per lane: two lanes share a bank, 16 KB).
 constexpr int kLutWide = 0, kLutLane32 = 1, kLutLane16 = 2;
@@ -357,12 +398,13 @@ constexpr int kLutWide = 0, kLutLane32 = 1, kLutLane16 = 2;
 template <bool STAGED, int KIND>
 struct LaneDecoder {
   static constexpr bool FAST = KIND != kLutWide;
-  WordSource<STAGED> src;
-  uint32_t pos, b_hi, b_lo, b_next, lut, my_lut;
+  SubStream<STAGED, +1> s0;
+  SubStream<STAGED, -1> s1;
+  uint32_t lut, my_lut;
 
   // record in shared memory at rec_s (STAGED) or in global memory at rec_g; lut =
   // shared address of the lane table (FAST) or the wide table (!FAST).  Turns the
-  // record's 32 bit counts into this lane's start by a warp-shuffle prefix sum.
+  // record's 32 bit counts into this lane's range by a warp-shuffle prefix sum.
   // Returns false (warp-uniform) if the counts overrun the record.
   __device__ __forceinline__ bool init(uint32_t rec_s, const uint8_t *rec_g, uint32_t rec_bytes, uint32_t lut_addr,
                                        uint32_t lane) {
@@ -377,13 +419,15 @@ struct LaneDecoder {
     }
     const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
     if (64u * 8u + total > rec_bytes * 8u) return false;
-    const uint32_t start = incl - my_bits;
-    src.at_s = rec_s + 64 + 4 * (start >> 5);
-    src.at_g = reinterpret_cast<const uint32_t *>(rec_g + 64) + (start >> 5);
-    pos = start & 31;
-    b_hi = src.pop();
-    b_lo = src.pop();
-    b_next = src.pop();
+    const uint32_t *floor = reinterpret_cast<const uint32_t *>(rec_g);
+    const uint32_t *words_g = floor + 16;
+    const uint32_t words_s = rec_s + 64;
+    const uint32_t S = incl - my_bits;
+    s0.start(words_s, words_g, floor, (int32_t)(S >> 5), S & 31u);
+    // the backward stream's next bit is bit incl - 1 (bit -1, in the word before the bit area, if the
+    // range is empty and starts at 0: nothing is decoded from it then)
+    const uint32_t y = incl + 31u;   // that bit, plus one word
+    s1.start(words_s, words_g, floor, (int32_t)(y >> 5) - 1, 31u - (y & 31u));
     lut = lut_addr;
     my_lut = lut_addr + (KIND == kLutLane16 ? 2 : 4) * lane;
     return true;
@@ -393,51 +437,100 @@ struct LaneDecoder {
     if (KIND == kLutLane16) return lds_u16(mad_u32(w >> (32 - kLaneLutBits), 64u, my_lut));
     return lds_u16(mad_u32(w >> (32 - kWideLutBits), 2u, lut));
   }
-  __device__ __forceinline__ void pair(uint32_t &ea, uint32_t &eb) {   // two codes from the 32 bits at pos
-    uint32_t w = __funnelshift_l(b_lo, b_hi, pos);
-    ea = lookup(w);
-    w = __funnelshift_l(0u, w, ea);
-    eb = lookup(w);
-    pos += ea + eb;
-    src.advance(pos, b_hi, b_lo, b_next);
+  __device__ static __forceinline__ uint32_t next(uint32_t w, uint32_t entry) {   // drop the code just decoded
+    return __funnelshift_l(0u, w, entry);
   }
-  __device__ __forceinline__ void quad(uint32_t &ea, uint32_t &eb, uint32_t &ec, uint32_t &ed) {   // four codes <= 8 bits
-    uint32_t w = __funnelshift_l(b_lo, b_hi, pos);
-    ea = lookup(w);
-    w = __funnelshift_l(0u, w, ea);
-    eb = lookup(w);
-    w = __funnelshift_l(0u, w, eb);
-    ec = lookup(w);
-    w = __funnelshift_l(0u, w, ec);
-    ed = lookup(w);
-    pos += (ea + eb) + (ec + ed);
-    src.advance(pos, b_hi, b_lo, b_next);
+  // 8 exponent entries and 8 sign+mantissa bytes -> 8 bf16
+  __device__ static __forceinline__ uint4 merge(const uint2 smv, const uint32_t (&e)[8]) {
+    constexpr uint32_t kKeep = 0x807F807Fu;   // sign and mantissa bits of two bf16
+    uint4 o;
+    o.x = (__byte_perm(smv.x, 0, 0x1100) & kKeep) | (mad_u32(e[1], 65536u, e[0]) & ~kKeep);
+    o.y = (__byte_perm(smv.x, 0, 0x3322) & kKeep) | (mad_u32(e[3], 65536u, e[2]) & ~kKeep);
+    o.z = (__byte_perm(smv.y, 0, 0x1100) & kKeep) | (mad_u32(e[5], 65536u, e[4]) & ~kKeep);
+    o.w = (__byte_perm(smv.y, 0, 0x3322) & kKeep) | (mad_u32(e[7], 65536u, e[6]) & ~kKeep);
+    return o;
   }
+  // The next 8 elements of both sub-streams (one group of an even iteration and one of the
+  // following odd iteration) merged with their sign+mantissa bytes.  The two decode chains are
+  // written interleaved so that each one's lookup latency is covered by the other's work.
+  __device__ __forceinline__ void group2(const uint2 sm0, const uint2 sm1, uint4 &o0, uint4 &o1) {
+    uint32_t e[8], f[8];
+    if (FAST) {
+#pragma unroll
+      for (int h = 0; h < 8; h += 4) {
+        uint32_t w = s0.window(), x = s1.window();
+        e[h] = lookup(w);
+        f[h] = lookup(x);
+        w = next(w, e[h]);
+        x = next(x, f[h]);
+        e[h + 1] = lookup(w);
+        f[h + 1] = lookup(x);
+        w = next(w, e[h + 1]);
+        x = next(x, f[h + 1]);
+        e[h + 2] = lookup(w);
+        f[h + 2] = lookup(x);
+        w = next(w, e[h + 2]);
+        x = next(x, f[h + 2]);
+        e[h + 3] = lookup(w);
+        f[h + 3] = lookup(x);
+        s0.pos += (e[h] + e[h + 1]) + (e[h + 2] + e[h + 3]);
+        s1.pos += (f[h] + f[h + 1]) + (f[h + 2] + f[h + 3]);
+        s0.advance();
+        s1.advance();
+      }
+    } else {
+#pragma unroll
+      for (int h = 0; h < 8; h += 2) {
+        uint32_t w = s0.window(), x = s1.window();
+        e[h] = lookup(w);
+        f[h] = lookup(x);
+        w = next(w, e[h]);
+        x = next(x, f[h]);
+        e[h + 1] = lookup(w);
+        f[h + 1] = lookup(x);
+        s0.pos += e[h] + e[h + 1];
+        s1.pos += f[h] + f[h + 1];
+        s0.advance();
+        s1.advance();
+      }
+    }
+    o0 = merge(sm0, e);
+    o1 = merge(sm1, f);
+  }
+  // one code of sub-stream WHICH
+  template <int WHICH>
   __device__ __forceinline__ uint32_t single() {
-    const uint32_t e = lookup(__funnelshift_l(b_lo, b_hi, pos));
-    pos += e;
-    src.advance(pos, b_hi, b_lo, b_next);
+    uint32_t e;
+    if (WHICH == 0) {
+      e = lookup(s0.window());
+      s0.pos += e;
+      s0.advance();
+    } else {
+      e = lookup(s1.window());
+      s1.pos += e;
+      s1.advance();
+    }
     return e;
   }
-  // the next 8 elements of this lane merged with their sign+mantissa bytes: 8 bf16
-  __device__ __forceinline__ uint4 group(const uint2 smv) {
-    constexpr uint32_t kKeep = 0x807F807Fu;   // sign and mantissa bits of two bf16
-    uint32_t e0, e1, e2, e3, e4, e5, e6, e7;
-    if (FAST) {
-      quad(e0, e1, e2, e3);
-      quad(e4, e5, e6, e7);
-    } else {
-      pair(e0, e1);
-      pair(e2, e3);
-      pair(e4, e5);
-      pair(e6, e7);
+  // the next 8 elements of sub-stream WHICH alone (the ragged end of a tensor)
+  template <int WHICH>
+  __device__ __forceinline__ uint4 group1(const uint2 smv) {
+    uint32_t e[8];
+#pragma unroll
+    for (int h = 0; h < 8; h += 2) {
+      uint32_t w = WHICH == 0 ? s0.window() : s1.window();
+      e[h] = lookup(w);
+      w = next(w, e[h]);
+      e[h + 1] = lookup(w);
+      if (WHICH == 0) {
+        s0.pos += e[h] + e[h + 1];
+        s0.advance();
+      } else {
+        s1.pos += e[h] + e[h + 1];
+        s1.advance();
+      }
     }
-    uint4 o;
-    o.x = (__byte_perm(smv.x, 0, 0x1100) & kKeep) | (mad_u32(e1, 65536u, e0) & ~kKeep);
-    o.y = (__byte_perm(smv.x, 0, 0x3322) & kKeep) | (mad_u32(e3, 65536u, e2) & ~kKeep);
-    o.z = (__byte_perm(smv.y, 0, 0x1100) & kKeep) | (mad_u32(e5, 65536u, e4) & ~kKeep);
-    o.w = (__byte_perm(smv.y, 0, 0x3322) & kKeep) | (mad_u32(e7, 65536u, e6) & ~kKeep);
-    return o;
+    return merge(smv, e);
   }
 };
 
@@ -458,8 +551,7 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
                                                 uint32_t lane, Feed &feed, Sink &sink) {
   LaneDecoder<STAGED, FAST ? kLutLane32 : kLutWide> dec;
   if (!dec.init(rec_s, rec_g, rec_bytes, lut, lane)) return kStatusBadBitCount;
-  auto group = [&](uint32_t sm_at) -> uint4 { return dec.group(lds_v2(sm_at)); };
-  auto single = [&]() -> uint32_t { return dec.single(); };
+  static_assert(kPieceIters % 2 == 0, "a piece holds whole pairs of iterations");
 
   const uint32_t pieces = (iters + kPieceIters - 1) / kPieceIters;
   if (valid == iters * 256u && (iters % kPieceIters) == 0) {
@@ -469,28 +561,48 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
       if (sm_s == 0xFFFFFFFFu) return kStatusWaitTimeout;
       const uint32_t sm_lane = sm_s + lane * 8;
 #pragma unroll
-      for (uint32_t k = 0; k < kPieceIters; ++k) sink.group(kPieceIters * p + k, lane, group(sm_lane + k * 256));
+      for (uint32_t k = 0; k < kPieceIters; k += 2) {
+        uint4 o0, o1;
+        dec.group2(lds_v2(sm_lane + k * 256), lds_v2(sm_lane + (k + 1) * 256), o0, o1);
+        sink.group(kPieceIters * p + k, lane, o0);
+        sink.group(kPieceIters * p + k + 1, lane, o1);
+      }
       feed.end(p);
     }
     return 0;
   }
+  // one group of sub-stream WHICH that may be short or absent (decided per lane)
+  auto ragged = [&](auto which, uint32_t i, uint32_t sm_s) {
+    constexpr int WHICH = decltype(which)::value;
+    const uint32_t pos_e = (i * 32 + lane) * 8;
+    const uint32_t sm_at = sm_s + ((i % kPieceIters) * 32 + lane) * 8;
+    if (pos_e + 8 <= valid) {
+      sink.group(i, lane, dec.template group1<WHICH>(lds_v2(sm_at)));
+    } else if (pos_e < valid) {   // the one short group at the end of a linear tensor
+      const uint32_t cnt = valid - pos_e;
+      for (uint32_t j = 0; j < cnt; ++j) {
+        const uint32_t e = dec.template single<WHICH>();
+        const uint32_t at = sm_at + j;
+        const uint32_t smb = (lds_u32(at & ~3u) >> (8 * (at & 3u))) & 0xFFu;
+        sink.elem(i, lane, j, (uint16_t)(((smb & 0x80u) << 8) | (e & 0x7F80u) | (smb & 0x7Fu)));
+      }
+    }
+  };
   for (uint32_t p = 0; p < pieces; ++p) {
     const uint32_t sm_s = feed.begin(p);
     if (sm_s == 0xFFFFFFFFu) return kStatusWaitTimeout;
     const uint32_t i_end = min(iters, kPieceIters * (p + 1));
 #pragma unroll 1
-    for (uint32_t i = kPieceIters * p; i < i_end; ++i) {
-      const uint32_t pos_e = (i * 32 + lane) * 8;
-      if (pos_e + 8 <= valid) {
-        sink.group(i, lane, group(sm_s + ((i % kPieceIters) * 32 + lane) * 8));
-      } else if (pos_e < valid) {   // the one short group at the end of a linear tensor
-        const uint32_t cnt = valid - pos_e;
-        for (uint32_t j = 0; j < cnt; ++j) {
-          const uint32_t e = single();
-          const uint32_t at = ((i % kPieceIters) * 32 + lane) * 8 + j;
-          const uint32_t smb = (lds_u32(sm_s + (at & ~3u)) >> (8 * (at & 3u))) & 0xFFu;
-          sink.elem(i, lane, j, (uint16_t)(((smb & 0x80u) << 8) | (e & 0x7F80u) | (smb & 0x7Fu)));
-        }
+    for (uint32_t i = kPieceIters * p; i < i_end; i += 2) {
+      if (i + 2 <= i_end && (i + 2) * 256u <= valid) {   // both iterations are complete for every lane
+        uint4 o0, o1;
+        const uint32_t sm_at = sm_s + ((i % kPieceIters) * 32 + lane) * 8;
+        dec.group2(lds_v2(sm_at), lds_v2(sm_at + 256), o0, o1);
+        sink.group(i, lane, o0);
+        sink.group(i + 1, lane, o1);
+      } else {
+        ragged(std::integral_constant<int, 0>{}, i, sm_s);
+        if (i + 1 < i_end) ragged(std::integral_constant<int, 1>{}, i + 1, sm_s);
       }
     }
     feed.end(p);

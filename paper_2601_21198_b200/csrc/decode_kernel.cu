@@ -27,7 +27,7 @@
 namespace zipmoe_dev {
 
 #ifndef ZIPMOE_WARPS
-#define ZIPMOE_WARPS 20
+#define ZIPMOE_WARPS 16
 #endif
 constexpr int kWarps = ZIPMOE_WARPS;                 // warps per CTA, one CTA per SM
 constexpr int kThreads = kWarps * 32;
@@ -146,14 +146,21 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
       report(a.status, kStatusBadDescriptor);
       break;
     }
-    uint32_t g = g0 + warp;
+    // Each warp takes a contiguous share of the segment's tiles: consecutive tiles sit in the same chunk, so the
+    // descriptor and the tile-table entries of the next tile are usually in the first-level cache already.
+    const uint32_t share = (seg_end - g0 + kWarps - 1) / kWarps;
+    uint32_t g = g0 + warp * share;
+    const uint32_t g_end = min(seg_end, g + share);
     uint32_t stage = 0;
     // descriptor and tile-in-chunk of this warp's next tile, stepped without divisions
-    uint32_t tc = run_first_chunk + (g - run_first_tile) / tpc, tt = (g - run_first_tile) % tpc;
+    uint32_t tc = 0, tt = 0;
+    if (g < g_end) {
+      tc = run_first_chunk + (g - run_first_tile) / tpc;
+      tt = (g - run_first_tile) % tpc;
+    }
     auto step = [&]() {
-      tt += kWarps;
-      while (tt >= tpc) {
-        tt -= tpc;
+      if (++tt == tpc) {
+        tt = 0;
         ++tc;
       }
     };
@@ -161,7 +168,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
     // slots are free: it has finished its tiles of the previous segment)
     TileWork cur;
     cur.ok = false;
-    if (g < seg_end && !dead) {
+    if (g < g_end && !dead) {
       cur = resolve_tile(a, tc, tt, WIDE);
       if (!cur.ok) report(a.status, kStatusBadDescriptor);
       else {
@@ -173,12 +180,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
     const bool fast = build_lut(kThreads, a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <=
                       (uint32_t)kLaneLutBits;
 
-    for (; g < seg_end && !dead; g += kWarps) {
+    for (; g < g_end && !dead; ++g) {
       TileWork nxt;
       nxt.ok = false;
       uint32_t nxt_issued = 0;
-      const uint32_t g2 = g + kWarps;
-      if (g2 < seg_end) {
+      if (g + 1 < g_end) {
         step();
         nxt = resolve_tile(a, tc, tt, WIDE);
         if (!nxt.ok) report(a.status, kStatusBadDescriptor);

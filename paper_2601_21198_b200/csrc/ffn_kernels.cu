@@ -375,10 +375,12 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
           for (int k = 0; k < 8; ++k) smB[k] = ldg_v2_early(cur.sm + (8 + k) * 256 + lane * 8);
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
-            // the first four iterations are decoded into registers while the previous half's MMAs may still run
+            // the first four rows (two from each of the lane's sub-streams) are decoded into registers while
+            // the previous half's MMAs may still run
             uint4 v[4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) v[k] = dec.group(half ? smB[k] : smA[k]);
+            for (int k = 0; k < 4; k += 2)
+              dec.group2(half ? smB[k] : smA[k], half ? smB[k + 1] : smA[k + 1], v[k], v[k + 1]);
             if (!buffer_free()) {
               report(a.la.status, kStatusWaitTimeout);
               publish();
@@ -388,7 +390,12 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
 #pragma unroll
             for (int k = 0; k < 4; ++k) sts_v4(buf + lane * kBLbo + k * 16, v[k]);
 #pragma unroll
-            for (int k = 4; k < 8; ++k) sts_v4(buf + lane * kBLbo + k * 16, dec.group(half ? smB[k] : smA[k]));
+            for (int k = 4; k < 8; k += 2) {
+              uint4 o0, o1;
+              dec.group2(half ? smB[k] : smA[k], half ? smB[k + 1] : smA[k + 1], o0, o1);
+              sts_v4(buf + lane * kBLbo + k * 16, o0);
+              sts_v4(buf + lane * kBLbo + (k + 1) * 16, o1);
+            }
             if (half == 0 && have_next) {
 #pragma unroll
               for (int k = 0; k < 8; ++k) smA[k] = ldg_v2_early(nxt.sm + k * 256 + lane * 8);

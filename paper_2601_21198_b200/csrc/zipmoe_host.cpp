@@ -122,6 +122,13 @@ void canonical_codes(const uint8_t *len, uint32_t *code) {
   for (int s = 0; s < 256; ++s) code[s] = len[s] ? next[len[s]]++ : 0;
 }
 
+// the low n bits of v in reverse order
+inline uint32_t reverse_bits(uint32_t v, uint32_t n) {
+  uint32_t r = 0;
+  for (uint32_t b = 0; b < n; ++b) r |= ((v >> b) & 1u) << (n - 1 - b);
+  return r;
+}
+
 // Appends codes to a u32 word stream, most significant bit of each word first.
 struct BitWriter {
   uint8_t *dst;
@@ -307,6 +314,10 @@ zipmoe_status zipmoe_encode(const uint16_t *bf16, uint64_t rows, uint64_t cols, 
       BitWriter bw(rec + kRecordHeadBytes);
       for (uint32_t lane = 0; lane < kLanes; ++lane) {
         const uint64_t before = bw.total;
+        // sub-stream 0 (even iterations) forwards; sub-stream 1 (odd iterations) is read backwards from the
+        // end of the lane's bit range, so it is appended last code first, every code with its bits reversed
+        uint8_t odd[ZIPMOE_TILE_ELEMS_MAX / kIterElems / 2 * kGroup];
+        uint32_t n_odd = 0;
         for (uint32_t i = 0; i < g.iters; ++i) {
           uint32_t pos = (i * kLanes + lane) * kGroup;
           if (pos >= valid) break;
@@ -314,8 +325,13 @@ zipmoe_status zipmoe_encode(const uint16_t *bf16, uint64_t rows, uint64_t cols, 
           const uint16_t *p = bf16 + origin + i * pitch + lane * kGroup;
           for (uint32_t j = 0; j < cnt; ++j) {
             uint32_t s = (p[j] >> 7) & 0xFF;
-            bw.put(code[s], len[s]);
+            if (i & 1) odd[n_odd++] = (uint8_t)s;
+            else bw.put(code[s], len[s]);
           }
+        }
+        while (n_odd) {
+          const uint32_t s = odd[--n_odd];
+          bw.put(reverse_bits(code[s], len[s]), len[s]);
         }
         store_le<uint16_t>(rec + 2 * lane, (uint16_t)(bw.total - before));
       }
