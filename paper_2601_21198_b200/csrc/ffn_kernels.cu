@@ -6,9 +6,15 @@
 // tcgen05 tensor-core MMAs, so decoded weights never reach global memory.
 //
 // One kernel, ffn_matmul_kernel, computes  Y[slot, row] = sum_k W[row, k] * X[slot, k]
-// for the token slots routed to one expert, a group of 16-row strips of one
-// compressed matrix W (blocked layout: tiles of 16 rows x 256 columns) and a
-// range of K:
+// for the token slots routed to the experts that have tokens.  A job is one
+// expert, one compressed matrix W (blocked layout: tiles of 16 rows x 256 columns)
+// and one group of 16-row strips; a job has K / 256 steps.  The kernel is
+// persistent: the steps of all jobs form one sequence that is cut into equal,
+// contiguous shares, one per CTA (one CTA per SM), so that every SM decodes the
+// same number of tiles whatever the number of experts with tokens.  A CTA works
+// through its share piece by piece (a piece = consecutive steps of one job);
+// where a job is cut between CTAs each writes a partial sum, added later by the
+// elementwise kernels.  Within a piece:
 //   * each decode warp owns one strip and walks its tiles along K.  A tile is
 //     decoded in two halves of 8 rows.  Eight warps form a group: their eight
 //     half-tile buffers (8 rows x 256 columns each, K-major, no swizzle) are
@@ -22,9 +28,7 @@
 //     x 256 bf16) in a two-stage ring shared by all groups;
 //   * at the end four warps read the accumulators back (tcgen05.ld) and store Y.
 // The host wrapper runs it for W1 and W3 (gate, up), applies SiLU(g)*u, runs it
-// for W2, and combines the experts of every token; K is split over several
-// CTAs where few experts are active, the partial sums are added by the
-// elementwise kernels.
+// for W2, and combines the experts of every token.
 // Every wait on a barrier is bounded; a wait that runs out is reported through
 // the status word and the kernel still runs to its end and frees tensor memory.
 #include <cuda_bf16.h>
@@ -61,20 +65,42 @@ struct FfnArgs {
   LaunchArgs la;                       // descriptors, tables, payload and SM buffers of all expert tensors
   const uint32_t *tensor_first_chunk;  // [3E] first descriptor of tensor e*3 + {0 w1, 1 w3, 2 w2}
   const uint32_t *expert_offset;       // [E+1] first slot of each expert
-  const uint32_t *active;              // [0] number of experts with tokens, [1..] their ids; blockIdx.y indexes this list
+  const uint32_t *active;              // [0] number of experts with tokens, [1..] their ids
   const uint32_t *slot_token;          // [S] token of each slot, or null when X rows are the slots themselves
   const uint16_t *x;                   // bf16 activations, row pitch K
-  float *y;                            // [gridDim.z][S][rows]
-  uint32_t rows, K;                    // the matrix is [rows, K]
-  uint32_t tensor_base;                // tensor in expert = tensor_base + blockIdx.z / splits
-  uint32_t splits, steps_per_split;    // K split = blockIdx.z % splits, K steps of 256 per split
+  float *y;                            // [n_mats][max_parts][S][rows] partial sums
+  uint32_t rows, K;                    // every matrix of the launch is [rows, K]
+  uint32_t tensor_base, n_mats;        // tensors tensor_base .. tensor_base + n_mats - 1 of every active expert
+  uint32_t n_groups;                   // strip groups (16 * n_warps rows each) per matrix
+  uint32_t min_units, max_parts;       // smallest share of a CTA in steps; bound on the CTAs a job is cut between
   uint32_t n_warps, groups, S;         // decode warps, 8-row groups of token rows per stage, total slots
   uint32_t smem_bytes;                 // dynamic shared memory of the launch
 };
 
+// ---- how the steps of a launch are shared out --------------------------------------------------
+// U units (steps of all jobs, job-major) go to P CTAs; CTA c takes [c*U/P, (c+1)*U/P).  P is chosen so that
+// every CTA gets at least min_units units, hence a job of `steps` units is cut between at most
+// ceil(steps / min_units) + 1 CTAs.
+__host__ __device__ inline uint32_t ffn_ctas_in_use(uint64_t U, uint32_t grid, uint32_t min_units) {
+  uint64_t p = U / (min_units ? min_units : 1);
+  if (p < 1) p = 1;
+  return p < grid ? (uint32_t)p : grid;
+}
+__host__ __device__ inline uint64_t ffn_first_unit(uint32_t c, uint64_t U, uint32_t P) { return (uint64_t)c * U / P; }
+__host__ __device__ inline uint32_t ffn_cta_of_unit(uint64_t u, uint64_t U, uint32_t P) {
+  return (uint32_t)(((u + 1) * P - 1) / U);
+}
+// the CTAs that share job `job`: the first one, and how many
+__host__ __device__ inline void ffn_job_parts(uint64_t job, uint32_t steps, uint64_t U, uint32_t P, uint32_t *first_cta,
+                                              uint32_t *parts) {
+  const uint32_t c0 = ffn_cta_of_unit(job * steps, U, P), c1 = ffn_cta_of_unit(job * steps + steps - 1, U, P);
+  *first_cta = c0;
+  *parts = c1 - c0 + 1;
+}
+
 // shared-memory layout: [X stages][per-warp buffers][tables][table scratch][barriers][tmem slot]
 __host__ __device__ inline uint32_t ffn_bar_count(uint32_t n_warps) {
-  return 2 * n_warps + 2 * (n_warps / kGroupWarps) + 4;
+  return 2 * n_warps + 2 * (n_warps / kGroupWarps) + 4;   // the word after them is the CTA's give-up flag
 }
 __host__ __device__ inline uint32_t ffn_smem_bytes(uint32_t n_warps, uint32_t groups, bool lane16) {
   const uint32_t after_warps = (lane16 ? kFfnLutBytes : (uint32_t)kLutBytes) + kLutScratchBytes + ffn_bar_count(n_warps) * 8 + 16;
@@ -123,15 +149,16 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   extern __shared__ __align__(128) uint8_t smem[];
   const uint32_t NW = a.n_warps, G = a.groups, Q = NW / kGroupWarps, NCOL = 8 * G;
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (blockIdx.y >= __ldg(a.active)) return;   // fewer experts have tokens than the grid allows for
-  const uint32_t e = __ldg(a.active + 1 + blockIdx.y), z = blockIdx.z;
-  const uint32_t off = __ldg(a.expert_offset + e);
-  uint32_t Te = __ldg(a.expert_offset + e + 1) - off;
-  if (Te == 0) return;   // nothing routed to this expert
-  if (Te > NCOL) {       // more slots than the stage holds (a token listing the same expert twice)
-    report(a.la.status, kStatusBadDescriptor);
-    Te = NCOL;
-  }
+
+  // ---- this CTA's share of the launch's steps ----
+  const uint32_t n_active = __ldg(a.active);   // experts that have tokens
+  const uint32_t steps = a.K >> 8;
+  const uint32_t U = n_active * a.n_mats * a.n_groups * steps;   // (the host made sure that this fits 32 bits)
+  if (U == 0) return;
+  const uint32_t P = ffn_ctas_in_use(U, gridDim.x, a.min_units);
+  if (blockIdx.x >= P) return;
+  uint32_t u = (uint32_t)ffn_first_unit(blockIdx.x, U, P);
+  const uint32_t u_end = (uint32_t)ffn_first_unit(blockIdx.x + 1, U, P);
 
   uint8_t *x_raw = smem;                                   // [2][G][4096]
   uint8_t *warp_raw = x_raw + 2 * G * kXGroupBytes;        // [NW][2 record stages | half-tile buffer]
@@ -139,19 +166,13 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   uint8_t *lut_scratch = lut_raw + kMyLutBytes;
   uint64_t *bars = reinterpret_cast<uint64_t *>(lut_scratch + kLutScratchBytes);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + ffn_bar_count(NW));
+  volatile uint32_t *give_up = tmem_slot + 1;              // set once a wait ran out: the CTA stops after the piece
   // barriers: [NW][2] record stages, [Q] group's half written, [Q] group's MMAs done, [2] X full, [2] X empty
   const uint32_t bar0 = smem_addr(bars);
   const uint32_t quad_full = bar0 + 8 * (2 * NW), quad_done = quad_full + 8 * Q;
   const uint32_t x_full = quad_done + 8 * Q, x_empty = x_full + 16;
   const uint32_t x_addr = smem_addr(x_raw), lut = smem_addr(lut_raw);
   const bool is_decode = warp < NW, is_mma = warp >= NW && warp < NW + Q, is_loader = warp == NW + Q;
-
-  const uint32_t n_strips = a.rows >> 4, strip = blockIdx.x * NW + warp;
-  const bool has_strip = is_decode && strip < n_strips;
-  const uint32_t tensor = e * 3 + a.tensor_base + z / a.splits, split = z % a.splits;
-  const uint32_t steps_total = a.K >> 8;
-  const uint32_t s0 = min(split * a.steps_per_split, steps_total), s1 = min(s0 + a.steps_per_split, steps_total);
-  const uint32_t n_steps = s1 - s0;
 
   uint32_t tmem_cols = 32;
   while (tmem_cols < 2 * Q * NCOL) tmem_cols <<= 1;
@@ -165,6 +186,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
     mbar_init(x_full + 8, 1);
     mbar_init(x_empty, Q);
     mbar_init(x_empty + 8, Q);
+    *give_up = 0;
   }
   fence_barrier_init();
   if (warp == 0) {
@@ -178,285 +200,343 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  // the tensor: blocked layout, 16 x 256 tiles, one Huffman table
-  const uint32_t c0 = __ldg(a.tensor_first_chunk + tensor);
-  bool ok = c0 < a.la.n_chunks && 2 * Q * NCOL <= 512 && kGroupWarps * Q == NW;
-  uint32_t table_id = 0, tpc = 1;
-  if (ok) {
-    const zipmoe_chunk_desc *d = a.la.chunks + c0;
-    table_id = __ldg(&d->table_id);
-    tpc = __ldg(&d->tiles_per_chunk);
-    ok = table_id < a.la.n_tables && tpc != 0 && __ldg(&d->row_pitch) == a.K &&
-         __ldg(&d->tiles_per_rowblk) == steps_total && __ldg(&d->tile_elems) == ZIPMOE_TILE_ELEMS_MAX &&
-         __ldg(&d->tile0) == 0;
-  }
-  if (!ok) report(a.la.status, kStatusBadDescriptor);
-  // ---- decode warps: where the strip's tiles are, and the first fetches, while the table is being built ----
-  bool failed = !has_strip || n_steps == 0 || !ok;
+  const bool shape_ok = 2 * Q * NCOL <= 512 && kGroupWarps * Q == NW && steps > 0 && steps <= 64 && a.n_mats > 0 &&
+                        a.n_groups > 0;
+  if (!shape_ok) report(a.la.status, kStatusBadDescriptor);
+
+  // The barriers are initialised once; every role counts what it has put through them since the kernel began,
+  // so that the parity to wait for carries over from one piece to the next.
   const uint32_t my = smem_addr(warp_raw + (is_decode ? warp : 0) * kFfnWarpBytes);
   const uint32_t rec_bar = bar0 + 8 * (2 * (is_decode ? warp : 0));
-
-  // Where the strip's tiles are: lane i (and i + 32) looks up record start and length of the i-th tile of
-  // the K range once, so that the loop below touches global memory only for the data itself.
-  uint32_t rec_at[2] = {0, 0}, rec_len[2] = {0, 0};   // in 16-byte units from the start of the payload buffer
-  const uint8_t *sm_strip = a.la.sm;                  // sign+mantissa bytes of the strip's first tile
-  if (!failed) {
-    const uint32_t tq0 = strip * steps_total + s0;
-    bool bad = n_steps > 64;
-    for (uint32_t r = 0; r < 2; ++r) {
-      const uint32_t i = lane + 32 * r;
-      if (i >= n_steps || bad) continue;
-      const uint32_t tq = tq0 + i, c = c0 + tq / tpc, t = tq % tpc;
-      if (c >= a.la.n_chunks) {
-        bad = true;
-        continue;
-      }
-      const zipmoe_chunk_desc *d = a.la.chunks + c;
-      const uint64_t pay_off = __ldg(&d->payload_off);
-      if (t >= __ldg(&d->n_tiles) || __ldg(&d->tile_elems) != ZIPMOE_TILE_ELEMS_MAX || (pay_off & 15) ||
-          __ldg(&d->table_id) != table_id || pay_off + 4ull * (t + 2) > a.la.payload_bytes ||
-          (t + 1 == __ldg(&d->n_tiles) && __ldg(&d->last_tile_elems) != ZIPMOE_TILE_ELEMS_MAX)) {
-        bad = true;
-        continue;
-      }
-      const uint32_t *tab = reinterpret_cast<const uint32_t *>(a.la.payload + pay_off);
-      const uint32_t o0 = __ldg(tab + t), o1 = __ldg(tab + t + 1);
-      if (o1 <= o0 || o1 - o0 < 4 || o1 - o0 > (64 + ZIPMOE_TILE_ELEMS_MAX / 8 * ZIPMOE_MAX_CODE_LEN) / 16 + 1 ||
-          pay_off + 16ull * o1 > a.la.payload_bytes) {
-        bad = true;
-        continue;
-      }
-      rec_at[r] = (uint32_t)(pay_off >> 4) + o0;
-      rec_len[r] = o1 - o0;
-    }
-    const uint64_t sm_first = __ldg(&a.la.chunks[c0].sm_off) + (uint64_t)tq0 * ZIPMOE_TILE_ELEMS_MAX;
-    if ((sm_first & 15) || sm_first + (uint64_t)n_steps * ZIPMOE_TILE_ELEMS_MAX > a.la.sm_bytes) bad = true;
-    sm_strip = a.la.sm + sm_first;
-    if (__any_sync(0xFFFFFFFFu, bad)) {
-      report(a.la.status, kStatusBadDescriptor);
-      failed = true;
-    }
-  }
-  struct Tile {
-    const uint8_t *rec, *sm;
-    uint32_t rec_bytes;
-    bool staged;
-  };
-  auto tile = [&](uint32_t i) -> Tile {   // the i-th tile of the K range (all lanes call this)
-    const uint32_t at = __shfl_sync(0xFFFFFFFFu, i < 32 ? rec_at[0] : rec_at[1], i & 31);
-    const uint32_t len = __shfl_sync(0xFFFFFFFFu, i < 32 ? rec_len[0] : rec_len[1], i & 31);
-    Tile t;
-    t.rec = a.la.payload + (size_t)at * 16;
-    t.rec_bytes = len * 16;
-    t.sm = sm_strip + (size_t)i * ZIPMOE_TILE_ELEMS_MAX;
-    t.staged = t.rec_bytes <= (uint32_t)kPayBuf;
-    return t;
-  };
-  Tile cur = {a.la.payload, a.la.sm, 0, false};
-  uint2 smA[8], smB[8];
-  if (!failed) {
-    cur = tile(0);
-    if (cur.staged && lane == 0) bulk_load(my, cur.rec, cur.rec_bytes, rec_bar);
-#pragma unroll
-    for (int k = 0; k < 8; ++k) smA[k] = ldg_v2_early(cur.sm + k * 256 + lane * 8);
-  }
-
+  uint32_t rec_phase = 0, stage = 0;   // decode warp: parity of its two record stages, the stage of its next tile
+  uint32_t hn = 0;                     // decode and MMA warps: halves the group has handed over so far
+  uint32_t xs = 0;                     // loader and MMA warps: K steps staged / consumed so far
+  uint32_t lut_tensor = 0xFFFFFFFFu;   // the tensor whose table is in shared memory
   bool fast = true;
-  if (ok) fast = build_lut(blockDim.x, a.la.tables[table_id].code_len, lut_raw, lut_scratch, a.la.status, LANE16) <=
-                 (uint32_t)kLaneLutBits;
-  // (build_lut ends with a CTA barrier)
 
-  if (ok && is_loader) {
-    // ---- activations: one K step (8G token rows x 256 columns) per stage ----
-    for (uint32_t s = 0; s < n_steps; ++s) {
-      const uint32_t b = s & 1, n = s >> 1;
-      if (n > 0 && !mbar_wait_bounded(x_empty + 8 * b, (n - 1) & 1)) {
-        report(a.la.status, kStatusWaitTimeout);
-        break;
-      }
-      const uint32_t stage = x_addr + b * G * kXGroupBytes;
-      for (uint32_t row = lane; row < NCOL; row += 32) {
-        const uint16_t *src = a.x;
-        uint32_t src_bytes = 0;   // rows past the expert's last slot are filled with zeros
-        if (row < Te) {
-          const uint32_t xr = a.slot_token ? __ldg(a.slot_token + off + row) : off + row;
-          src = a.x + (size_t)xr * a.K + (size_t)(s0 + s) * 256;
-          src_bytes = 16;
-        }
-        const uint32_t dst = stage + (row >> 3) * kXGroupBytes + (row & 7) * 16;
-#pragma unroll 8
-        for (uint32_t k8 = 0; k8 < 32; ++k8)
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + k8 * 128),
-                       "l"(src + (src_bytes ? k8 * 8 : 0)), "r"(src_bytes)
-                       : "memory");
-      }
-      asm volatile("cp.async.wait_all;" ::: "memory");
-      fence_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(x_full + 8 * b);
+  while (shape_ok && u < u_end) {
+    // ---- the piece: steps [s0, s0 + n_steps) of one job ----
+    const uint32_t job = u / steps;
+    const uint32_t s0 = u - job * steps;
+    const uint32_t n_steps = min(steps - s0, u_end - u);
+    const uint32_t grp = job % a.n_groups;
+    const uint32_t jm = job / a.n_groups, mat = jm % a.n_mats, a_idx = jm / a.n_mats;
+    const uint32_t part = blockIdx.x - ffn_cta_of_unit((uint64_t)job * steps, U, P);   // which of the job's partial sums
+    u += n_steps;
+    const uint32_t e = __ldg(a.active + 1 + a_idx);
+    const uint32_t off = __ldg(a.expert_offset + e);
+    uint32_t Te = __ldg(a.expert_offset + e + 1) - off;
+    if (Te > NCOL) {       // more slots than the stage holds (a token listing the same expert twice)
+      report(a.la.status, kStatusBadDescriptor);
+      Te = NCOL;
     }
-  } else if (ok && is_mma) {
-    // ---- one MMA warp per group; one lane issues, per half-tile: D[64 x N] (+)= A[64 x 256] * X[N x 256]^T ----
-    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (G << 17) | ((uint32_t)(kGroupWarps / 2) << 24);   // bf16 x bf16 -> fp32, N = 8G, M = 8 * kGroupWarps
-    const uint32_t q = warp - NW;
-    const uint32_t abuf = smem_addr(warp_raw) + 2 * kPayStage + kGroupWarps * q * kFfnWarpBytes;
-    const uint64_t a_desc0 = smem_desc(abuf, kBLbo, kFfnWarpBytes);
-    bool alive = true;
-    for (uint32_t s = 0; s < n_steps && alive; ++s) {
-      const uint32_t xb = s & 1;
-      const uint64_t b_desc0 = smem_desc(x_addr + xb * G * kXGroupBytes, 128, kXGroupBytes);
-      if (!mbar_wait_bounded(x_full + 8 * xb, (s >> 1) & 1)) alive = false;
-      for (uint32_t half = 0; half < 2 && alive; ++half) {
-        const uint32_t hn = 2 * s + half;
-        if (!mbar_wait_bounded(quad_full + 8 * q, hn & 1)) {
-          alive = false;
+    const uint32_t n_strips = a.rows >> 4, strip = grp * NW + warp;
+    const bool has_strip = is_decode && strip < n_strips;
+    const uint32_t tensor = e * 3 + a.tensor_base + mat;
+
+    // the tensor: blocked layout, 16 x 256 tiles, one Huffman table
+    const uint32_t c0 = __ldg(a.tensor_first_chunk + tensor);
+    bool ok = c0 < a.la.n_chunks && part < a.max_parts && Te > 0;
+    uint32_t table_id = 0, tpc = 1;
+    if (ok) {
+      const zipmoe_chunk_desc *d = a.la.chunks + c0;
+      table_id = __ldg(&d->table_id);
+      tpc = __ldg(&d->tiles_per_chunk);
+      ok = table_id < a.la.n_tables && tpc != 0 && __ldg(&d->row_pitch) == a.K &&
+           __ldg(&d->tiles_per_rowblk) == steps && __ldg(&d->tile_elems) == ZIPMOE_TILE_ELEMS_MAX &&
+           __ldg(&d->tile0) == 0;
+    }
+    if (!ok) {   // the same for every thread of the CTA: the piece is skipped
+      report(a.la.status, kStatusBadDescriptor);
+      continue;
+    }
+    // ---- decode warps: where the strip's tiles are, and the first fetches, while the table is being built ----
+    bool failed = !has_strip;
+
+    // Where the strip's tiles are: lane i (and i + 32) looks up record start and length of the i-th tile of
+    // the piece once, so that the loop below touches global memory only for the data itself.
+    uint32_t rec_at[2] = {0, 0}, rec_len[2] = {0, 0};   // in 16-byte units from the start of the payload buffer
+    const uint8_t *sm_strip = a.la.sm;                  // sign+mantissa bytes of the strip's first tile
+    if (!failed) {
+      const uint32_t tq0 = strip * steps + s0;
+      bool bad = false;
+      for (uint32_t r = 0; r < 2; ++r) {
+        const uint32_t i = lane + 32 * r;
+        if (i >= n_steps || bad) continue;
+        const uint32_t tq = tq0 + i, c = c0 + tq / tpc, t = tq % tpc;
+        if (c >= a.la.n_chunks) {
+          bad = true;
+          continue;
+        }
+        const zipmoe_chunk_desc *d = a.la.chunks + c;
+        const uint64_t pay_off = __ldg(&d->payload_off);
+        if (t >= __ldg(&d->n_tiles) || __ldg(&d->tile_elems) != ZIPMOE_TILE_ELEMS_MAX || (pay_off & 15) ||
+            __ldg(&d->table_id) != table_id || pay_off + 4ull * (t + 2) > a.la.payload_bytes ||
+            (t + 1 == __ldg(&d->n_tiles) && __ldg(&d->last_tile_elems) != ZIPMOE_TILE_ELEMS_MAX)) {
+          bad = true;
+          continue;
+        }
+        const uint32_t *tab = reinterpret_cast<const uint32_t *>(a.la.payload + pay_off);
+        const uint32_t o0 = __ldg(tab + t), o1 = __ldg(tab + t + 1);
+        if (o1 <= o0 || o1 - o0 < 4 || o1 - o0 > (64 + ZIPMOE_TILE_ELEMS_MAX / 8 * ZIPMOE_MAX_CODE_LEN) / 16 + 1 ||
+            pay_off + 16ull * o1 > a.la.payload_bytes) {
+          bad = true;
+          continue;
+        }
+        rec_at[r] = (uint32_t)(pay_off >> 4) + o0;
+        rec_len[r] = o1 - o0;
+      }
+      const uint64_t sm_first = __ldg(&a.la.chunks[c0].sm_off) + (uint64_t)tq0 * ZIPMOE_TILE_ELEMS_MAX;
+      if ((sm_first & 15) || sm_first + (uint64_t)n_steps * ZIPMOE_TILE_ELEMS_MAX > a.la.sm_bytes) bad = true;
+      sm_strip = a.la.sm + sm_first;
+      if (__any_sync(0xFFFFFFFFu, bad)) {
+        report(a.la.status, kStatusBadDescriptor);
+        failed = true;
+      }
+    }
+    struct Tile {
+      const uint8_t *rec, *sm;
+      uint32_t rec_bytes;
+      bool staged;
+    };
+    auto tile = [&](uint32_t i) -> Tile {   // the i-th tile of the piece (all lanes call this)
+      const uint32_t at = __shfl_sync(0xFFFFFFFFu, i < 32 ? rec_at[0] : rec_at[1], i & 31);
+      const uint32_t len = __shfl_sync(0xFFFFFFFFu, i < 32 ? rec_len[0] : rec_len[1], i & 31);
+      Tile t;
+      t.rec = a.la.payload + (size_t)at * 16;
+      t.rec_bytes = len * 16;
+      t.sm = sm_strip + (size_t)i * ZIPMOE_TILE_ELEMS_MAX;
+      t.staged = t.rec_bytes <= (uint32_t)kPayBuf;
+      return t;
+    };
+    Tile cur = {a.la.payload, a.la.sm, 0, false};
+    uint2 sm[8];   // sign+mantissa bytes of the lane's groups in the 8 rows of a half-tile
+    if (!failed) {
+      cur = tile(0);
+      if (cur.staged && lane == 0) bulk_load(my + stage * kPayStage, cur.rec, cur.rec_bytes, rec_bar + 8 * stage);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) sm[k] = ldg_v2_early(cur.sm + k * 256 + lane * 8);
+    }
+
+    if (tensor != lut_tensor) {   // (every warp is done with the previous table: a piece ends with CTA barriers)
+      fast = build_lut(blockDim.x, a.la.tables[table_id].code_len, lut_raw, lut_scratch, a.la.status, LANE16) <=
+             (uint32_t)kLaneLutBits;
+      lut_tensor = tensor;
+    }
+
+    if (is_loader) {
+      // ---- activations: one K step (8G token rows x 256 columns) per stage ----
+      for (uint32_t s = 0; s < n_steps; ++s, ++xs) {
+        const uint32_t b = xs & 1, n = xs >> 1;
+        if (n > 0 && !mbar_wait_bounded(x_empty + 8 * b, (n - 1) & 1)) {
+          report(a.la.status, kStatusWaitTimeout);
+          *give_up = 1;
           break;
         }
-        if (lane == 0) {
-          tc_fence_after();
-          const uint32_t d_tmem = tmem + (2 * q + half) * NCOL;
-          // the K slice j of an operand starts 2 cores further: the start-address field counts 16-byte units
-#pragma unroll
-          for (uint32_t j = 0; j < 16; ++j)
-            mma_bf16(d_tmem, a_desc0 + j * (2 * kBLbo / 16), b_desc0 + j * (256 / 16), idesc, (s > 0 || j > 0) ? 1u : 0u);
-          mma_commit(quad_done + 8 * q);
-          if (half == 1) mma_commit(x_empty + 8 * xb);   // this group is done with the X stage
-        }
-        __syncwarp();
-      }
-    }
-    if (!alive) report(a.la.status, kStatusWaitTimeout);
-  } else if (ok && is_decode) {
-    // ---- one strip of 16 rows: decode tile after tile along K, hand half-tiles to the group's A operand ----
-    const uint32_t buf = my + 2 * kPayStage;
-    const uint32_t q = warp / kGroupWarps;
-    uint32_t rec_phase = 0, hn = 0;
-    // hand-over of one half in two moves: before the first store, wait until the MMAs of the previous half have
-    // read the buffer; after the last store, make the stores visible to the tensor core and tell the MMA warp
-    auto buffer_free = [&]() -> bool {
-      if (hn == 0) return true;
-      return mbar_wait_bounded(quad_done + 8 * q, (hn - 1) & 1, failed ? kFfnShortTries : (1u << 20));
-    };
-    auto publish = [&]() {
-      fence_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(quad_full + 8 * q);
-      ++hn;
-    };
-    uint32_t stage = 0;
-    for (uint32_t s = 0; s < n_steps; ++s) {
-      Tile nxt = cur;
-      const bool have_next = !failed && s + 1 < n_steps;
-      if (have_next) {
-        nxt = tile(s + 1);
-        if (nxt.staged && lane == 0)
-          bulk_load(my + (stage ^ 1) * kPayStage, nxt.rec, nxt.rec_bytes, rec_bar + 8 * (stage ^ 1));
-      }
-      bool step_done = false;
-      if (!failed) {
-        bool good = true;
-        if (cur.staged) {
-          good = mbar_wait_bounded(rec_bar + 8 * stage, (rec_phase >> stage) & 1);
-          rec_phase ^= 1u << stage;
-          if (!good) report(a.la.status, kStatusWaitTimeout);
-        }
-        // both halves of the tile, for every combination of record location and table kind
-        auto run = [&](auto staged_c, auto fast_c) -> bool {
-          LaneDecoder<decltype(staged_c)::value, !decltype(fast_c)::value ? kLutWide : LANE16 ? kLutLane16 : kLutLane32> dec;
-          if (!dec.init(my + stage * kPayStage, cur.rec, cur.rec_bytes, lut, lane)) {
-            report(a.la.status, kStatusBadBitCount);
-            buffer_free();
-            publish();   // keep the count of halves
-            buffer_free();
-            publish();
-            return false;
+        const uint32_t xstage = x_addr + b * G * kXGroupBytes;
+        for (uint32_t row = lane; row < NCOL; row += 32) {
+          const uint16_t *src = a.x;
+          uint32_t src_bytes = 0;   // rows past the expert's last slot are filled with zeros
+          if (row < Te) {
+            const uint32_t xr = a.slot_token ? __ldg(a.slot_token + off + row) : off + row;
+            src = a.x + (size_t)xr * a.K + (size_t)(s0 + s) * 256;
+            src_bytes = 16;
           }
+          const uint32_t dst = xstage + (row >> 3) * kXGroupBytes + (row & 7) * 16;
+#pragma unroll 8
+          for (uint32_t k8 = 0; k8 < 32; ++k8)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + k8 * 128),
+                         "l"(src + (src_bytes ? k8 * 8 : 0)), "r"(src_bytes)
+                         : "memory");
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(x_full + 8 * b);
+      }
+    } else if (is_mma) {
+      // ---- one MMA warp per group; one lane issues, per half-tile: D[64 x N] (+)= A[64 x 256] * X[N x 256]^T ----
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (G << 17) | ((uint32_t)(kGroupWarps / 2) << 24);   // bf16 x bf16 -> fp32, N = 8G, M = 8 * kGroupWarps
+      const uint32_t q = warp - NW;
+      const uint32_t abuf = smem_addr(warp_raw) + 2 * kPayStage + kGroupWarps * q * kFfnWarpBytes;
+      const uint64_t a_desc0 = smem_desc(abuf, kBLbo, kFfnWarpBytes);
+      bool alive = true;
+      for (uint32_t s = 0; s < n_steps && alive; ++s, ++xs) {
+        const uint32_t xb = xs & 1;
+        const uint64_t b_desc0 = smem_desc(x_addr + xb * G * kXGroupBytes, 128, kXGroupBytes);
+        if (!mbar_wait_bounded(x_full + 8 * xb, (xs >> 1) & 1)) alive = false;
+        for (uint32_t half = 0; half < 2 && alive; ++half, ++hn) {
+          if (!mbar_wait_bounded(quad_full + 8 * q, hn & 1)) {
+            alive = false;
+            break;
+          }
+          if (lane == 0) {
+            tc_fence_after();
+            const uint32_t d_tmem = tmem + (2 * q + half) * NCOL;
+            // the K slice j of an operand starts 2 cores further: the start-address field counts 16-byte units
 #pragma unroll
-          for (int k = 0; k < 8; ++k) smB[k] = ldg_v2_early(cur.sm + (8 + k) * 256 + lane * 8);
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            // the first four rows (two from each of the lane's sub-streams) are decoded into registers while
-            // the previous half's MMAs may still run
-            uint4 v[4];
-#pragma unroll
-            for (int k = 0; k < 4; k += 2)
-              dec.group2(half ? smB[k] : smA[k], half ? smB[k + 1] : smA[k + 1], v[k], v[k + 1]);
-            if (!buffer_free()) {
+            for (uint32_t j = 0; j < 16; ++j)
+              mma_bf16(d_tmem, a_desc0 + j * (2 * kBLbo / 16), b_desc0 + j * (256 / 16), idesc, (s > 0 || j > 0) ? 1u : 0u);
+            mma_commit(quad_done + 8 * q);
+            if (half == 1) mma_commit(x_empty + 8 * xb);   // this group is done with the X stage
+          }
+          __syncwarp();
+        }
+      }
+      if (!alive) {
+        report(a.la.status, kStatusWaitTimeout);
+        *give_up = 1;
+      }
+    } else if (is_decode) {
+      // ---- one strip of 16 rows: decode tile after tile along K, hand half-tiles to the group's A operand ----
+      const uint32_t buf = my + 2 * kPayStage;
+      const uint32_t q = warp / kGroupWarps;
+      // hand-over of one half in two moves: before the first store, wait until the MMAs of the previous half have
+      // read the buffer; after the last store, make the stores visible to the tensor core and tell the MMA warp
+      auto buffer_free = [&]() -> bool {
+        if (hn == 0) return true;
+        return mbar_wait_bounded(quad_done + 8 * q, (hn - 1) & 1, (failed || *give_up) ? kFfnShortTries : (1u << 20));
+      };
+      auto publish = [&]() {
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(quad_full + 8 * q);
+        ++hn;
+      };
+      for (uint32_t s = 0; s < n_steps; ++s) {
+        Tile nxt = cur;
+        const bool have_next = !failed && s + 1 < n_steps;
+        if (have_next) {
+          nxt = tile(s + 1);
+          if (nxt.staged && lane == 0)
+            bulk_load(my + (stage ^ 1) * kPayStage, nxt.rec, nxt.rec_bytes, rec_bar + 8 * (stage ^ 1));
+        }
+        bool step_done = false;
+        if (!failed) {
+          bool good = true;
+          if (cur.staged) {
+            good = mbar_wait_bounded(rec_bar + 8 * stage, (rec_phase >> stage) & 1);
+            rec_phase ^= 1u << stage;
+            if (!good) {
               report(a.la.status, kStatusWaitTimeout);
+              *give_up = 1;
+            }
+          }
+          // both halves of the tile, for every combination of record location and table kind
+          auto run = [&](auto staged_c, auto fast_c) -> bool {
+            LaneDecoder<decltype(staged_c)::value, !decltype(fast_c)::value ? kLutWide : LANE16 ? kLutLane16 : kLutLane32> dec;
+            if (!dec.init(my + stage * kPayStage, cur.rec, cur.rec_bytes, lut, lane)) {
+              report(a.la.status, kStatusBadBitCount);
+              buffer_free();
+              publish();   // keep the count of halves
+              buffer_free();
               publish();
-              if (half == 0) publish();   // keep the count of halves
               return false;
             }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) sts_v4(buf + lane * kBLbo + k * 16, v[k]);
+            for (int half = 0; half < 2; ++half) {
+              // Sign+mantissa bytes: sm[k] holds row k of the half being decoded; as soon as a row has been
+              // used its register is refilled with the same row of the half after this one (the tile's second
+              // half, or the first half of the strip's next tile), a whole half ahead of its use.
+              const uint8_t *ahead = half == 0 ? cur.sm + 8 * 256 + lane * 8 : nxt.sm + lane * 8;
+              const bool more = half == 0 || have_next;
+              // the first four rows (two from each of the lane's sub-streams) are decoded into registers while
+              // the previous half's MMAs may still run
+              uint4 v[4];
 #pragma unroll
-            for (int k = 4; k < 8; k += 2) {
-              uint4 o0, o1;
-              dec.group2(half ? smB[k] : smA[k], half ? smB[k + 1] : smA[k + 1], o0, o1);
-              sts_v4(buf + lane * kBLbo + k * 16, o0);
-              sts_v4(buf + lane * kBLbo + (k + 1) * 16, o1);
-            }
-            if (half == 0 && have_next) {
+              for (int k = 0; k < 4; k += 2) {
+                dec.group2(sm[k], sm[k + 1], v[k], v[k + 1]);
+                if (more) {
+                  sm[k] = ldg_v2_early(ahead + k * 256);
+                  sm[k + 1] = ldg_v2_early(ahead + (k + 1) * 256);
+                }
+              }
+              if (!buffer_free()) {
+                report(a.la.status, kStatusWaitTimeout);
+                *give_up = 1;
+                publish();
+                if (half == 0) publish();   // keep the count of halves
+                return false;
+              }
 #pragma unroll
-              for (int k = 0; k < 8; ++k) smA[k] = ldg_v2_early(nxt.sm + k * 256 + lane * 8);
+              for (int k = 0; k < 4; ++k) sts_v4(buf + lane * kBLbo + k * 16, v[k]);
+#pragma unroll
+              for (int k = 4; k < 8; k += 2) {
+                uint4 o0, o1;
+                dec.group2(sm[k], sm[k + 1], o0, o1);
+                if (more) {
+                  sm[k] = ldg_v2_early(ahead + k * 256);
+                  sm[k + 1] = ldg_v2_early(ahead + (k + 1) * 256);
+                }
+                sts_v4(buf + lane * kBLbo + k * 16, o0);
+                sts_v4(buf + lane * kBLbo + (k + 1) * 16, o1);
+              }
+              publish();
             }
-            publish();
+            return true;
+          };
+          if (good) {
+            if (cur.staged) good = fast ? run(std::true_type{}, std::true_type{}) : run(std::true_type{}, std::false_type{});
+            else good = fast ? run(std::false_type{}, std::true_type{}) : run(std::false_type{}, std::false_type{});
+            step_done = true;   // run() publishes both halves even when it fails
           }
-          return true;
-        };
-        if (good) {
-          if (cur.staged) good = fast ? run(std::true_type{}, std::true_type{}) : run(std::true_type{}, std::false_type{});
-          else good = fast ? run(std::false_type{}, std::true_type{}) : run(std::false_type{}, std::false_type{});
-          step_done = true;   // run() publishes both halves even when it fails
+          if (!good) failed = true;
         }
-        if (!good) failed = true;
+        if (!step_done) {   // nothing to contribute: keep the group's hand-over going with whatever the buffer holds
+          buffer_free();
+          publish();
+          buffer_free();
+          publish();
+        }
+        cur = nxt;
+        stage ^= 1;
       }
-      if (!step_done) {   // nothing to contribute: keep the group's hand-over going with whatever the buffer holds
-        buffer_free();
-        publish();
-        buffer_free();
-        publish();
+      // the accumulators are final once the MMAs of the last half are done
+      if (hn > 0 && !mbar_wait_bounded(quad_done + 8 * q, (hn - 1) & 1, (failed || *give_up) ? kFfnShortTries : (1u << 20))) {
+        report(a.la.status, kStatusWaitTimeout);
+        *give_up = 1;
       }
-      cur = nxt;
-      stage ^= 1;
     }
-    // the accumulators are final once the MMAs of the last half are done
-    if (hn > 0 && !mbar_wait_bounded(quad_done + 8 * q, (hn - 1) & 1, failed ? kFfnShortTries : (1u << 20)))
-      report(a.la.status, kStatusWaitTimeout);
-  }
 
-  // ---- accumulators -> Y ----
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  if (ok && warp < 4 && n_steps) {
-    // With M = 64, D row 16j + i sits in tensor-memory lane 32j + i (i < 16): warp j reads rows 16j..16j+15,
-    // the halves of the group's warps 2j and 2j + 1.
-    // With M = 128, D row r sits in lane r: warp j reads rows 32j..32j+31, the halves of warps 4j..4j+3.
-    const uint32_t wg = kGroupWarps == 8 ? 2 * warp + ((lane >> 3) & 1) : 4 * warp + (lane >> 3), r = lane & 7;
-    const uint32_t live_lanes = kGroupWarps == 8 ? 16 : 32;
-    for (uint32_t q = 0; q < Q; ++q) {
-      const uint32_t st = blockIdx.x * NW + kGroupWarps * q + wg;
-      for (uint32_t half = 0; half < 2; ++half) {
-        const uint32_t row = 16 * st + 8 * half + r;
-        for (uint32_t c = 0; c < G; ++c) {
-          uint32_t v[8];
-          const uint32_t taddr = tmem + ((32 * warp) << 16) + (2 * q + half) * NCOL + 8 * c;
-          asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-                       : "r"(taddr)
-                       : "memory");
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-          if (lane < live_lanes && st < n_strips) {
+    // ---- accumulators -> Y ----
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp < 4 && !*give_up) {
+      // With M = 64, D row 16j + i sits in tensor-memory lane 32j + i (i < 16): warp j reads rows 16j..16j+15,
+      // the halves of the group's warps 2j and 2j + 1.
+      // With M = 128, D row r sits in lane r: warp j reads rows 32j..32j+31, the halves of warps 4j..4j+3.
+      const uint32_t wg = kGroupWarps == 8 ? 2 * warp + ((lane >> 3) & 1) : 4 * warp + (lane >> 3), r = lane & 7;
+      const uint32_t live_lanes = kGroupWarps == 8 ? 16 : 32;
+      float *y = a.y + ((size_t)(mat * a.max_parts + part) * a.S + off) * a.rows;
+      for (uint32_t q = 0; q < Q; ++q) {
+        const uint32_t st = grp * NW + kGroupWarps * q + wg;
+        for (uint32_t half = 0; half < 2; ++half) {
+          const uint32_t row = 16 * st + 8 * half + r;
+          for (uint32_t c = 0; c < G; ++c) {
+            uint32_t v[8];
+            const uint32_t taddr = tmem + ((32 * warp) << 16) + (2 * q + half) * NCOL + 8 * c;
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                         : "r"(taddr)
+                         : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (lane < live_lanes && st < n_strips) {
 #pragma unroll
-            for (uint32_t n = 0; n < 8; ++n) {
-              const uint32_t tokrow = 8 * c + n;
-              if (tokrow < Te) a.y[((size_t)z * a.S + off + tokrow) * a.rows + row] = __uint_as_float(v[n]);
+              for (uint32_t n = 0; n < 8; ++n) {
+                const uint32_t tokrow = 8 * c + n;
+                if (tokrow < Te) y[(size_t)tokrow * a.rows + row] = __uint_as_float(v[n]);
+              }
             }
           }
         }
       }
     }
+    // the next piece's MMAs overwrite the accumulators: only once they have been read
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (*give_up) break;
   }
   tc_fence_before();
   __syncthreads();
@@ -466,14 +546,16 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
 
 // ---- routing: slots grouped by expert ---------------------------------------------------
 // slot_of[t*k + j] = slot of the j-th choice of token t (0xFFFFFFFF for an id out of range);
-// slots of an expert are consecutive, in token order.
+// slots of an expert are consecutive, in token order.  active[0] = number of experts with
+// tokens, active[1..] their ids in ascending order; slot_active[slot] = position of the slot's
+// expert in that list.
 __global__ void route_kernel(const int32_t *topk_ids, uint32_t S, uint32_t k, uint32_t E, uint32_t max_per_expert,
                              uint32_t *expert_offset, uint32_t *active, uint32_t *slot_token, uint32_t *slot_of,
-                             uint32_t *status) {
-  extern __shared__ uint32_t sh[];   // [E] counts, [E] cursors, [S] ids
-  uint32_t *cnt = sh, *cursor = sh + E;
-  int32_t *ids = reinterpret_cast<int32_t *>(sh + 2 * E);
-  for (uint32_t i = threadIdx.x; i < 2 * E; i += blockDim.x) sh[i] = 0;
+                             uint32_t *slot_active, uint32_t *status) {
+  extern __shared__ uint32_t sh[];   // [E] counts, [E] cursors, [E] position in the active list, [S] ids
+  uint32_t *cnt = sh, *cursor = sh + E, *apos = sh + 2 * E;
+  int32_t *ids = reinterpret_cast<int32_t *>(sh + 3 * E);
+  for (uint32_t i = threadIdx.x; i < 3 * E; i += blockDim.x) sh[i] = 0;
   __syncthreads();
   for (uint32_t i = threadIdx.x; i < S; i += blockDim.x) {
     const int32_t ex = topk_ids[i];
@@ -488,7 +570,10 @@ __global__ void route_kernel(const int32_t *topk_ids, uint32_t S, uint32_t k, ui
       expert_offset[x] = run;
       cursor[x] = run;
       if (cnt[x] > max_per_expert) report(status, kStatusBadDescriptor);
-      if (cnt[x]) active[1 + n_active++] = x;
+      if (cnt[x]) {
+        apos[x] = n_active;
+        active[1 + n_active++] = x;
+      }
       run += cnt[x];
     }
     expert_offset[E] = run;
@@ -499,29 +584,48 @@ __global__ void route_kernel(const int32_t *topk_ids, uint32_t S, uint32_t k, ui
       if (ex >= 0 && (uint32_t)ex < E) {
         slot = cursor[ex]++;
         slot_token[slot] = i / k;
+        slot_active[slot] = apos[ex];
       }
       slot_of[i] = slot;
     }
   }
 }
 
-// h = bf16(SiLU(g) * u); g = sum of the `splits` partial blocks gu[0 .. splits), u of gu[splits .. 2*splits),
-// each block fp32 [n]
-__global__ void swiglu_kernel(const float *gu, uint32_t splits, uint16_t *h, uint64_t n) {
-  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
-    float gv = 0.f, uv = 0.f;
-    for (uint32_t sp = 0; sp < splits; ++sp) {
-      gv += gu[(uint64_t)sp * n + i];
-      uv += gu[(uint64_t)(splits + sp) * n + i];
-    }
-    const float hv = gv / (1.0f + __expf(-gv)) * uv;
-    h[i] = __bfloat16_as_ushort(__float2bfloat16_rn(hv));
+// How a matmul launch shared out its steps, for the kernels that add its partial sums.
+struct PartsOf {
+  const uint32_t *active;       // [0] = experts with tokens
+  const uint32_t *slot_active;  // [S]
+  uint32_t n_mats, n_groups, steps, min_units, max_parts, grid, rows_per_group;
+  // number of partial sums of (slot, matrix, row)
+  __device__ __forceinline__ uint32_t parts(uint32_t slot, uint32_t mat, uint32_t row) const {
+    const uint64_t U = (uint64_t)__ldg(active) * n_mats * n_groups * steps;
+    if (U == 0) return 0;
+    const uint32_t P = ffn_ctas_in_use(U, grid, min_units);
+    const uint64_t job = ((uint64_t)__ldg(slot_active + slot) * n_mats + mat) * n_groups + row / rows_per_group;
+    uint32_t c0, n;
+    ffn_job_parts(job, steps, U, P, &c0, &n);
+    return n < max_parts ? n : max_parts;
   }
+};
+
+// h = bf16(SiLU(g) * u) for the slots in use; g = sum of the partial blocks gu[0][p], u of gu[1][p], each block
+// fp32 [S][I].  grid = (ceil(I / blockDim), S)
+__global__ void swiglu_kernel(const float *gu, const PartsOf po, const uint32_t *expert_offset, uint32_t E, uint32_t S,
+                              uint32_t I, uint16_t *h) {
+  const uint32_t slot = blockIdx.y, row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= I || slot >= __ldg(expert_offset + E)) return;
+  const size_t at = (size_t)slot * I + row, block = (size_t)S * I;
+  float gv = 0.f, uv = 0.f;
+  const uint32_t pg = po.parts(slot, 0, row), pu = po.parts(slot, 1, row);
+  for (uint32_t p = 0; p < pg; ++p) gv += gu[p * block + at];
+  for (uint32_t p = 0; p < pu; ++p) uv += gu[(po.max_parts + p) * block + at];
+  const float hv = gv / (1.0f + __expf(-gv)) * uv;
+  h[at] = __bfloat16_as_ushort(__float2bfloat16_rn(hv));
 }
 
-// out[t] = bf16( sum_j w[t,j] * sum_split y[split][slot_of[t,j]] )
-__global__ void combine_kernel(const float *y, const uint32_t *slot_of, const float *topk_weights, uint32_t T,
-                               uint32_t k, uint32_t S, uint32_t H, uint32_t splits, uint16_t *out) {
+// out[t] = bf16( sum_j w[t,j] * sum_p y[p][slot_of[t,j]] )
+__global__ void combine_kernel(const float *y, const PartsOf po, const uint32_t *slot_of, const float *topk_weights,
+                               uint32_t T, uint32_t k, uint32_t S, uint32_t H, uint16_t *out) {
   const uint32_t t = blockIdx.y;
   for (uint32_t c = blockIdx.x * blockDim.x + threadIdx.x; c < H; c += gridDim.x * blockDim.x) {
     float acc = 0.f;
@@ -529,7 +633,8 @@ __global__ void combine_kernel(const float *y, const uint32_t *slot_of, const fl
       const uint32_t slot = slot_of[t * k + j];
       if (slot == 0xFFFFFFFFu) continue;
       float v = 0.f;
-      for (uint32_t sp = 0; sp < splits; ++sp) v += y[((size_t)sp * S + slot) * H + c];
+      const uint32_t n = po.parts(slot, 0, c);
+      for (uint32_t p = 0; p < n; ++p) v += y[((size_t)p * S + slot) * H + c];
       acc += (topk_weights ? topk_weights[t * k + j] : 1.0f) * v;
     }
     out[(size_t)t * H + c] = __bfloat16_as_ushort(__float2bfloat16_rn(acc));
@@ -541,26 +646,34 @@ __global__ void combine_kernel(const float *y, const uint32_t *slot_of, const fl
 namespace {
 
 struct FfnPlan {
-  uint32_t S, groups, n_warps, smem, splits_gu, splits_dn;
+  uint32_t S, groups, n_warps, smem, grid;
+  uint32_t groups_gu, groups_dn;     // strip groups per matrix
+  uint32_t min_gu, min_dn;           // smallest share of a CTA, in K steps
+  uint32_t parts_gu, parts_dn;       // bound on the partial sums of a job
   bool lane16;
-  uint64_t off_offsets, off_active, off_slot_token, off_slot_of, off_gu, off_h, off_y, total;
-  uint32_t max_active;
+  uint64_t off_offsets, off_active, off_slot_token, off_slot_of, off_slot_active, off_gu, off_h, off_y, total;
 };
 
-// K splits so that the CTAs of the busiest plausible case fill the GPU a few times over:
-// `ctas` CTAs exist without splitting, `steps` K steps are there to split
-uint32_t pick_splits(uint32_t ctas, uint32_t steps) {
-  const uint32_t target = 4 * 148;
-  uint32_t splits = 1;
-  while (splits * 2 <= 8 && ctas * splits < target && steps / (splits * 2) >= 2) splits *= 2;
-  return splits;
+// Smallest share of a CTA in K steps, for a launch whose jobs have `steps` steps each and that has at least
+// `units_min` steps in all (one expert with tokens): as large as keeps `grid` CTAs busy even then, but never so
+// small that a job is cut into more than nine partial sums.
+uint32_t pick_min_units(uint64_t units_min, uint32_t steps, uint32_t grid) {
+  uint64_t m = units_min / grid;
+  if (m > steps) m = steps;
+  const uint32_t floor_ = (steps + 7) / 8;
+  return m < floor_ ? floor_ : (uint32_t)m;
 }
 
-zipmoe_status make_plan(uint32_t T, uint32_t k, const zipmoe_compressed_experts *ex, FfnPlan *p) {
+int g_sm_count[64];
+
+zipmoe_status make_plan(uint32_t T, uint32_t k, const zipmoe_compressed_experts *ex, uint32_t grid, FfnPlan *p) {
   if (!ex || T == 0 || k == 0 || T > 64 || k > 8 || ex->n_experts == 0 || ex->n_experts > 256) return ZIPMOE_ERR_UNSUPPORTED;
   if (ex->hidden == 0 || ex->inter == 0 || ex->hidden % 256 || ex->inter % 256) return ZIPMOE_ERR_UNSUPPORTED;
+  if (ex->hidden > 64 * 256 || ex->inter > 64 * 256) return ZIPMOE_ERR_UNSUPPORTED;   // a strip's tiles are looked up by 64
+                                                                                      // lanes; step counts stay in 32 bits
   p->S = T * k;
   p->groups = (T + 7) / 8;
+  p->grid = grid;
   // as many decode warps as fit; the 32 KB conflict-free table if it still fits beside them, else the 16 KB one
   uint32_t nw = zipmoe_dev::kFfnMaxWarps;
   p->lane16 = zipmoe_dev::ffn_smem_bytes(nw, p->groups, false) > 227u * 1024u;
@@ -569,21 +682,42 @@ zipmoe_status make_plan(uint32_t T, uint32_t k, const zipmoe_compressed_experts 
   if (zipmoe_dev::ffn_smem_bytes(nw, p->groups, p->lane16) > 227u * 1024u) return ZIPMOE_ERR_UNSUPPORTED;
   p->n_warps = nw;
   p->smem = zipmoe_dev::ffn_smem_bytes(nw, p->groups, p->lane16);
-  const uint32_t active = p->S < ex->n_experts ? p->S : ex->n_experts;   // at most this many experts get tokens
-  p->splits_gu = pick_splits(active * 2 * ((ex->inter / 16 + nw - 1) / nw), ex->hidden / 256);
-  p->splits_dn = pick_splits(active * ((ex->hidden / 16 + nw - 1) / nw), ex->inter / 256);
+  const uint32_t steps_gu = ex->hidden / 256, steps_dn = ex->inter / 256;
+  p->groups_gu = (ex->inter / 16 + nw - 1) / nw;
+  p->groups_dn = (ex->hidden / 16 + nw - 1) / nw;
+  p->min_gu = pick_min_units(2ull * p->groups_gu * steps_gu, steps_gu, grid);
+  p->min_dn = pick_min_units(1ull * p->groups_dn * steps_dn, steps_dn, grid);
+  p->parts_gu = (steps_gu + p->min_gu - 1) / p->min_gu + 1;
+  p->parts_dn = (steps_dn + p->min_dn - 1) / p->min_dn + 1;
   auto up = [](uint64_t v) { return (v + 255) / 256 * 256; };
   uint64_t at = 0;
   p->off_offsets = at; at = up(at + 4ull * (ex->n_experts + 1));
   p->off_active = at; at = up(at + 4ull * (ex->n_experts + 1));
-  p->max_active = active;
   p->off_slot_token = at; at = up(at + 4ull * p->S);
   p->off_slot_of = at; at = up(at + 4ull * p->S);
-  p->off_gu = at; at = up(at + 2ull * p->splits_gu * p->S * ex->inter * 4);
+  p->off_slot_active = at; at = up(at + 4ull * p->S);
+  p->off_gu = at; at = up(at + 2ull * p->parts_gu * p->S * ex->inter * 4);
   p->off_h = at; at = up(at + (uint64_t)p->S * ex->inter * 2);
-  p->off_y = at; at = up(at + (uint64_t)p->splits_dn * p->S * ex->hidden * 4);
+  p->off_y = at; at = up(at + (uint64_t)p->parts_dn * p->S * ex->hidden * 4);
   p->total = at;
   return ZIPMOE_OK;
+}
+
+// The workspace is sized for a grid of this many CTAs when no device is there to ask (a host-only size query);
+// with a device, its number of SMs is used.  Fewer CTAs never need more partial sums.
+constexpr uint32_t kPlanGridDefault = 148;
+
+uint32_t plan_grid() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
+    if (g_sm_count[dev] > 0) return (uint32_t)g_sm_count[dev];
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
+      g_sm_count[dev] = sms;
+      return (uint32_t)sms;
+    }
+  }
+  (void)cudaGetLastError();   // no device: not an error for a size query
+  return kPlanGridDefault;
 }
 
 bool g_ffn_ready[64];
@@ -594,7 +728,7 @@ extern "C" zipmoe_status zipmoe_ffn_workspace_bytes(uint32_t T, uint32_t k, cons
                                                     uint64_t *workspace_bytes) {
   if (!workspace_bytes) return ZIPMOE_ERR_INVALID_ARG;
   FfnPlan p;
-  zipmoe_status rc = make_plan(T, k, experts, &p);
+  zipmoe_status rc = make_plan(T, k, experts, plan_grid(), &p);
   if (rc != ZIPMOE_OK) return rc;
   *workspace_bytes = p.total;
   return ZIPMOE_OK;
@@ -607,7 +741,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
                                                   zipmoe_stream stream_) {
   using namespace zipmoe_dev;
   FfnPlan p;
-  zipmoe_status rc = make_plan(T, k, ex, &p);
+  zipmoe_status rc = make_plan(T, k, ex, plan_grid(), &p);
   if (rc != ZIPMOE_OK) return rc;
   if (!tokens || !topk_ids || !out || !workspace || !ex->chunks || !ex->tensor_first_chunk || !ex->tables ||
       !ex->payload || !ex->sm || ex->n_chunks == 0 || ex->n_tables == 0)
@@ -636,13 +770,14 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   uint32_t *active = reinterpret_cast<uint32_t *>(ws + p.off_active);
   uint32_t *slot_token = reinterpret_cast<uint32_t *>(ws + p.off_slot_token);
   uint32_t *slot_of = reinterpret_cast<uint32_t *>(ws + p.off_slot_of);
+  uint32_t *slot_active = reinterpret_cast<uint32_t *>(ws + p.off_slot_active);
   float *gu = reinterpret_cast<float *>(ws + p.off_gu);
   uint16_t *h = reinterpret_cast<uint16_t *>(ws + p.off_h);
   float *y = reinterpret_cast<float *>(ws + p.off_y);
   const uint32_t E = ex->n_experts, H = ex->hidden, I = ex->inter, S = p.S;
 
-  route_kernel<<<1, 256, (2 * E + S) * sizeof(uint32_t), stream>>>(topk_ids, S, k, E, 8 * p.groups, expert_offset, active,
-                                                                   slot_token, slot_of, status_word);
+  route_kernel<<<1, 256, (3 * E + S) * sizeof(uint32_t), stream>>>(topk_ids, S, k, E, 8 * p.groups, expert_offset, active,
+                                                                   slot_token, slot_of, slot_active, status_word);
 
   FfnArgs a;
   a.la.chunks = ex->chunks;
@@ -666,38 +801,53 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.S = S;
   a.smem_bytes = p.smem;
   const uint32_t threads = (p.n_warps + p.n_warps / zipmoe_dev::kGroupWarps + 1) * 32;
+  PartsOf po;
+  po.active = active;
+  po.slot_active = slot_active;
+  po.grid = p.grid;
+  po.rows_per_group = 16 * p.n_warps;
 
-  // gate and up: partial Y[matrix][split] = W_{1,3}[:, split] X[:, split]
+  // gate and up: partial sums of W_{1,3} X over the pieces of each job
   a.slot_token = slot_token;
   a.x = tokens;
   a.y = gu;
   a.rows = I;
   a.K = H;
   a.tensor_base = 0;
-  a.splits = p.splits_gu;
-  a.steps_per_split = (H / 256 + p.splits_gu - 1) / p.splits_gu;
-  dim3 grid_gu((I / 16 + p.n_warps - 1) / p.n_warps, p.max_active, 2 * p.splits_gu);
-  if (p.lane16) ffn_matmul_kernel<true><<<grid_gu, threads, p.smem, stream>>>(a);
-  else ffn_matmul_kernel<false><<<grid_gu, threads, p.smem, stream>>>(a);
+  a.n_mats = 2;
+  a.n_groups = p.groups_gu;
+  a.min_units = p.min_gu;
+  a.max_parts = p.parts_gu;
+  if (p.lane16) ffn_matmul_kernel<true><<<p.grid, threads, p.smem, stream>>>(a);
+  else ffn_matmul_kernel<false><<<p.grid, threads, p.smem, stream>>>(a);
 
-  const uint64_t n_h = (uint64_t)S * I;
-  const unsigned act_blocks = (unsigned)((n_h + 1023) / 1024 < 592 ? (n_h + 1023) / 1024 : 592);
-  swiglu_kernel<<<act_blocks, 256, 0, stream>>>(gu, p.splits_gu, h, n_h);
+  po.n_mats = 2;
+  po.n_groups = p.groups_gu;
+  po.steps = H / 256;
+  po.min_units = p.min_gu;
+  po.max_parts = p.parts_gu;
+  swiglu_kernel<<<dim3((I + 255) / 256, S), 256, 0, stream>>>(gu, po, expert_offset, E, S, I, h);
 
-  // down: partial Y[split] = W_2[:, split] H[:, split]
+  // down: partial sums of W_2 H
   a.slot_token = nullptr;
   a.x = h;
   a.y = y;
   a.rows = H;
   a.K = I;
   a.tensor_base = 2;
-  a.splits = p.splits_dn;
-  a.steps_per_split = (I / 256 + p.splits_dn - 1) / p.splits_dn;
-  dim3 grid_dn((H / 16 + p.n_warps - 1) / p.n_warps, p.max_active, p.splits_dn);
-  if (p.lane16) ffn_matmul_kernel<true><<<grid_dn, threads, p.smem, stream>>>(a);
-  else ffn_matmul_kernel<false><<<grid_dn, threads, p.smem, stream>>>(a);
+  a.n_mats = 1;
+  a.n_groups = p.groups_dn;
+  a.min_units = p.min_dn;
+  a.max_parts = p.parts_dn;
+  if (p.lane16) ffn_matmul_kernel<true><<<p.grid, threads, p.smem, stream>>>(a);
+  else ffn_matmul_kernel<false><<<p.grid, threads, p.smem, stream>>>(a);
 
-  combine_kernel<<<dim3((H + 255) / 256, T), 256, 0, stream>>>(y, slot_of, topk_weights, T, k, S, H, p.splits_dn, out);
+  po.n_mats = 1;
+  po.n_groups = p.groups_dn;
+  po.steps = I / 256;
+  po.min_units = p.min_dn;
+  po.max_parts = p.parts_dn;
+  combine_kernel<<<dim3((H + 255) / 256, T), 256, 0, stream>>>(y, po, slot_of, topk_weights, T, k, S, H, out);
   return cudaGetLastError() == cudaSuccess ? ZIPMOE_OK : ZIPMOE_ERR_CUDA;
 }
 
