@@ -178,22 +178,34 @@ class ClockSampler(threading.Thread):
 
 
 # ----------------------------------------------------------------------------- fused expert FFN
-def bench_ffn(dev, iters=20, cpu_tokens=2, token_counts=(1, 16, 64)):
-    """Fused decode + expert SwiGLU FFN on 8 experts of 4096 -> 14336 -> 4096 (top-2 of 8, Zipf(1.2)
-    popularity) for T = 1, 16, 64 tokens, against decode-then-GEMM: zipmoe_decode of the routed experts
-    into bf16 followed by torch matmuls on the same stream.  Also times the CPU oracle's FFN on a few tokens."""
+def bench_ffn(dev, iters=20, cpu_tokens=2, token_counts=(1, 16, 64), config="large"):
+    """Fused decode + expert SwiGLU FFN against decode-then-GEMM (zipmoe_decode of the routed experts into bf16
+    followed by torch matmuls on the same stream), Zipf(1.2) expert popularity.
+      config "large": 8 experts of 4096 -> 14336 -> 4096, top-2, T = 1, 16, 64 tokens; also times the CPU oracle's
+                      FFN on a few tokens;
+      config "small": the 64 experts of the paper's own model shape, 2048 -> 1408 -> 2048 (intermediate size
+                      zero-padded to 1536 before encoding), top-6, T = 1, 16 tokens."""
     import torch
     from paper_2601_21198_b200 import binding, inputs, workloads
-    w = workloads.large_layer(layout=binding.LAYOUT_BLOCKED, keep_originals=True)
-    ex = binding.DeviceExperts(w.blobs, 4096, 14336, dev)
-    per_expert = [binding.DecodePlan(w.blobs[3 * e: 3 * e + 3]).to_device(dev) for e in range(8)]
+    if config == "large":
+        w = workloads.large_layer(layout=binding.LAYOUT_BLOCKED, keep_originals=True)
+        E, H, I, k = 8, 4096, 14336, 2
+        label = "8 experts 4096->14336->4096 bf16 (blocked layout, 256K-element chunks), top-2, Zipf(1.2)"
+    else:
+        w = workloads.small_layer_ffn(keep_originals=False)
+        E, H, I, k = 64, w.hidden, w.inter, 6
+        label = "64 experts 2048->1408->2048 bf16, intermediate size zero-padded to 1536 (blocked layout, 64K-element chunks), top-6, Zipf(1.2)"
+        token_counts = tuple(t for t in token_counts if t <= 16)
+        cpu_tokens = 0
+    ex = binding.DeviceExperts(w.blobs, H, I, dev)
+    per_expert = [binding.DecodePlan(w.blobs[3 * e: 3 * e + 3]).to_device(dev) for e in range(E)]
     dense = [p.new_output() for p in per_expert]
     expert_bytes = [sum(i.payload_bytes + i.n_elems for i in p.plan.infos) for p in per_expert]
     stream = torch.cuda.current_stream(dev)
     out = {}
     for T in token_counts:
-        tok = inputs.tokens(T, 4096, seed=100 + T)
-        ids, wts = inputs.routing(T, n_experts=8, k=2, seed=T)
+        tok = inputs.tokens(T, H, seed=100 + T)
+        ids, wts = inputs.routing(T, n_experts=E, k=k, seed=T)
         d_tok = torch.from_numpy(tok.view(np.int16)).to(dev)
         d_ids = torch.from_numpy(ids).to(dev)
         d_wts = torch.from_numpy(wts).to(dev)
@@ -206,16 +218,16 @@ def bench_ffn(dev, iters=20, cpu_tokens=2, token_counts=(1, 16, 64)):
         x_bf = d_tok.view(torch.bfloat16)
         sel = {e: (torch.from_numpy(np.nonzero(ids == e)[0]).to(dev), torch.from_numpy(wts[ids == e]).to(dev))
                for e in active}
-        acc = torch.zeros(T, 4096, dtype=torch.float32, device=dev)
+        acc = torch.zeros(T, H, dtype=torch.float32, device=dev)
 
         def unfused():
             acc.zero_()
             for e in active:
                 per_expert[e].decode(dense[e])
                 p = per_expert[e].plan
-                w1 = p.tensor_slice(dense[e], 0).view(torch.bfloat16).view(14336, 4096)
-                w3 = p.tensor_slice(dense[e], 1).view(torch.bfloat16).view(14336, 4096)
-                w2 = p.tensor_slice(dense[e], 2).view(torch.bfloat16).view(4096, 14336)
+                w1 = p.tensor_slice(dense[e], 0).view(torch.bfloat16).view(I, H)
+                w3 = p.tensor_slice(dense[e], 1).view(torch.bfloat16).view(I, H)
+                w2 = p.tensor_slice(dense[e], 2).view(torch.bfloat16).view(H, I)
                 rows, wt = sel[e]
                 xe = x_bf[rows]
                 h = torch.nn.functional.silu(xe @ w1.T) * (xe @ w3.T)
@@ -242,7 +254,7 @@ def bench_ffn(dev, iters=20, cpu_tokens=2, token_counts=(1, 16, 64)):
                           "compressed_gbs": nbytes / us_f / 1e3, "decode_then_gemm_us": us_u,
                           "speedup_vs_decode_then_gemm": us_u / us_f, "max_abs_diff_vs_decode_then_gemm": diff,
                           "status": int(ex.dev.status.item())}
-    out["config"] = "8 experts 4096->14336->4096 bf16 (blocked layout, 256K-element chunks), top-2, Zipf(1.2)"
+    out["config"] = label
     if not cpu_tokens:
         return out
     # CPU oracle FFN on a few tokens of the T = 16 case (fp64 numpy)
@@ -274,7 +286,7 @@ def run_ours(args):
     from paper_2601_21198_b200 import binding, build
     build.build()
     if args.ffn_only:      # profiling captures of the fused kernels on one token count
-        res = bench_ffn(dev, iters=args.ffn_iters, cpu_tokens=0, token_counts=(args.ffn_only,))
+        res = bench_ffn(dev, iters=args.ffn_iters, cpu_tokens=0, token_counts=(args.ffn_only,), config=args.ffn_config)
         print(json.dumps({"ffn": res}))
         return
     w = build_workload(args.workload, keep_originals=False, experts=args.experts, max_code_len=args.max_code_len)
@@ -415,6 +427,7 @@ def run_ours(args):
             del dplan, out, h_pay, h_sm, h_out
             torch.cuda.empty_cache()
             line["ffn"] = bench_ffn(dev)
+            line["ffn_small_experts"] = bench_ffn(dev, config="small")
         if world == 1:
             cores = os.cpu_count() or 1
             count = int(max(cores, 20.0 / oracle_seconds_per_tensor(w.blobs[0])))   # ~20 s of CPU work
@@ -447,6 +460,8 @@ def main():
     ap.add_argument("--ffn-only", type=int, default=0, metavar="T",
                     help="run only the fused expert-FFN section for T tokens (profiling captures)")
     ap.add_argument("--ffn-iters", type=int, default=20)
+    ap.add_argument("--ffn-config", default="large", choices=["large", "small"],
+                    help="expert shapes of --ffn-only: 8 x 4096->14336->4096 top-2, or 64 x 2048->1408->2048 top-6")
     ap.add_argument("--no-ffn", action="store_true", help="skip the fused expert-FFN section of the report")
     ap.add_argument("--max-code-len", type=int, default=0, help="longest Huffman code the encoder may use (8..12)")
     ap.add_argument("--experts", type=int, default=None,

@@ -271,6 +271,23 @@ class DevicePlan:
                       self.sm, p.sm_bytes, out, p.out_elems, self.status, s.cuda_stream, p.max_record_bytes)
 
 
+def pad_expert_inter(w1, w3, w2, multiple=256):
+    """The fused expert FFN takes experts whose hidden and intermediate sizes are multiples of 256.  An expert with
+    another intermediate size (w1, w3 [inter, hidden]; w2 [hidden, inter], uint16 bf16 patterns) is padded with zero
+    rows (w1, w3) and zero columns (w2) up to the next multiple: the added units compute SiLU(0) * 0 = 0 and feed
+    zero weights, so the FFN's result is unchanged.  Returns (w1, w3, w2, padded inter)."""
+    inter, hidden = w1.shape
+    assert w3.shape == (inter, hidden) and w2.shape == (hidden, inter)
+    padded = -(-inter // multiple) * multiple
+    if padded == inter:
+        return w1, w3, w2, inter
+    a = np.zeros((padded, hidden), np.uint16)
+    b = np.zeros((padded, hidden), np.uint16)
+    c = np.zeros((hidden, padded), np.uint16)
+    a[:inter], b[:inter], c[:, :inter] = w1, w3, w2
+    return a, b, c, padded
+
+
 class DeviceExperts:
     """The compressed experts of one layer on the device: blobs[3*e + j] (j: 0 w1, 1 w3, 2 w2, blocked
     layout) laid out by DecodePlan, plus the CompressedExperts struct the fused call takes."""

@@ -70,6 +70,26 @@ def small_layer(n_experts=64, keep_originals=True, layout=0, max_code_len=0):
     return Workload("moe%d_2048x1408_chunk64K" % n_experts, *_encode_all(items, 65536, layout, keep_originals, max_code_len))
 
 
+def small_layer_ffn(n_experts=64, keep_originals=True, max_code_len=0):
+    """The 64-expert layer for the fused FFN: every expert's intermediate size 1408 is padded to 1536 with zero
+    units (binding.pad_expert_inter) and its three matrices are encoded with the blocked layout.  `originals`
+    keeps the unpadded matrices; `inter` is the padded size."""
+    def padded(e, j):
+        ws = [inputs.small_expert_tensor(e, t) for t in range(3)]
+        return binding.pad_expert_inter(*ws)[j]
+
+    items = []
+    for e in range(n_experts):
+        for j, (name, _) in enumerate(inputs.SMALL_EXPERT_TENSORS):
+            items.append(("e%d.%s" % (e, name), lambda e=e, j=j: padded(e, j)))
+    w = Workload("moe%d_ffn_2048x1408_pad1536" % n_experts,
+                 *_encode_all(items, 65536, binding.LAYOUT_BLOCKED, False, max_code_len))
+    w.hidden, w.inter = 2048, 1536
+    if keep_originals:
+        w.originals = [inputs.small_expert_tensor(e, j) for e in range(n_experts) for j in range(3)]
+    return w
+
+
 def large_layer(n_experts=8, keep_originals=True, layout=0, hidden=4096, inter=14336, chunk_elems=262144,
                 max_code_len=0):
     """8 experts x {w1, w3 [14336,4096]; w2 [4096,14336]} with outlier channels, 256K-element chunks (~2.8 GB bf16)."""

@@ -119,6 +119,27 @@ def test_large_experts_config(zb, T):
     check(out.cpu().numpy().view(np.uint16)[rows], want, ("large", T))
 
 
+@pytest.mark.parametrize("T", [1, 16])
+def test_paper_shape_experts_with_padded_intermediate_size(zb, T):
+    """Experts of the paper's own models, 2048 -> 1408 -> 2048, top-6: the intermediate size is not a multiple of
+    256, so the experts are zero-padded to 1536 before they are encoded.  The oracle FFN runs on the unpadded
+    matrices: the padding must not change the result.  16 of the 64 experts keep the test short."""
+    import torch
+    from paper_2601_21198_b200 import workloads
+    E, k = 16, 6
+    w = workloads.small_layer_ffn(n_experts=E)
+    assert w.inter == 1536 and all(i.rows % 16 == 0 and i.cols % 256 == 0 for i in w.plan.infos)
+    ex = zb.DeviceExperts(w.blobs, w.hidden, w.inter)
+    tok = inputs.tokens(T, w.hidden, seed=300 + T)
+    ids, wts = inputs.routing(T, n_experts=E, k=k, seed=300 + T)
+    out = ex.ffn(torch.from_numpy(tok.view(np.int16)).cuda(), torch.from_numpy(ids).cuda(), torch.from_numpy(wts).cuda())
+    torch.cuda.synchronize()
+    assert int(ex.dev.status.item()) == 0
+    rows = np.arange(T) if T <= 4 else np.random.default_rng(T).choice(T, 4, replace=False)
+    want, _ = oracle_out(w.originals, tok, ids, wts, rows)
+    check(out.cpu().numpy().view(np.uint16)[rows], want, ("paper shape", T))
+
+
 _cache = {}
 
 
