@@ -116,7 +116,7 @@ __device__ __forceinline__ void sts_v4(uint32_t addr, const uint4 &v) {
 // ordered with the other volatile asm of the decoder, so the load is issued where it is written: early
 __device__ __forceinline__ uint2 ldg_v2_early(const uint8_t *p) {
   uint2 v;
-  asm volatile("ld.global.nc.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
   return v;
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
