@@ -71,9 +71,12 @@
  *       its k-th bit is bit S + k;
  *     sub-stream 1 codes those of the odd iterations i = 1, 3, 5, ... < I and
  *       runs backwards from E: its k-th bit is bit E - 1 - k.
- *   The two meet without a gap.  (Two independent streams per lane let a decoder
- *   work on two codes at a time at no cost in size; the paper leaves the order
- *   of elements inside a shard open.)
+ *   Bits of the range that belong to neither sub-stream lie between their ends:
+ *   at most 63 of them, all zero (an encoder may insert them, e.g. to keep lanes
+ *   of equal length from starting at the same word offset; this oracle's
+ *   encoder inserts none).  (Two independent streams per lane let a decoder work
+ *   on two codes at a time at no cost in size; the paper leaves the order of
+ *   elements inside a shard open.)
  *
  *   Sign+mantissa section: byte q*tile_elems + pos holds
  *     (sign << 7) | mantissa  of the element at (q, pos); zero padded to 16.
@@ -524,7 +527,10 @@ int zo_decode_chunk(const uint8_t *blob, uint64_t bytes, uint32_t k, uint16_t *o
           uint8_t s = smsec[q * h.tile_elems + pos];
           zo_merge(&e, &s, 1, &out[f]);
         }
-      if (fwd != bwd) return ZO_ERR_CORRUPT; /* the sub-streams must meet exactly */
+      /* what is left between the sub-streams is padding: short and zero */
+      if (bwd - fwd > 63) return ZO_ERR_CORRUPT;
+      for (uint64_t g = fwd; g < bwd; ++g)
+        if (get_bit(rec + ZO_REC_HEAD, g)) return ZO_ERR_CORRUPT;
       p = p_end;
     }
   }

@@ -208,8 +208,7 @@ struct TileWork {
   const uint8_t *sm;    // global address of the tile's sign+mantissa bytes
   uint16_t *out;        // global address of the tile's first element
   uint32_t rec_bytes, pitch, valid, iters, pieces;
-  bool ok, staged;
-  bool wide;            // staged across both record stages (a record of up to 2 * kPayStage - kPaySlack bytes)
+  bool ok, staged;      // staged: the record fits a record stage of the calling kernel
 };
 
 struct LaunchArgs {
@@ -242,11 +241,10 @@ static_assert(sizeof(zipmoe_chunk_desc) == 80, "descriptor is read as five 16-by
 
 // Everything the decoder needs about tile t of descriptor c, with every offset
 // checked against the sizes of the buffers the launch was given.
-__device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_t t, const bool allow_wide = false) {
+__device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_t t, const uint32_t stage_buf) {
   TileWork w;
   w.ok = false;
   w.staged = false;
-  w.wide = false;
   if (c >= a.n_chunks) return w;
   const uint4 *d = reinterpret_cast<const uint4 *>(a.chunks + c);
   const uint4 d0 = __ldg(d), d1 = __ldg(d + 1), d2 = __ldg(d + 2), d3 = __ldg(d + 3);
@@ -263,7 +261,7 @@ __device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c
   const uint64_t rec_off = pay_off + 16ull * o0;
   if (o1 <= o0) return w;
   w.rec_bytes = (o1 - o0) * 16u;
-  if (w.rec_bytes < 64 || w.rec_bytes > 64 + tile_elems / 8 * ZIPMOE_MAX_CODE_LEN + 16 ||
+  if (w.rec_bytes < 64 || w.rec_bytes > 64 + tile_elems / 8 * ZIPMOE_MAX_CODE_LEN + 32 * 8 + 16 ||   // codes, padding
       rec_off + w.rec_bytes > a.payload_bytes)
     return w;
   w.iters = tile_elems >> 8;
@@ -281,8 +279,7 @@ __device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c
   w.sm = a.sm + sm_tile;
   w.out = a.out + origin;
   w.pitch = pitch;
-  w.wide = allow_wide && w.rec_bytes > (uint32_t)kPayBuf && w.rec_bytes <= (uint32_t)(2 * kPayStage - kPaySlack);
-  w.staged = w.rec_bytes <= (uint32_t)kPayBuf || w.wide;
+  w.staged = w.rec_bytes <= stage_buf;
   w.ok = true;
   return w;
 }

@@ -29,13 +29,30 @@ namespace zipmoe_dev {
 #ifndef ZIPMOE_WARPS
 #define ZIPMOE_WARPS 16
 #endif
-constexpr int kWarps = ZIPMOE_WARPS;                 // warps per CTA, one CTA per SM
-constexpr int kThreads = kWarps * 32;
 constexpr int kPayStages = 2;
 constexpr int kBarsPerWarp = kPayStages + kSmPieces;   // two record stages, one barrier per sign+mantissa slot
-constexpr int kWarpBytes = kPayStages * kPayStage + kSmPieces * kSmPieceBytes;
-constexpr int kSmemBytes = kLutBytes + kWarps * kWarpBytes + kWarps * kBarsPerWarp * 8 + kLutScratchBytes;
-static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
+
+// Two instantiations of the kernel, chosen by the host from the launch's largest tile record:
+//   WIDE = false: record stages of kPayStage bytes (records of up to 2048 bytes: every tensor whose codes average
+//                 less than ~3.9 bits), 16 warps per CTA;
+//   WIDE = true : record stages of 4352 bytes (records of up to 4288 bytes: 8-bit codes everywhere plus the word of
+//                 padding per lane that the encoder gives such tiles, e.g. tensors with near-uniform exponents),
+//                 one warp fewer so that the stages still fit.
+// A record longer than its stage is read from global memory word by word (correct, slow).
+template <bool WIDE>
+struct Cfg {
+#ifndef ZIPMOE_CTAS_PER_SM
+#define ZIPMOE_CTAS_PER_SM 1
+#endif
+  static constexpr int kCtasPerSm = WIDE ? 1 : ZIPMOE_CTAS_PER_SM;
+  static constexpr int kWarps = WIDE ? ZIPMOE_WARPS - 1 : ZIPMOE_WARPS / kCtasPerSm;   // warps per CTA
+  static constexpr int kThreads = kWarps * 32;
+  static constexpr int kStage = WIDE ? 64 + 4096 + 32 * 4 + kPaySlack : kPayStage;   // bytes of a record stage
+  static constexpr int kBuf = kStage - kPaySlack;                         // longest staged record
+  static constexpr int kWarpBytes = kPayStages * kStage + kSmPieces * kSmPieceBytes;
+  static constexpr int kSmemBytes = kLutBytes + kWarps * kWarpBytes + kWarps * kBarsPerWarp * 8 + kLutScratchBytes;
+  static_assert(kCtasPerSm * (kSmemBytes + 1024) <= 228 * 1024, "shared memory per SM");
+};
 
 // Per-warp asynchronous pipeline.  A warp decodes its tiles one after the other;
 // the record of the next tile is copied into the other record stage while the
@@ -43,6 +60,7 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
 // copied into slot p as soon as the current tile is done with its piece p.
 struct WarpPipe {
   uint32_t pay_addr, sm_addr, bar_addr;   // shared addresses: record stages, SM slots, barriers
+  uint32_t stage_bytes;                   // bytes of a record stage
   uint32_t phase;                         // bit b = parity to wait for on barrier b
   uint32_t pending;                       // bit b = a copy on barrier b has been started and not waited for
   uint32_t lane;
@@ -55,13 +73,9 @@ struct WarpPipe {
     return true;
   }
   // all lanes call these; one lane starts the copy
-  // a record of ordinary size goes into `stage`; a wide one (8-bit codes everywhere: 4160 bytes) spans both
-  // stages and uses the first stage's barrier, so no other record can be in flight beside it
-  template <bool WIDE>
   __device__ __forceinline__ void load_record(const TileWork &t, uint32_t stage) {
     if (!t.staged) return;
-    if (WIDE && t.wide) stage = 0;
-    if (lane == 0) bulk_load(pay_addr + stage * kPayStage, t.rec, t.rec_bytes, bar(stage));
+    if (lane == 0) bulk_load(pay_addr + stage * stage_bytes, t.rec, t.rec_bytes, bar(stage));
     pending |= 1u << stage;
   }
   __device__ __forceinline__ void load_sm_piece(const TileWork &t, uint32_t p) {
@@ -105,10 +119,10 @@ struct GlobalSink {
   }
 };
 
-// WIDE: records longer than one record stage may be staged across both (near-incompressible tensors); the
-// host picks the instantiation without it when it knows that no record of the launch is that long.
 template <bool WIDE>
-__global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a) {
+__global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) decode_kernel(const LaunchArgs a) {
+  constexpr int kWarps = Cfg<WIDE>::kWarps, kThreads = Cfg<WIDE>::kThreads, kWarpBytes = Cfg<WIDE>::kWarpBytes;
+  constexpr uint32_t kBuf = Cfg<WIDE>::kBuf;
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t *lut_raw = smem;
   uint8_t *warp_base = smem + kLutBytes;
@@ -122,7 +136,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
 
   WarpPipe pipe;
   pipe.pay_addr = smem_addr(warp_base + warp * kWarpBytes);
-  pipe.sm_addr = pipe.pay_addr + kPayStages * kPayStage;
+  pipe.stage_bytes = Cfg<WIDE>::kStage;
+  pipe.sm_addr = pipe.pay_addr + kPayStages * Cfg<WIDE>::kStage;
   pipe.bar_addr = smem_addr(bars + warp * kBarsPerWarp);
   pipe.phase = 0;
   pipe.pending = 0;
@@ -169,10 +184,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
     TileWork cur;
     cur.ok = false;
     if (g < g_end && !dead) {
-      cur = resolve_tile(a, tc, tt, WIDE);
+      cur = resolve_tile(a, tc, tt, kBuf);
       if (!cur.ok) report(a.status, kStatusBadDescriptor);
       else {
-        pipe.template load_record<WIDE>(cur, stage);
+        pipe.load_record(cur, stage);
         for (uint32_t p = 0; p < cur.pieces; ++p) pipe.load_sm_piece(cur, p);
       }
     }
@@ -186,18 +201,16 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
       uint32_t nxt_issued = 0;
       if (g + 1 < g_end) {
         step();
-        nxt = resolve_tile(a, tc, tt, WIDE);
+        nxt = resolve_tile(a, tc, tt, kBuf);
         if (!nxt.ok) report(a.status, kStatusBadDescriptor);
       }
-      // the next record is fetched while this one is decoded, unless one of the two needs both stages
-      const bool prefetch = nxt.ok && (!WIDE || (!nxt.wide && !(cur.ok && cur.wide)));
-      if (prefetch) pipe.template load_record<WIDE>(nxt, stage ^ 1);   // that stage was released by the __syncwarp below
+      // the next record is fetched while this one is decoded
+      if (nxt.ok) pipe.load_record(nxt, stage ^ 1);   // that stage was released by the __syncwarp below
       if (cur.ok) {
         uint32_t rc = 0;
-        const uint32_t rec_stage = (WIDE && cur.wide) ? 0 : stage;
-        if (cur.staged && !pipe.wait(rec_stage)) rc = kStatusWaitTimeout;
+        if (cur.staged && !pipe.wait(stage)) rc = kStatusWaitTimeout;
         if (rc == 0) {
-          const uint32_t rec_s = pipe.pay_addr + rec_stage * kPayStage;
+          const uint32_t rec_s = pipe.pay_addr + stage * pipe.stage_bytes;
           SmFeed feed{pipe, nxt, nxt_issued};
           GlobalSink sink{cur.out, cur.pitch};
           if (cur.staged) {
@@ -231,7 +244,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const LaunchArgs a)
         }
       }
       __syncwarp();   // every lane is done with the current record stage and SM slots
-      if (WIDE && nxt.ok && !prefetch) pipe.template load_record<WIDE>(nxt, stage ^ 1);
       if (nxt.ok)
         for (; nxt_issued < nxt.pieces; ++nxt_issued) pipe.load_sm_piece(nxt, nxt_issued);
       cur = nxt;
@@ -264,9 +276,9 @@ zipmoe_status prepare_device(int *sm_count) {
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ZIPMOE_ERR_CUDA;
     if (major != 10) return ZIPMOE_ERR_UNSUPPORTED;
     if (cudaFuncSetAttribute(zipmoe_dev::decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             zipmoe_dev::kSmemBytes) != cudaSuccess ||
+                             zipmoe_dev::Cfg<true>::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(zipmoe_dev::decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             zipmoe_dev::kSmemBytes) != cudaSuccess)
+                             zipmoe_dev::Cfg<false>::kSmemBytes) != cudaSuccess)
       return ZIPMOE_ERR_CUDA;
     g_dev[dev].sm_count = sms;
     g_dev[dev].ready = true;
@@ -304,15 +316,18 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
   a.n_chunks = n_chunks;
   a.n_tiles = n_tiles;
   a.n_tables = n_tables;
-  // one CTA per SM, each with a contiguous range of tiles
-  uint32_t ctas = (uint32_t)sms;
+  // CTAs to fill the SMs once, each with a contiguous range of tiles
+  const bool narrow = max_record_bytes != 0 && max_record_bytes <= (uint32_t)zipmoe_dev::Cfg<false>::kBuf;
+  uint32_t ctas = (uint32_t)sms * (narrow ? zipmoe_dev::Cfg<false>::kCtasPerSm : zipmoe_dev::Cfg<true>::kCtasPerSm);
   if (n_tiles < ctas) ctas = n_tiles;
   a.tiles_per_cta = (n_tiles + ctas - 1) / ctas;
   ctas = (n_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  if (max_record_bytes != 0 && max_record_bytes <= (uint32_t)zipmoe_dev::kPayBuf)
-    zipmoe_dev::decode_kernel<false><<<ctas, zipmoe_dev::kThreads, zipmoe_dev::kSmemBytes, st>>>(a);
+  using Narrow = zipmoe_dev::Cfg<false>;
+  using Wide = zipmoe_dev::Cfg<true>;
+  if (narrow)
+    zipmoe_dev::decode_kernel<false><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
   else
-    zipmoe_dev::decode_kernel<true><<<ctas, zipmoe_dev::kThreads, zipmoe_dev::kSmemBytes, st>>>(a);
+    zipmoe_dev::decode_kernel<true><<<ctas, Wide::kThreads, Wide::kSmemBytes, st>>>(a);
   return cudaGetLastError() == cudaSuccess ? ZIPMOE_OK : ZIPMOE_ERR_CUDA;
 }

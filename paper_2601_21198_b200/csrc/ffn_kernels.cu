@@ -278,7 +278,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
         }
         const uint32_t *tab = reinterpret_cast<const uint32_t *>(a.la.payload + pay_off);
         const uint32_t o0 = __ldg(tab + t), o1 = __ldg(tab + t + 1);
-        if (o1 <= o0 || o1 - o0 < 4 || o1 - o0 > (64 + ZIPMOE_TILE_ELEMS_MAX / 8 * ZIPMOE_MAX_CODE_LEN) / 16 + 1 ||
+        if (o1 <= o0 || o1 - o0 < 4 || o1 - o0 > (64 + ZIPMOE_TILE_ELEMS_MAX / 8 * ZIPMOE_MAX_CODE_LEN + 32 * 8) / 16 + 1 ||
             pay_off + 16ull * o1 > a.la.payload_bytes) {
           bad = true;
           continue;

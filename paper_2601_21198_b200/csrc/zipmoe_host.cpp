@@ -62,7 +62,7 @@ zipmoe_status resolve_opts(const zipmoe_encode_opts *o, Opts *r) {
 }
 
 uint64_t tile_record_max(uint32_t tile_elems) {
-  return align_up(kRecordHeadBytes + (uint64_t)tile_elems * ZIPMOE_MAX_CODE_LEN / 8, 16);
+  return align_up(kRecordHeadBytes + (uint64_t)tile_elems * ZIPMOE_MAX_CODE_LEN / 8 + kLanes * 8, 16);   // codes + padding
 }
 
 // Huffman code lengths by the usual greedy merge on a min-heap.  When the tree
@@ -170,6 +170,17 @@ void parallel_for(uint32_t n, uint32_t n_threads, F body) {
   for (auto &th : pool) th.join();
 }
 
+// Zero bits the encoder leaves between a lane's two sub-streams (the format allows up to 63).  When every lane
+// of a tile has the same number of code bits and that number is a multiple of 256 -- a fixed-length code, as
+// near-uniform exponents give -- the lanes' words would all start at the same offsets modulo 8 words, and a decoder
+// that keeps the record in banked shared memory would serialise its word loads.  One word of padding per lane
+// staggers them.
+uint32_t lane_padding_bits(const uint32_t *lane_bits) {
+  for (uint32_t lane = 1; lane < kLanes; ++lane)
+    if (lane_bits[lane] != lane_bits[0]) return 0;
+  return (lane_bits[0] != 0 && lane_bits[0] % 256 == 0) ? 32u : 0u;
+}
+
 // bits of every lane's sub-stream of tile q; returns their sum
 uint64_t tile_lane_bits(const Geometry &g, const uint16_t *x, const uint8_t *len, uint32_t q, uint32_t *lane_bits) {
   const uint32_t valid = g.tile_valid(q);
@@ -259,6 +270,7 @@ zipmoe_status zipmoe_encode(const uint16_t *bf16, uint64_t rows, uint64_t cols, 
     uint32_t q0 = k * g.tiles_per_chunk, m = g.chunk_tiles(k), lane_bits[kLanes];
     for (uint32_t t = 0; t < m; ++t) {
       uint64_t bits = tile_lane_bits(g, bf16, len, q0 + t, lane_bits);
+      bits += (uint64_t)kLanes * lane_padding_bits(lane_bits);
       rec_units[q0 + t] = (uint32_t)(align_up(kRecordHeadBytes + (bits + 7) / 8, 16) / 16);
     }
   });
@@ -312,6 +324,9 @@ zipmoe_status zipmoe_encode(const uint16_t *bf16, uint64_t rows, uint64_t cols, 
       const uint32_t valid = g.tile_valid(q);
       const uint64_t origin = g.tile_origin(q), pitch = g.row_pitch();
       BitWriter bw(rec + kRecordHeadBytes);
+      uint32_t lane_bits[kLanes];
+      tile_lane_bits(g, bf16, len, q, lane_bits);
+      const uint32_t pad_bits = lane_padding_bits(lane_bits);
       for (uint32_t lane = 0; lane < kLanes; ++lane) {
         const uint64_t before = bw.total;
         // sub-stream 0 (even iterations) forwards; sub-stream 1 (odd iterations) is read backwards from the
@@ -329,6 +344,7 @@ zipmoe_status zipmoe_encode(const uint16_t *bf16, uint64_t rows, uint64_t cols, 
             else bw.put(code[s], len[s]);
           }
         }
+        if (pad_bits) bw.put(0, pad_bits);
         while (n_odd) {
           const uint32_t s = odd[--n_odd];
           bw.put(reverse_bits(code[s], len[s]), len[s]);
@@ -436,7 +452,7 @@ zipmoe_status zipmoe_blob_validate(const void *blob_v, uint64_t bytes) {
           uint32_t pos = (i * kLanes + lane) * kGroup;
           if (pos < valid) elems += std::min(kGroup, valid - pos);
         }
-        if (b < elems || b > elems * info.max_code_len) return ZIPMOE_ERR_BAD_FORMAT;
+        if (b < elems || b > elems * info.max_code_len + 63) return ZIPMOE_ERR_BAD_FORMAT;   // up to 63 padding bits
         bits += b;
       }
       if (kRecordHeadBytes * 8 + bits > (r1 - r0) * 8) return ZIPMOE_ERR_BAD_FORMAT;

@@ -157,10 +157,34 @@ def test_ffn_planning_on_the_host(zb):
     assert ctypes.sizeof(zb.CompressedExperts) == 80
 
 
+def test_equal_length_lanes_are_padded_and_still_decode(zb):
+    """Fixed-length codes (all 256 exponents equally frequent) give every lane of a tile the same number of code
+    bits; the encoder then leaves one zero word between each lane's two sub-streams.  The oracle, which inserts
+    no padding itself, must accept and decode such a blob."""
+    from oracle import codec
+    rng = np.random.default_rng(3)
+    e = np.tile(np.arange(256, dtype=np.uint16), 40)
+    rng.shuffle(e)
+    x = (e << 7 | 0x0033).astype(np.uint16)                   # 10240 elements: two full tiles and a half one
+    blob = zb.zipmoe_encode(x, chunk_elems=4096)
+    assert (blob[64:320] == 8).all() and zb.zipmoe_blob_validate(blob) == zb.OK
+    info = zb.zipmoe_blob_info_get(blob)
+    rec = blob[info.payload_off + 16:]
+    assert (rec[:64].view(np.uint16) == 128 * 8 + 32).all()   # first tile: 128 codes of 8 bits and the padding
+    assert np.array_equal(codec.decode(blob), x)
+    bad = blob.copy()
+    bad[info.payload_off + 16 + 64 + 16 * 4] = 1              # lane 0: 16 words forwards, then the padding word
+    with pytest.raises(ValueError):
+        codec.decode(bad)                                     # padding must be zero
+    y = x.copy()
+    y[5] = (7 << 7) | 0x33                                    # no longer a fixed-length code?  still decodes
+    assert np.array_equal(codec.decode(zb.zipmoe_encode(y, chunk_elems=4096)), y)
+
+
 def test_plan_reports_the_largest_tile_record(zb):
     x = inputs.gaussian((64, 1408), 0.02, 5)
     plan = zb.DecodePlan([zb.zipmoe_encode(x, chunk_elems=4096)])
     assert 1300 < plan.max_record_bytes < 1700
     u = np.random.default_rng(0).integers(0, 1 << 16, 20000, dtype=np.uint16)
     plan = zb.DecodePlan([zb.zipmoe_encode(u, chunk_elems=4096)])
-    assert plan.max_record_bytes == 64 + 4096         # 8-bit codes everywhere
+    assert plan.max_record_bytes == 64 + 4096 + 32 * 4   # 8-bit codes everywhere, one word of padding per lane
