@@ -47,7 +47,7 @@ namespace zipmoe_dev {
 #endif
 constexpr int kFfnMaxWarps = ZIPMOE_FFN_WARPS;            // decode warps per CTA, a multiple of the group size
 #ifndef ZIPMOE_FFN_GROUP
-#define ZIPMOE_FFN_GROUP 8
+#define ZIPMOE_FFN_GROUP 16
 #endif
 constexpr int kGroupWarps = ZIPMOE_FFN_GROUP;            // decode warps whose half-tiles form one operand of M = 8 * kGroupWarps (64 or 128)
 static_assert(kGroupWarps == 8 || kGroupWarps == 16, "M is 64 or 128");
