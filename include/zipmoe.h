@@ -263,6 +263,67 @@ zipmoe_status zipmoe_decode_expert_ffn_noalloc(const uint16_t *tokens, uint32_t 
                                                const zipmoe_compressed_experts *experts, uint16_t *out,
                                                uint32_t *status_word, zipmoe_stream stream);
 
+/* ---- cache-pool planning (host only, no CUDA) ------------------------------
+ * The paper's planner sizes four cache pools for experts in different compression states -- F full
+ * tensors, C compressed (E-chunks and SM-chunks), S SM-chunks only, E E-chunks only -- from a
+ * rank-based activation model (Section 3.4 "Compression-Aware Cache Management", Appendix
+ * "Hierarchical Cache Pool Planning": Algorithms 2-4, and the iterative proportional fitting of the
+ * appendix on the maximum-entropy property).  The delays c, v, u it takes are measured by the caller,
+ * e.g. from zipmoe_decode timings.  Pool order everywhere: 0 = F, 1 = C, 2 = S, 3 = E. */
+
+/* Algorithm 2: distribution of the number of experts selected among n ranks that are selected
+ * independently with probabilities q[0..n): phi[h] = P(exactly h), h = 0..n (Poisson binomial).
+ * host in: q (each in [0, 1]); host out: phi[n + 1]. */
+zipmoe_status zipmoe_plan_hit_distribution(const double *q, uint32_t n, double *phi);
+
+/* Selection probabilities q from marginal inclusion probabilities f (0 < f[i] < 1, sum = k) by the
+ * modified iterative proportional fitting of the appendix: weights w start at f and are multiplied
+ * by f[i] / f_t[i], f_t[i] = w[i] R(k-1, N \ {i}) / R(k, N) with R the elementary symmetric
+ * polynomial, until max |f_t - f| <= tol or max_iters passes; q[i] = w[i] / (1 + w[i]).  Choosing
+ * k of the n ranks with probability proportional to the product of their w then includes rank i
+ * with probability f[i].
+ * host in: f[n], k (1 <= k < n <= 512); host out: q[n], *iters_done (may be NULL).
+ * Returns ZIPMOE_ERR_INVALID_ARG if f is not feasible (some f outside (0, 1), or sum != k within 1e-6). */
+zipmoe_status zipmoe_plan_selection_probs(const double *f, uint32_t n, uint32_t k, uint32_t max_iters, double tol,
+                                          double *q, uint32_t *iters_done);
+
+typedef struct {
+  double c;           /* decompression delay of one E-chunk                         */
+  double v;           /* read delay of one E-chunk                                  */
+  double u;           /* read delay of one SM-chunk (one tensor's sign+mantissa)    */
+  uint32_t L;         /* decompression workers                                      */
+  uint32_t K;         /* E-chunks (exponent shards) per tensor                      */
+  uint32_t n_tensors; /* tensors per expert                                         */
+} zipmoe_plan_costs;
+
+/* Algorithm 3: estimated makespan of a sparse layer (without token execution) when k experts are
+ * activated and hits[p] of them are found in pool p: max(T_IO, T_decomp) with
+ *   n_SM = n_tensors (k - h_F - h_C - h_S),  n_E = n_tensors K (k - h_F - h_C - h_E),
+ *   n_D = n_tensors K (k - h_F),  T_IO = n_SM u + n_E v,  T_decomp = (n_E v + n_D c) / L.
+ * host in: k, hits[4] (sum <= k), costs; host out: *makespan. */
+zipmoe_status zipmoe_plan_makespan(uint32_t k, const uint32_t hits[4], const zipmoe_plan_costs *costs, double *makespan);
+
+/* Expected makespan of a cache partition: pools of capacity[p] experts (0 = pool not used) laid on
+ * the popularity ranks in the order F, C, S, E, the remaining ranks being misses; the probability of
+ * a hit pattern h given that exactly k experts are selected is
+ *   Phi_M(k - sum h) / Phi_N(k) * prod_p Phi_p(h_p)      (Section 3.4),
+ * each Phi from Algorithm 2 on the pool's rank interval.
+ * host in: q[n] (selection probabilities by rank), k, capacity[4] (sum <= n), costs; host out: *expected. */
+zipmoe_status zipmoe_plan_expected_makespan(const double *q, uint32_t n, uint32_t k, const uint32_t capacity[4],
+                                            const zipmoe_plan_costs *costs, double *expected);
+
+/* Algorithm 4: grid search over the memory ratios of the pools named in pool_mask (bit p = pool p may
+ * be used; the others get ratio 0), step `step` (0 < step <= 1, 1 / step an integer up to 100).  A
+ * pool with ratio g holds floor(g * budget / expert_size[p]) experts, `budget` and expert_size[p]
+ * (memory of one expert in state p) in the same unit; capacities are cut, in the order F, C, S, E,
+ * so that they sum to at most n.  Returns the ratios with the smallest expected makespan (ties: the
+ * first one in the enumeration order, ratios of F varying slowest) and that makespan.
+ * host in: f[n] inclusion probabilities by rank (as for zipmoe_plan_selection_probs), k, pool_mask,
+ * budget, expert_size[4], costs, step; host out: ratios[4], capacity[4], *expected. */
+zipmoe_status zipmoe_plan_cache_pools(const double *f, uint32_t n, uint32_t k, uint32_t pool_mask, double budget,
+                                      const double expert_size[4], const zipmoe_plan_costs *costs, double step,
+                                      double ratios[4], uint32_t capacity[4], double *expected);
+
 /* Name of a status code (static string). */
 const char *zipmoe_status_string(zipmoe_status s);
 

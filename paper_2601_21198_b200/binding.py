@@ -171,6 +171,78 @@ def zipmoe_recover(exp, sm, n_elems, out_bf16, stream=None):
     _check("zipmoe_recover", _lib.zipmoe_recover(_ptr(exp), _ptr(sm), n_elems, _ptr(out_bf16), _ptr(stream)))
 
 
+# ---- cache-pool planning (host only) ------------------------------------------------------------
+class PlanCosts(ctypes.Structure):
+    """zipmoe_plan_costs: delays c (decompress one E-chunk), v (read one E-chunk), u (read one SM-chunk),
+    L decompression workers, K E-chunks per tensor, n_tensors per expert."""
+    _fields_ = [("c", ctypes.c_double), ("v", ctypes.c_double), ("u", ctypes.c_double), ("L", _u32), ("K", _u32),
+                ("n_tensors", _u32)]
+
+
+_dp = ctypes.POINTER(ctypes.c_double)
+_lib.zipmoe_plan_hit_distribution.argtypes = [_dp, _u32, _dp]
+_lib.zipmoe_plan_selection_probs.argtypes = [_dp, _u32, _u32, _u32, ctypes.c_double, _dp, ctypes.POINTER(_u32)]
+_lib.zipmoe_plan_makespan.argtypes = [_u32, ctypes.POINTER(_u32), ctypes.POINTER(PlanCosts), _dp]
+_lib.zipmoe_plan_expected_makespan.argtypes = [_dp, _u32, _u32, ctypes.POINTER(_u32), ctypes.POINTER(PlanCosts), _dp]
+_lib.zipmoe_plan_cache_pools.argtypes = [_dp, _u32, _u32, _u32, ctypes.c_double, _dp, ctypes.POINTER(PlanCosts),
+                                         ctypes.c_double, _dp, ctypes.POINTER(_u32), _dp]
+for _f in ("zipmoe_plan_hit_distribution", "zipmoe_plan_selection_probs", "zipmoe_plan_makespan",
+           "zipmoe_plan_expected_makespan", "zipmoe_plan_cache_pools"):
+    getattr(_lib, _f).restype = _int
+
+
+def _dbl(a):
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    return a, a.ctypes.data_as(_dp)
+
+
+def _u32x4(v):
+    return (_u32 * 4)(*[int(x) for x in v])
+
+
+def zipmoe_plan_hit_distribution(q):
+    q, qp = _dbl(q)
+    phi = np.zeros(q.size + 1)
+    _check("zipmoe_plan_hit_distribution", _lib.zipmoe_plan_hit_distribution(qp, q.size, phi.ctypes.data_as(_dp)))
+    return phi
+
+
+def zipmoe_plan_selection_probs(f, k, max_iters=1000, tol=1e-12):
+    f, fp = _dbl(f)
+    q = np.zeros(f.size)
+    it = _u32(0)
+    _check("zipmoe_plan_selection_probs",
+           _lib.zipmoe_plan_selection_probs(fp, f.size, k, max_iters, tol, q.ctypes.data_as(_dp), ctypes.byref(it)))
+    return q, int(it.value)
+
+
+def zipmoe_plan_makespan(k, hits, costs):
+    out = ctypes.c_double(0)
+    _check("zipmoe_plan_makespan", _lib.zipmoe_plan_makespan(k, _u32x4(hits), ctypes.byref(costs), ctypes.byref(out)))
+    return out.value
+
+
+def zipmoe_plan_expected_makespan(q, k, capacity, costs):
+    q, qp = _dbl(q)
+    out = ctypes.c_double(0)
+    _check("zipmoe_plan_expected_makespan",
+           _lib.zipmoe_plan_expected_makespan(qp, q.size, k, _u32x4(capacity), ctypes.byref(costs), ctypes.byref(out)))
+    return out.value
+
+
+def zipmoe_plan_cache_pools(f, k, pool_mask, budget, expert_size, costs, step):
+    """Returns (ratios[4], capacity[4], expected makespan)."""
+    f, fp = _dbl(f)
+    size, sp = _dbl(expert_size)
+    ratios = np.zeros(4)
+    cap = (_u32 * 4)()
+    out = ctypes.c_double(0)
+    _check("zipmoe_plan_cache_pools",
+           _lib.zipmoe_plan_cache_pools(fp, f.size, k, pool_mask, budget, sp, ctypes.byref(costs), step,
+                                        ratios.ctypes.data_as(_dp), cap, ctypes.byref(out)))
+    return ratios, [int(c) for c in cap], out.value
+
+
 def zipmoe_ffn_workspace_bytes(T, k, experts):
     out = _u64(0)
     _check("zipmoe_ffn_workspace_bytes", _lib.zipmoe_ffn_workspace_bytes(T, k, ctypes.byref(experts), ctypes.byref(out)))
