@@ -51,7 +51,8 @@ constexpr int kFfnMaxWarps = ZIPMOE_FFN_WARPS;            // decode warps per CT
 #endif
 constexpr int kGroupWarps = ZIPMOE_FFN_GROUP;            // decode warps whose half-tiles form one operand of M = 8 * kGroupWarps (64 or 128)
 static_assert(kGroupWarps == 8 || kGroupWarps == 16, "M is 64 or 128");
-constexpr int kFfnMaxThreads = (kFfnMaxWarps + kFfnMaxWarps / kGroupWarps + 1) * 32;   // decode, one MMA warp per group, loader
+constexpr int kFfnGroups = (kFfnMaxWarps + kGroupWarps - 1) / kGroupWarps;             // the last group may be incomplete
+constexpr int kFfnMaxThreads = (kFfnMaxWarps + kFfnGroups + 1) * 32;                   // decode, one MMA warp per group, loader
 constexpr uint32_t kBLbo = 144;                          // bytes between the 8x8 cores of a half-tile along K: 128 + 16 of
                                                          // padding, so that the 32 lanes' 16-byte stores spread over all banks
 constexpr uint32_t kBBufBytes = 32 * kBLbo;              // one half-tile: 8 rows x 256 columns
@@ -100,7 +101,7 @@ __host__ __device__ inline void ffn_job_parts(uint64_t job, uint32_t steps, uint
 
 // shared-memory layout: [X stages][per-warp buffers][tables][table scratch][barriers][tmem slot]
 __host__ __device__ inline uint32_t ffn_bar_count(uint32_t n_warps) {
-  return 2 * n_warps + 2 * (n_warps / kGroupWarps) + 4;   // the word after them is the CTA's give-up flag
+  return 2 * n_warps + 2 * ((n_warps + kGroupWarps - 1) / kGroupWarps) + 4;   // the word after them is the CTA's give-up flag
 }
 __host__ __device__ inline uint32_t ffn_smem_bytes(uint32_t n_warps, uint32_t groups, bool lane16) {
   const uint32_t after_warps = (lane16 ? kFfnLutBytes : (uint32_t)kLutBytes) + kLutScratchBytes + ffn_bar_count(n_warps) * 8 + 16;
@@ -147,7 +148,7 @@ template <bool LANE16>
 __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const FfnArgs a) {
   constexpr uint32_t kMyLutBytes = LANE16 ? kFfnLutBytes : kLutBytes;
   extern __shared__ __align__(128) uint8_t smem[];
-  const uint32_t NW = a.n_warps, G = a.groups, Q = NW / kGroupWarps, NCOL = 8 * G;
+  const uint32_t NW = a.n_warps, G = a.groups, Q = (NW + kGroupWarps - 1) / kGroupWarps, NCOL = 8 * G;
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   // ---- this CTA's share of the launch's steps ----
@@ -179,7 +180,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   if (tid == 0) {
     for (uint32_t b = 0; b < 2 * NW; ++b) mbar_init(bar0 + 8 * b, 1);
     for (uint32_t q = 0; q < Q; ++q) {
-      mbar_init(quad_full + 8 * q, kGroupWarps);
+      mbar_init(quad_full + 8 * q, min((uint32_t)kGroupWarps, NW - q * kGroupWarps));   // the group's decode warps
       mbar_init(quad_done + 8 * q, 1);
     }
     mbar_init(x_full, 1);
@@ -200,7 +201,9 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  const bool shape_ok = 2 * Q * NCOL <= 512 && kGroupWarps * Q == NW && steps > 0 && steps <= 64 && a.n_mats > 0 &&
+  // (an incomplete last group: the MMA operand then also covers the bytes after the last warp's buffer, which
+  // are the lookup table's, inside the allocation; the accumulator rows they produce are never read)
+  const bool shape_ok = 2 * Q * NCOL <= 512 && (kGroupWarps * Q - NW) * kFfnWarpBytes <= kMyLutBytes && steps > 0 && steps <= 64 && a.n_mats > 0 &&
                         a.n_groups > 0;
   if (!shape_ok) report(a.la.status, kStatusBadDescriptor);
 
@@ -507,7 +510,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
       // the halves of the group's warps 2j and 2j + 1.
       // With M = 128, D row r sits in lane r: warp j reads rows 32j..32j+31, the halves of warps 4j..4j+3.
       const uint32_t wg = kGroupWarps == 8 ? 2 * warp + ((lane >> 3) & 1) : 4 * warp + (lane >> 3), r = lane & 7;
-      const uint32_t live_lanes = kGroupWarps == 8 ? 16 : 32;
+      const uint32_t live_lanes = kGroupWarps == 8 ? 16 : 32;   // (rows of warps the group does not have are skipped below)
       float *y = a.y + ((size_t)(mat * a.max_parts + part) * a.S + off) * a.rows;
       for (uint32_t q = 0; q < Q; ++q) {
         const uint32_t st = grp * NW + kGroupWarps * q + wg;
@@ -521,7 +524,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
                          : "r"(taddr)
                          : "memory");
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            if (lane < live_lanes && st < n_strips) {
+            if (lane < live_lanes && kGroupWarps * q + wg < NW && st < n_strips) {
 #pragma unroll
               for (uint32_t n = 0; n < 8; ++n) {
                 const uint32_t tokrow = 8 * c + n;
@@ -800,7 +803,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.groups = p.groups;
   a.S = S;
   a.smem_bytes = p.smem;
-  const uint32_t threads = (p.n_warps + p.n_warps / zipmoe_dev::kGroupWarps + 1) * 32;
+  const uint32_t threads = (p.n_warps + (p.n_warps + zipmoe_dev::kGroupWarps - 1) / zipmoe_dev::kGroupWarps + 1) * 32;
   PartsOf po;
   po.active = active;
   po.slot_active = slot_active;
