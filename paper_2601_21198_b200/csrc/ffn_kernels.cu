@@ -615,11 +615,18 @@ struct PartsOf {
 // fp32 [S][I].  grid = (ceil(I / blockDim), S)
 __global__ void swiglu_kernel(const float *gu, const PartsOf po, const uint32_t *expert_offset, uint32_t E, uint32_t S,
                               uint32_t I, uint16_t *h) {
-  const uint32_t slot = blockIdx.y, row = blockIdx.x * blockDim.x + threadIdx.x;
-  if (row >= I || slot >= __ldg(expert_offset + E)) return;
+  // the numbers of partial sums are the same for all rows of a strip group: looked up once for the group of the
+  // block's first row, and again by the threads whose row lies in another group
+  __shared__ uint32_t s_parts[2];
+  const uint32_t slot = blockIdx.y, row0 = blockIdx.x * blockDim.x, row = row0 + threadIdx.x;
+  if (slot >= __ldg(expert_offset + E)) return;
+  if (threadIdx.x < 2) s_parts[threadIdx.x] = po.parts(slot, threadIdx.x, row0);
+  __syncthreads();
+  if (row >= I) return;
+  const bool same = row / po.rows_per_group == row0 / po.rows_per_group;
+  const uint32_t pg = same ? s_parts[0] : po.parts(slot, 0, row), pu = same ? s_parts[1] : po.parts(slot, 1, row);
   const size_t at = (size_t)slot * I + row, block = (size_t)S * I;
   float gv = 0.f, uv = 0.f;
-  const uint32_t pg = po.parts(slot, 0, row), pu = po.parts(slot, 1, row);
   for (uint32_t p = 0; p < pg; ++p) gv += gu[p * block + at];
   for (uint32_t p = 0; p < pu; ++p) uv += gu[(po.max_parts + p) * block + at];
   const float hv = gv / (1.0f + __expf(-gv)) * uv;
@@ -629,19 +636,27 @@ __global__ void swiglu_kernel(const float *gu, const PartsOf po, const uint32_t 
 // out[t] = bf16( sum_j w[t,j] * sum_p y[p][slot_of[t,j]] )
 __global__ void combine_kernel(const float *y, const PartsOf po, const uint32_t *slot_of, const float *topk_weights,
                                uint32_t T, uint32_t k, uint32_t S, uint32_t H, uint16_t *out) {
-  const uint32_t t = blockIdx.y;
-  for (uint32_t c = blockIdx.x * blockDim.x + threadIdx.x; c < H; c += gridDim.x * blockDim.x) {
-    float acc = 0.f;
-    for (uint32_t j = 0; j < k; ++j) {
-      const uint32_t slot = slot_of[t * k + j];
-      if (slot == 0xFFFFFFFFu) continue;
-      float v = 0.f;
-      const uint32_t n = po.parts(slot, 0, c);
-      for (uint32_t p = 0; p < n; ++p) v += y[((size_t)p * S + slot) * H + c];
-      acc += (topk_weights ? topk_weights[t * k + j] : 1.0f) * v;
-    }
-    out[(size_t)t * H + c] = __bfloat16_as_ushort(__float2bfloat16_rn(acc));
+  // grid = (ceil(H / blockDim), T); the numbers of partial sums of the token's k slots, for the strip group of the
+  // block's first column, are looked up once per block
+  __shared__ uint32_t s_parts[8];
+  const uint32_t t = blockIdx.y, c0 = blockIdx.x * blockDim.x, c = c0 + threadIdx.x;
+  if (threadIdx.x < k && threadIdx.x < 8) {
+    const uint32_t slot = slot_of[t * k + threadIdx.x];
+    s_parts[threadIdx.x] = slot == 0xFFFFFFFFu ? 0u : po.parts(slot, 0, c0);
   }
+  __syncthreads();
+  if (c >= H) return;
+  const bool same = c / po.rows_per_group == c0 / po.rows_per_group;
+  float acc = 0.f;
+  for (uint32_t j = 0; j < k; ++j) {
+    const uint32_t slot = slot_of[t * k + j];
+    if (slot == 0xFFFFFFFFu) continue;
+    float v = 0.f;
+    const uint32_t n = (same && j < 8) ? s_parts[j] : po.parts(slot, 0, c);
+    for (uint32_t p = 0; p < n; ++p) v += y[((size_t)p * S + slot) * H + c];
+    acc += (topk_weights ? topk_weights[t * k + j] : 1.0f) * v;
+  }
+  out[(size_t)t * H + c] = __bfloat16_as_ushort(__float2bfloat16_rn(acc));
 }
 
 }  // namespace zipmoe_dev
