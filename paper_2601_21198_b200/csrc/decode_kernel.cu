@@ -119,7 +119,54 @@ struct GlobalSink {
   }
 };
 
-template <bool WIDE>
+// A resolved tile in five words, so that the 32 lanes of a warp can each resolve one of the warp's next 32 tiles at
+// once and hand them out by shuffle: resolving a tile costs a warp ~100 instructions, fetching a resolved one ~15.
+//   rec16  : record, 16-byte units from `payload`;  sm16 : sign+mantissa bytes, 16-byte units from `sm`;
+//   out8   : first element, 8-element units from `out`;  pitch;
+//   bits   : valid (13 bits) | iterations << 13 (5) | record size in 16-byte units << 18 (10) | staged << 30 | ok << 31
+struct PackedTile {
+  uint32_t rec16, sm16, out8, pitch, bits;
+};
+__device__ __forceinline__ PackedTile pack_tile(const LaunchArgs &a, const TileWork &w) {
+  PackedTile p = {0, 0, 0, 0, 0};
+  if (!w.ok) return p;
+  const uint64_t r = (uint64_t)(w.rec - a.payload) >> 4, s = (uint64_t)(w.sm - a.sm) >> 4;
+  const uint64_t o = (uint64_t)(w.out - a.out) >> 3;
+  if ((r | s | o) >> 32) return p;   // beyond what the packed form addresses (64 GB of input, 32 G elements of output)
+  p.rec16 = (uint32_t)r;
+  p.sm16 = (uint32_t)s;
+  p.out8 = (uint32_t)o;
+  p.pitch = w.pitch;
+  p.bits = w.valid | (w.iters << 13) | ((w.rec_bytes >> 4) << 18) | ((w.staged ? 1u : 0u) << 30) | (1u << 31);
+  return p;
+}
+// lane `src`'s packed tile, unpacked in every lane
+__device__ __forceinline__ TileWork fetch_tile(const LaunchArgs &a, const PackedTile &mine, uint32_t src) {
+  // a warp-wide OR over "lane src's word, zero elsewhere" instead of a shuffle: the result of a warp reduction is
+  // known to be the same in every lane, so the tile's addresses and sizes live in uniform registers
+  const bool me = (threadIdx.x & 31u) == src;
+  const uint32_t bits = __reduce_or_sync(0xFFFFFFFFu, me ? mine.bits : 0u);
+  const uint32_t rec16 = __reduce_or_sync(0xFFFFFFFFu, me ? mine.rec16 : 0u);
+  const uint32_t sm16 = __reduce_or_sync(0xFFFFFFFFu, me ? mine.sm16 : 0u);
+  const uint32_t out8 = __reduce_or_sync(0xFFFFFFFFu, me ? mine.out8 : 0u);
+  TileWork w;
+  w.pitch = __reduce_or_sync(0xFFFFFFFFu, me ? mine.pitch : 0u);
+  w.ok = bits >> 31;
+  w.staged = (bits >> 30) & 1u;
+  w.valid = bits & 0x1FFFu;
+  w.iters = (bits >> 13) & 31u;
+  w.pieces = (w.iters + kPieceIters - 1) / kPieceIters;
+  w.rec_bytes = ((bits >> 18) & 0x3FFu) << 4;
+  w.rec = a.payload + ((size_t)rec16 << 4);
+  w.sm = a.sm + ((size_t)sm16 << 4);
+  w.out = a.out + ((size_t)out8 << 3);
+  return w;
+}
+
+// BATCHED: tiles are resolved 32 at a time, one per lane, instead of one by one by the whole warp.  That pays when
+// tiles are small or tensors many; with few large tensors of full tiles the one-by-one form keeps the hot loop leaner
+// and is 3 % faster.  The host picks by the launch's tiles per tensor.
+template <bool WIDE, bool BATCHED>
 __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) decode_kernel(const LaunchArgs a) {
   constexpr int kWarps = Cfg<WIDE>::kWarps, kThreads = Cfg<WIDE>::kThreads, kWarpBytes = Cfg<WIDE>::kWarpBytes;
   constexpr uint32_t kBuf = Cfg<WIDE>::kBuf;
@@ -167,24 +214,36 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
     uint32_t g = g0 + warp * share;
     const uint32_t g_end = min(seg_end, g + share);
     uint32_t stage = 0;
-    // descriptor and tile-in-chunk of this warp's next tile, stepped without divisions
-    uint32_t tc = 0, tt = 0;
+    constexpr bool batched = BATCHED;
+    uint32_t tc = 0, tt = 0;   // descriptor and tile-in-chunk of this warp's next tile, stepped without divisions
     if (g < g_end) {
       tc = run_first_chunk + (g - run_first_tile) / tpc;
       tt = (g - run_first_tile) % tpc;
     }
-    auto step = [&]() {
-      if (++tt == tpc) {
-        tt = 0;
-        ++tc;
+    // Lane L resolves tile `first + L` of the warp's share: descriptor, tile-table entry and every bounds check
+    // for 32 tiles at the price of one.  (An unresolvable tile comes back with ok = false.)
+    auto resolve_batch = [&](uint32_t first) -> PackedTile {
+      TileWork w;
+      w.ok = false;
+      const uint32_t mine = first + lane;
+      if (mine < g_end) {
+        const uint32_t rel = mine - run_first_tile;
+        w = resolve_tile(a, run_first_chunk + rel / tpc, rel % tpc, kBuf);
       }
+      return pack_tile(a, w);
     };
     // the warp's first tile of the segment is fetched while the table is being built (its own stages and
     // slots are free: it has finished its tiles of the previous segment)
+    PackedTile batch = {0, 0, 0, 0, 0};
     TileWork cur;
     cur.ok = false;
     if (g < g_end && !dead) {
-      cur = resolve_tile(a, tc, tt, kBuf);
+      if (batched) {
+        batch = resolve_batch(g);
+        cur = fetch_tile(a, batch, 0);
+      } else {
+        cur = resolve_tile(a, tc, tt, kBuf);
+      }
       if (!cur.ok) report(a.status, kStatusBadDescriptor);
       else {
         pipe.load_record(cur, stage);
@@ -195,13 +254,24 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
     const bool fast = build_lut(kThreads, a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <=
                       (uint32_t)kLaneLutBits;
 
-    for (; g < g_end && !dead; ++g) {
+    for (uint32_t in_batch = 0; g < g_end && !dead; ++g) {
       TileWork nxt;
       nxt.ok = false;
       uint32_t nxt_issued = 0;
       if (g + 1 < g_end) {
-        step();
-        nxt = resolve_tile(a, tc, tt, kBuf);
+        if (batched) {
+          if (++in_batch == 32) {   // the batch is used up (the current tile was fetched from it one step ago)
+            batch = resolve_batch(g + 1);
+            in_batch = 0;
+          }
+          nxt = fetch_tile(a, batch, in_batch);
+        } else {
+          if (++tt == tpc) {
+            tt = 0;
+            ++tc;
+          }
+          nxt = resolve_tile(a, tc, tt, kBuf);
+        }
         if (!nxt.ok) report(a.status, kStatusBadDescriptor);
       }
       // the next record is fetched while this one is decoded
@@ -275,10 +345,12 @@ zipmoe_status prepare_device(int *sm_count) {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ZIPMOE_ERR_CUDA;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ZIPMOE_ERR_CUDA;
     if (major != 10) return ZIPMOE_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(zipmoe_dev::decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             zipmoe_dev::Cfg<true>::kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(zipmoe_dev::decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             zipmoe_dev::Cfg<false>::kSmemBytes) != cudaSuccess)
+    using namespace zipmoe_dev;
+    const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    if (cudaFuncSetAttribute(decode_kernel<true, true>, at, Cfg<true>::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_kernel<true, false>, at, Cfg<true>::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_kernel<false, true>, at, Cfg<false>::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_kernel<false, false>, at, Cfg<false>::kSmemBytes) != cudaSuccess)
       return ZIPMOE_ERR_CUDA;
     g_dev[dev].sm_count = sms;
     g_dev[dev].ready = true;
@@ -325,9 +397,11 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   using Narrow = zipmoe_dev::Cfg<false>;
   using Wide = zipmoe_dev::Cfg<true>;
-  if (narrow)
-    zipmoe_dev::decode_kernel<false><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
-  else
-    zipmoe_dev::decode_kernel<true><<<ctas, Wide::kThreads, Wide::kSmemBytes, st>>>(a);
+  // few large tensors (at least 512 tiles each on average): tiles resolved one by one; else 32 at a time
+  const bool batched = (uint64_t)n_tiles < 512ull * n_tables;
+  if (narrow && batched) zipmoe_dev::decode_kernel<false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
+  else if (narrow) zipmoe_dev::decode_kernel<false, false><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
+  else if (batched) zipmoe_dev::decode_kernel<true, true><<<ctas, Wide::kThreads, Wide::kSmemBytes, st>>>(a);
+  else zipmoe_dev::decode_kernel<true, false><<<ctas, Wide::kThreads, Wide::kSmemBytes, st>>>(a);
   return cudaGetLastError() == cudaSuccess ? ZIPMOE_OK : ZIPMOE_ERR_CUDA;
 }
