@@ -167,8 +167,13 @@ zipmoe_status zipmoe_blob_plan(const void *blob, uint64_t blob_bytes, uint64_t p
  * n_tiles   : total tiles of the launch (sum of chunks[].n_tiles).
  * max_record_bytes : the largest chunks[].max_record_bytes of the launch, or 0 if unknown.  A host-side hint
  *             only: when no record exceeds 2048 bytes (every tensor but near-incompressible ones) a kernel
- *             variant without the handling of longer records runs, about 3 % faster.  A wrong hint costs
+ *             variant with smaller record stages and one more warp runs, about 3 % faster.  A wrong hint costs
  *             speed, never correctness.
+ * Work distribution: launches of few large tensors (n_tiles >= 512 * n_tables) give every CTA an equal range of
+ *             tiles; all others hand the tiles out dynamically through a 4-byte counter.  The counters are a
+ *             ring of 1024 words in the library's own device memory (nothing is allocated); a launch zeroes
+ *             its word on `stream` before the kernel (one cudaMemsetAsync).  More than 1024 such launches in
+ *             flight at once on one device would share counters: do not queue that many without synchronising.
  * All device pointers 16-byte aligned.  Errors found on the host (null or
  * misaligned pointers, zero table count with non-zero chunks) are returned
  * before anything is launched. */

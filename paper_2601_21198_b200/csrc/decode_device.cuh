@@ -220,6 +220,7 @@ struct LaunchArgs {
   uint32_t *status;
   uint64_t payload_bytes, sm_bytes, out_elems;
   uint32_t n_chunks, n_tiles, n_tables, tiles_per_cta;
+  uint32_t *work_counter;   // zeroed before the launch: next tile not yet handed to a CTA (dynamic distribution only)
 };
 
 // Which descriptor holds global tile g: exact guess for launches whose chunks
@@ -241,7 +242,8 @@ static_assert(sizeof(zipmoe_chunk_desc) == 80, "descriptor is read as five 16-by
 
 // Everything the decoder needs about tile t of descriptor c, with every offset
 // checked against the sizes of the buffers the launch was given.
-__device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_t t, const uint32_t stage_buf) {
+__device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c, uint32_t t, const uint32_t stage_buf,
+                                                 const uint32_t table_id) {
   TileWork w;
   w.ok = false;
   w.staged = false;
@@ -251,7 +253,7 @@ __device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c
   const uint64_t pay_off = ((uint64_t)d0.y << 32) | d0.x, sm_off = ((uint64_t)d0.w << 32) | d0.z;
   const uint64_t out_off = ((uint64_t)d1.y << 32) | d1.x;
   const uint32_t pitch = d1.z, tpr = d1.w, tile0 = d2.x, m = d2.y, tile_elems = d2.z, last = d2.w;
-  (void)d3;
+  if (d3.x != table_id) return w;   // every chunk of a run names the run's table
   if (t >= m || tpr == 0 || tile_elems == 0 || tile_elems > ZIPMOE_TILE_ELEMS_MAX || (tile_elems & 255) ||
       last == 0 || last > tile_elems || ((pitch & 7) | (pay_off & 15) | (sm_off & 15) | (out_off & 7)))
     return w;

@@ -18,6 +18,7 @@
 //                      512 contiguous bytes per iteration.
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdint>
 #include <type_traits>
 
@@ -178,8 +179,9 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
 
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint32_t g0 = blockIdx.x * a.tiles_per_cta;
-  const uint32_t g1 = min(g0 + a.tiles_per_cta, a.n_tiles);
-  if (g0 >= g1) return;
+  uint32_t g1 = min(g0 + a.tiles_per_cta, a.n_tiles);
+  if (!BATCHED && g0 >= g1) return;
+  __shared__ uint32_t s_grab[2];   // BATCHED: the range of tiles the CTA took last
 
   WarpPipe pipe;
   pipe.pay_addr = smem_addr(warp_base + warp * kWarpBytes);
@@ -196,6 +198,28 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
   __syncthreads();
 
   bool dead = false;    // this warp gave up after a wait ran out
+  uint32_t lut_table = 0xFFFFFFFFu;   // BATCHED: the table in shared memory
+  bool fast = true;
+  // BATCHED: the launch's tiles are handed out dynamically, in ranges that shrink as the work runs out (half of what
+  // an even split of the rest would give, at least kMinGrab tiles), because tiles and tensors of such launches differ
+  // too much in cost for equal shares to finish together.  Otherwise the CTA has its one fixed range.
+  constexpr uint32_t kMinGrab = 4 * kWarps;
+  for (;;) {
+  if (BATCHED) {
+    __syncthreads();   // s_grab of the previous round has been read by every thread
+    if (tid == 0) {
+      const uint32_t seen = *reinterpret_cast<volatile uint32_t *>(a.work_counter);
+      uint32_t take = seen < a.n_tiles ? (a.n_tiles - seen) / (2 * gridDim.x) : 0;
+      take = max(take, kMinGrab);
+      const uint32_t first = atomicAdd(a.work_counter, take);
+      s_grab[0] = first;
+      s_grab[1] = first < a.n_tiles ? min(a.n_tiles - first, take) + first : first;
+    }
+    __syncthreads();
+    g0 = s_grab[0];
+    g1 = s_grab[1];
+    if (g0 >= g1) break;
+  }
   uint32_t c = find_chunk(a, g0);
 
   while (g0 < g1) {
@@ -228,7 +252,7 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
       const uint32_t mine = first + lane;
       if (mine < g_end) {
         const uint32_t rel = mine - run_first_tile;
-        w = resolve_tile(a, run_first_chunk + rel / tpc, rel % tpc, kBuf);
+        w = resolve_tile(a, run_first_chunk + rel / tpc, rel % tpc, kBuf, table_id);
       }
       return pack_tile(a, w);
     };
@@ -242,7 +266,7 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
         batch = resolve_batch(g);
         cur = fetch_tile(a, batch, 0);
       } else {
-        cur = resolve_tile(a, tc, tt, kBuf);
+        cur = resolve_tile(a, tc, tt, kBuf, table_id);
       }
       if (!cur.ok) report(a.status, kStatusBadDescriptor);
       else {
@@ -250,9 +274,11 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
         for (uint32_t p = 0; p < cur.pieces; ++p) pipe.load_sm_piece(cur, p);
       }
     }
-    __syncthreads();  // every warp is done with the previous table
-    const bool fast = build_lut(kThreads, a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <=
-                      (uint32_t)kLaneLutBits;
+    if (!BATCHED || table_id != lut_table) {
+      __syncthreads();  // every warp is done with the previous table
+      fast = build_lut(kThreads, a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <= (uint32_t)kLaneLutBits;
+      lut_table = table_id;
+    }
 
     for (uint32_t in_batch = 0; g < g_end && !dead; ++g) {
       TileWork nxt;
@@ -270,7 +296,7 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
             tt = 0;
             ++tc;
           }
-          nxt = resolve_tile(a, tc, tt, kBuf);
+          nxt = resolve_tile(a, tc, tt, kBuf, table_id);
         }
         if (!nxt.ok) report(a.status, kStatusBadDescriptor);
       }
@@ -326,18 +352,28 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
       break;
     }
   }
+  if (!BATCHED) break;
+  }
 }
 
 }  // namespace zipmoe_dev
 
 namespace {
+// Work counters of the dynamically distributed launches: a small ring in the library's own device memory, one
+// word per launch, zeroed on the launch's stream right before the kernel.  A slot comes round again after
+// kCounterSlots launches of that kind; by then the launch that had it has long finished.
+constexpr uint32_t kCounterSlots = 1024;
+static __device__ uint32_t g_work_counters[kCounterSlots];
+std::atomic<uint32_t> g_next_slot{0};
+
 struct DeviceInfo {
   int sm_count = 0;
   bool ready = false;
+  uint32_t *counters = nullptr;   // device address of g_work_counters on this device
 };
 DeviceInfo g_dev[64];
 
-zipmoe_status prepare_device(int *sm_count) {
+zipmoe_status prepare_device(int *sm_count, uint32_t **counters) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ZIPMOE_ERR_CUDA;
   if (!g_dev[dev].ready) {
@@ -352,10 +388,14 @@ zipmoe_status prepare_device(int *sm_count) {
         cudaFuncSetAttribute(decode_kernel<false, true>, at, Cfg<false>::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(decode_kernel<false, false>, at, Cfg<false>::kSmemBytes) != cudaSuccess)
       return ZIPMOE_ERR_CUDA;
+    void *ptr = nullptr;   // (in host code the array's name is not a device address: ask for it)
+    if (cudaGetSymbolAddress(&ptr, g_work_counters) != cudaSuccess || !ptr) return ZIPMOE_ERR_CUDA;
+    g_dev[dev].counters = static_cast<uint32_t *>(ptr);
     g_dev[dev].sm_count = sms;
     g_dev[dev].ready = true;
   }
   *sm_count = g_dev[dev].sm_count;
+  *counters = g_dev[dev].counters;
   return ZIPMOE_OK;
 }
 }  // namespace
@@ -372,7 +412,8 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
     return ZIPMOE_ERR_INVALID_ARG;
   if (status_word && (reinterpret_cast<uintptr_t>(status_word) & 3)) return ZIPMOE_ERR_INVALID_ARG;
   int sms = 0;
-  zipmoe_status rc = prepare_device(&sms);
+  uint32_t *counters = nullptr;
+  zipmoe_status rc = prepare_device(&sms, &counters);
   if (rc != ZIPMOE_OK) return rc;
 
   zipmoe_dev::LaunchArgs a;
@@ -397,8 +438,17 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   using Narrow = zipmoe_dev::Cfg<false>;
   using Wide = zipmoe_dev::Cfg<true>;
-  // few large tensors (at least 512 tiles each on average): tiles resolved one by one; else 32 at a time
+  // few large tensors (at least 512 tiles each on average): tiles resolved one by one, an equal range of tiles per
+  // CTA; else tiles resolved 32 at a time and handed to the CTAs dynamically (one CTA per SM either way)
   const bool batched = (uint64_t)n_tiles < 512ull * n_tables;
+  a.work_counter = nullptr;
+  if (batched) {
+    a.work_counter = counters + (g_next_slot.fetch_add(1) % kCounterSlots);
+    if (cudaMemsetAsync(a.work_counter, 0, sizeof(uint32_t), st) != cudaSuccess) return ZIPMOE_ERR_CUDA;
+    ctas = (uint32_t)sms * (narrow ? zipmoe_dev::Cfg<false>::kCtasPerSm : 1u);
+    const uint32_t most = (n_tiles + 4 * 15 - 1) / (4 * 15);   // no more CTAs than smallest grabs
+    if (ctas > most) ctas = most;
+  }
   if (narrow && batched) zipmoe_dev::decode_kernel<false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
   else if (narrow) zipmoe_dev::decode_kernel<false, false><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
   else if (batched) zipmoe_dev::decode_kernel<true, true><<<ctas, Wide::kThreads, Wide::kSmemBytes, st>>>(a);

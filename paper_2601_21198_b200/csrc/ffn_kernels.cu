@@ -811,6 +811,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.la.n_tiles = 0;
   a.la.n_tables = ex->n_tables;
   a.la.tiles_per_cta = 0;
+  a.la.work_counter = nullptr;
   a.tensor_first_chunk = ex->tensor_first_chunk;
   a.expert_offset = expert_offset;
   a.active = active;
