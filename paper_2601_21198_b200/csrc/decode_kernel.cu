@@ -201,15 +201,21 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
   uint32_t lut_table = 0xFFFFFFFFu;   // BATCHED: the table in shared memory
   bool fast = true;
   // BATCHED: the launch's tiles are handed out dynamically, in ranges that shrink as the work runs out (half of what
-  // an even split of the rest would give, at least kMinGrab tiles), because tiles and tensors of such launches differ
+  // an even split of the rest would give, at least kMinGrab tiles: measured best among halves, thirds, quarters and minima of 1..32 tiles per warp), because tiles and tensors of such launches differ
   // too much in cost for equal shares to finish together.  Otherwise the CTA has its one fixed range.
-  constexpr uint32_t kMinGrab = 4 * kWarps;
+#ifndef ZIPMOE_GRAB_MIN
+#define ZIPMOE_GRAB_MIN 8
+#endif
+#ifndef ZIPMOE_GRAB_DIV
+#define ZIPMOE_GRAB_DIV 2
+#endif
+  constexpr uint32_t kMinGrab = ZIPMOE_GRAB_MIN * kWarps;
   for (;;) {
   if (BATCHED) {
     __syncthreads();   // s_grab of the previous round has been read by every thread
     if (tid == 0) {
       const uint32_t seen = *reinterpret_cast<volatile uint32_t *>(a.work_counter);
-      uint32_t take = seen < a.n_tiles ? (a.n_tiles - seen) / (2 * gridDim.x) : 0;
+      uint32_t take = seen < a.n_tiles ? (a.n_tiles - seen) / (ZIPMOE_GRAB_DIV * gridDim.x) : 0;
       take = max(take, kMinGrab);
       const uint32_t first = atomicAdd(a.work_counter, take);
       s_grab[0] = first;
@@ -446,7 +452,7 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
     a.work_counter = counters + (g_next_slot.fetch_add(1) % kCounterSlots);
     if (cudaMemsetAsync(a.work_counter, 0, sizeof(uint32_t), st) != cudaSuccess) return ZIPMOE_ERR_CUDA;
     ctas = (uint32_t)sms * (narrow ? zipmoe_dev::Cfg<false>::kCtasPerSm : 1u);
-    const uint32_t most = (n_tiles + 4 * 15 - 1) / (4 * 15);   // no more CTAs than smallest grabs
+    const uint32_t most = (n_tiles + 8 * 15 - 1) / (8 * 15);   // no more CTAs than smallest grabs
     if (ctas > most) ctas = most;
   }
   if (narrow && batched) zipmoe_dev::decode_kernel<false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
