@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
     if (tid == 0) {
       const uint32_t seen = *reinterpret_cast<volatile uint32_t *>(a.work_counter);
       uint32_t take = seen < a.n_tiles ? (a.n_tiles - seen) / (ZIPMOE_GRAB_DIV * gridDim.x) : 0;
-      take = max(take, kMinGrab);
+      take = max(take, max(1u, min(kMinGrab, a.n_tiles / gridDim.x)));   // small launches: spread over all CTAs
       const uint32_t first = atomicAdd(a.work_counter, take);
       s_grab[0] = first;
       s_grab[1] = first < a.n_tiles ? min(a.n_tiles - first, take) + first : first;
@@ -452,7 +452,7 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
     a.work_counter = counters + (g_next_slot.fetch_add(1) % kCounterSlots);
     if (cudaMemsetAsync(a.work_counter, 0, sizeof(uint32_t), st) != cudaSuccess) return ZIPMOE_ERR_CUDA;
     ctas = (uint32_t)sms * (narrow ? zipmoe_dev::Cfg<false>::kCtasPerSm : 1u);
-    const uint32_t most = (n_tiles + 8 * 15 - 1) / (8 * 15);   // no more CTAs than smallest grabs
+    const uint32_t most = (n_tiles + 15 - 1) / 15;   // a tile per warp at least
     if (ctas > most) ctas = most;
   }
   if (narrow && batched) zipmoe_dev::decode_kernel<false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
