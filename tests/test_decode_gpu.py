@@ -129,6 +129,34 @@ def test_stress_set_sample(zb):
         assert np.array_equal(got[i], codec.decode(blobs[i]))
 
 
+def test_dynamic_distribution_many_launches_in_a_row(zb):
+    """Launches of small or many tensors hand their tiles out through a work counter taken from a ring of 1024 in
+    the library's device memory: more launches than the ring has slots, two plans alternating on two streams, every
+    output bit-exact at the end and on the way."""
+    import torch
+    xs = [inputs.stress_tensor(i, max_elems=1 << 17)[0] for i in (0, 1, 5, 9, 12)]          # a few tiles to ~30 each
+    plans = [zb.DecodePlan([zb.zipmoe_encode(x, chunk_elems=c) for x in xs]) for c in (1024, 16384)]
+    assert all(p.n_tiles < 512 * p.n_tables for p in plans)                                 # dynamically distributed
+    devs = [p.to_device() for p in plans]
+    outs = [d.new_output() for d in devs]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    want = np.concatenate(xs)
+    torch.cuda.synchronize()
+    for it in range(1100):
+        k = it & 1
+        with torch.cuda.stream(streams[k]):
+            if it % 97 == 0:
+                outs[k].fill_(0x5555)
+            devs[k].decode(outs[k], stream=streams[k])
+        if it % 97 == 1 or it == 1099:
+            torch.cuda.synchronize()
+            for d, o, p in zip(devs, outs, plans):
+                assert int(d.status.item()) == 0
+                host = o.cpu().numpy().view(np.uint16)
+                got = np.concatenate([p.tensor_slice(host, i) for i in range(len(xs))])
+                assert np.array_equal(got, want), it
+
+
 def test_empty_launch_and_bad_arguments(zb):
     import torch
     zb.zipmoe_decode(None, 0, 0, None, 0, None, 0, None, 0, None, 0)       # nothing to do: OK
