@@ -330,32 +330,60 @@ def run_ours(args):
     clocks = sampler.summary(t0, t1)
     verified = verified and int(dplan.status.item()) == 0
 
-    # end to end: pinned host -> device, decode, device -> pinned host, every step
-    h_pay = torch.from_numpy(plan.payload).pin_memory()
-    h_sm = torch.from_numpy(plan.sm).pin_memory()
-    h_desc = torch.from_numpy(plan.descs.view(np.uint8).copy()).pin_memory()
-    h_tab = torch.from_numpy(plan.tables).pin_memory()
-    h_out = torch.empty(plan.out_elems, dtype=torch.int16).pin_memory()
+    # end to end: pinned host -> device, decode, device -> pinned host, every step.  The layer is cut into slices of
+    # tensors, each with its own zipmoe_decode call, spread over a few streams, so that one slice's copy to the host
+    # overlaps the next slice's copy to the device (the host link is full duplex) and its decode.
+    n_slices = max(1, min(args.e2e_slices, len(w.blobs)))
+    bounds = [len(w.blobs) * i // n_slices for i in range(n_slices + 1)]
+    slices = []
+    for i in range(n_slices):
+        sp = binding.DecodePlan(w.blobs[bounds[i]:bounds[i + 1]])
+        sd = sp.to_device(dev)
+        slices.append({
+            "plan": sp, "dev": sd, "out": sd.new_output(),
+            "h": [(sd.payload, torch.from_numpy(sp.payload).pin_memory()), (sd.sm, torch.from_numpy(sp.sm).pin_memory()),
+                  (sd.descs, torch.from_numpy(sp.descs.view(np.uint8).copy()).pin_memory()),
+                  (sd.tables, torch.from_numpy(sp.tables).pin_memory())],
+            "h_out": torch.empty(sp.out_elems, dtype=torch.int16).pin_memory()})
+    side = [torch.cuda.Stream(dev) for _ in range(min(3, n_slices))]
+    h2d_bytes = sum(h.numel() * h.element_size() for sl in slices for _, h in sl["h"])
+    d2h_bytes = sum(sl["h_out"].numel() * 2 for sl in slices)
     e2e_steps = max(1, min(args.steps, 10))
 
     def e2e_step():
-        dplan.payload.copy_(h_pay, non_blocking=True)
-        dplan.sm.copy_(h_sm, non_blocking=True)
-        dplan.descs.copy_(h_desc, non_blocking=True)
-        dplan.tables.copy_(h_tab, non_blocking=True)
-        dplan.decode(out)
-        h_out.copy_(out, non_blocking=True)
+        for i, sl in enumerate(slices):
+            st = side[i % len(side)]
+            with torch.cuda.stream(st):
+                for d_t, h_t in sl["h"]:
+                    d_t.copy_(h_t, non_blocking=True)
+                sl["dev"].decode(sl["out"], stream=st)
+                sl["h_out"].copy_(sl["out"], non_blocking=True)
 
-    for _ in range(2):
-        e2e_step()
+    def e2e_run(n):
+        start = torch.cuda.Event(enable_timing=True)
+        end = torch.cuda.Event(enable_timing=True)
+        start.record(stream)
+        for st in side:
+            st.wait_event(start)
+        for _ in range(n):
+            e2e_step()
+        for st in side:
+            done = torch.cuda.Event()
+            done.record(st)
+            stream.wait_event(done)
+        end.record(stream)
+        return start, end
+
+    e2e_run(2)
     barrier()
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record(stream)
-    for _ in range(e2e_steps):
-        e2e_step()
-    f1.record(stream)
+    f0, f1 = e2e_run(e2e_steps)
     barrier()
     e2e_ms = f0.elapsed_time(f1)
+    e2e_ok = all(int(sl["dev"].status.item()) == 0 for sl in slices)
+    if probe is not None:      # the first tensor of the first slice, as it arrived on the host
+        e2e_ok = e2e_ok and bool(np.array_equal(slices[0]["plan"].tensor_slice(slices[0]["h_out"].numpy().view(np.uint16), 0),
+                                                probe.ravel()))
+    verified = verified and e2e_ok
     sampler.stop_flag = True
 
     ms, e2e_ms = max_over_ranks([ms, e2e_ms], dev)
@@ -378,8 +406,8 @@ def run_ours(args):
                        "sharding": "every rank decodes its own copy of the layer; no collective"},
             "clocks": clocks,
             "e2e": {"value": whole_job_gbs(world, bf16_bytes, e2e_steps, e2e_ms), "unit": UNIT,
-                    "h2d_bytes_per_step": int(h_pay.numel() + h_sm.numel() + h_desc.numel() + h_tab.numel()),
-                    "d2h_bytes_per_step": int(h_out.numel() * 2), "steps": e2e_steps},
+                    "h2d_bytes_per_step": int(h2d_bytes), "d2h_bytes_per_step": int(d2h_bytes), "steps": e2e_steps,
+                    "slices": n_slices, "streams": len(side)},
             "gpu_launches": args.steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": achieved / peaks["hbm_gbs"], "traffic": TRAFFIC_BYTES.get(w.label),
@@ -407,6 +435,8 @@ def run_ours(args):
         if world == 1:
             # compression states: one stream stays in pinned host memory and is read in place over PCIe
             states = {}
+            h_pay = torch.from_numpy(plan.payload).pin_memory()
+            h_sm = torch.from_numpy(plan.sm).pin_memory()
             d_pay, d_sm = dplan.payload, dplan.sm
             for name, (pay, smb, moved) in {"sm_chunks_on_host": (d_pay, h_sm, int(h_sm.numel())),
                                             "e_chunks_on_host": (h_pay, d_sm, int(h_pay.numel()))}.items():
@@ -424,7 +454,7 @@ def run_ours(args):
             dplan.payload, dplan.sm = d_pay, d_sm
             line["compression_states"] = states
         if world == 1 and not args.no_ffn:
-            del dplan, out, h_pay, h_sm, h_out
+            del dplan, out, slices, h_pay, h_sm
             torch.cuda.empty_cache()
             line["ffn"] = bench_ffn(dev)
             line["ffn_small_experts"] = bench_ffn(dev, config="small")
@@ -460,6 +490,8 @@ def main():
     ap.add_argument("--ffn-only", type=int, default=0, metavar="T",
                     help="run only the fused expert-FFN section for T tokens (profiling captures)")
     ap.add_argument("--ffn-iters", type=int, default=20)
+    ap.add_argument("--e2e-slices", type=int, default=8,
+                    help="slices of tensors the end-to-end leg pipelines over its streams (1 = one call per step)")
     ap.add_argument("--ffn-config", default="large", choices=["large", "small"],
                     help="expert shapes of --ffn-only: 8 x 4096->14336->4096 top-2, or 64 x 2048->1408->2048 top-6")
     ap.add_argument("--no-ffn", action="store_true", help="skip the fused expert-FFN section of the report")
