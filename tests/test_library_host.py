@@ -120,6 +120,36 @@ def test_bad_arguments_and_corrupt_blobs(zb):
     assert zb.zipmoe_blob_validate(blob[:-1]) == zb.ERR_BAD_FORMAT
 
 
+def test_random_corruptions_are_rejected_or_decode_in_bounds(zb):
+    """Random byte damage anywhere in a blob: the validator either rejects it, or the blob is still structurally
+    sound, in which case the oracle decodes it (to other data) or reports the damage itself -- never a crash.
+    Damage to the header, the code table, the chunk offsets or a tile table must never pass the validator
+    unnoticed when it changes the structure."""
+    from oracle import codec
+    x = inputs.stress_tensor(1, max_elems=30000)[0]
+    blob = zb.zipmoe_encode(x, chunk_elems=1024)
+    info = zb.zipmoe_blob_info_get(blob)
+    rng = np.random.default_rng(17)
+    accepted = rejected = 0
+    for trial in range(400):
+        b = blob.copy()
+        region = trial % 4       # header + table, chunk offsets, payload, anywhere
+        lo, hi = [(0, 320), (320, info.payload_off), (info.payload_off, info.sm_off), (0, b.size)][region]
+        for _ in range(1 + trial % 3):
+            at = int(rng.integers(lo, hi))
+            b[at] ^= np.uint8(1 << int(rng.integers(0, 8)))
+        if zb.zipmoe_blob_validate(b) != zb.OK:
+            rejected += 1
+            continue
+        accepted += 1
+        try:
+            y = codec.decode(b)
+            assert y.size == x.size
+        except ValueError:
+            pass
+    assert accepted > 20 and rejected > 100, (accepted, rejected)
+
+
 def test_plan_descriptors(zb):
     a = inputs.gaussian((5, 4099), 0.02, 3)          # linear, 2 chunks of 16384, short last tile
     b = inputs.gaussian((32, 512), 0.02, 4)          # blocked, 4 tiles, chunks of 8192 (2 tiles)
