@@ -223,17 +223,25 @@ struct LaunchArgs {
   uint32_t *work_counter;   // zeroed before the launch: next tile not yet handed to a CTA (dynamic distribution only)
 };
 
-// Which descriptor holds global tile g: exact guess for launches whose chunks
-// all hold the same number of tiles, binary search on tile_prefix otherwise.
+// Which descriptor holds global tile g: exact guess for launches whose chunks all hold the same number of tiles,
+// else a search on tile_prefix in which the 32 lanes of the warp probe 32 evenly spaced descriptors per step
+// (three or four dependent loads for any launch, where a binary search needs up to seventeen).  Called by whole
+// warps; the result is the same in every lane.
 __device__ inline uint32_t find_chunk(const LaunchArgs &a, uint32_t g) {
   uint32_t c = (uint32_t)(((uint64_t)g * a.n_chunks) / a.n_tiles);
   if (c >= a.n_chunks) c = a.n_chunks - 1;
   uint32_t p = __ldg(&a.chunks[c].tile_prefix), m = __ldg(&a.chunks[c].n_tiles);
   if (g >= p && g - p < m) return c;
-  uint32_t lo = 0, hi = a.n_chunks;  // invariant: prefix[lo] <= g (prefix[0] = 0)
+  const uint32_t lane = threadIdx.x & 31u;
+  uint32_t lo = 0, hi = a.n_chunks;  // invariant: prefix[lo] <= g (prefix[0] = 0), and g < prefix[hi] where hi exists
   while (hi - lo > 1) {
-    uint32_t mid = (lo + hi) >> 1;
-    if (__ldg(&a.chunks[mid].tile_prefix) <= g) lo = mid; else hi = mid;
+    const uint32_t step = (hi - lo + 31) / 32;
+    const uint32_t at = lo + lane * step;
+    const bool below = at < hi && __ldg(&a.chunks[at].tile_prefix) <= g;
+    const uint32_t k = __popc(__ballot_sync(0xFFFFFFFFu, below));   // prefixes ascend: the lanes that are below come first
+    const uint32_t first = lo + (k ? k - 1 : 0) * step;
+    hi = min(hi, first + step);
+    lo = first;
   }
   return lo;
 }
