@@ -149,6 +149,10 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   constexpr uint32_t kMyLutBytes = LANE16 ? kFfnLutBytes : kLutBytes;
   extern __shared__ __align__(128) uint8_t smem[];
   const uint32_t NW = a.n_warps, G = a.groups, Q = (NW + kGroupWarps - 1) / kGroupWarps, NCOL = 8 * G;
+  // accumulator columns per group and half = N of the MMAs: with M = 128, N is a multiple of 16 (for up to 8 token
+  // rows the operand then also covers the 8 rows after the stage's, whose columns come out as garbage and are
+  // never read back)
+  const uint32_t NACC = kGroupWarps == 16 ? (NCOL + 15u) & ~15u : NCOL;
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   // ---- this CTA's share of the launch's steps ----
@@ -176,7 +180,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   const bool is_decode = warp < NW, is_mma = warp >= NW && warp < NW + Q, is_loader = warp == NW + Q;
 
   uint32_t tmem_cols = 32;
-  while (tmem_cols < 2 * Q * NCOL) tmem_cols <<= 1;
+  while (tmem_cols < 2 * Q * NACC) tmem_cols <<= 1;
   if (tid == 0) {
     for (uint32_t b = 0; b < 2 * NW; ++b) mbar_init(bar0 + 8 * b, 1);
     for (uint32_t q = 0; q < Q; ++q) {
@@ -203,7 +207,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
 
   // (an incomplete last group: the MMA operand then also covers the bytes after the last warp's buffer, which
   // are the lookup table's, inside the allocation; the accumulator rows they produce are never read)
-  const bool shape_ok = 2 * Q * NCOL <= 512 && (kGroupWarps * Q - NW) * kFfnWarpBytes <= kMyLutBytes && steps > 0 && steps <= 64 && a.n_mats > 0 &&
+  const bool shape_ok = 2 * Q * NACC <= 512 && (kGroupWarps * Q - NW) * kFfnWarpBytes <= kMyLutBytes && steps > 0 && steps <= 64 && a.n_mats > 0 &&
                         a.n_groups > 0;
   if (!shape_ok) report(a.la.status, kStatusBadDescriptor);
 
@@ -359,7 +363,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
       }
     } else if (is_mma) {
       // ---- one MMA warp per group; one lane issues, per half-tile: D[64 x N] (+)= A[64 x 256] * X[N x 256]^T ----
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (G << 17) | ((uint32_t)(kGroupWarps / 2) << 24);   // bf16 x bf16 -> fp32, N = 8G, M = 8 * kGroupWarps
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((NACC >> 3) << 17) | ((uint32_t)(kGroupWarps / 2) << 24);   // bf16 x bf16 -> fp32, N = NACC, M = 8 * kGroupWarps
       const uint32_t q = warp - NW;
       const uint32_t abuf = smem_addr(warp_raw) + 2 * kPayStage + kGroupWarps * q * kFfnWarpBytes;
       const uint64_t a_desc0 = smem_desc(abuf, kBLbo, kFfnWarpBytes);
@@ -375,7 +379,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
           }
           if (lane == 0) {
             tc_fence_after();
-            const uint32_t d_tmem = tmem + (2 * q + half) * NCOL;
+            const uint32_t d_tmem = tmem + (2 * q + half) * NACC;
             // the K slice j of an operand starts 2 cores further: the start-address field counts 16-byte units
 #pragma unroll
             for (uint32_t j = 0; j < 16; ++j)
@@ -518,7 +522,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
           const uint32_t row = 16 * st + 8 * half + r;
           for (uint32_t c = 0; c < G; ++c) {
             uint32_t v[8];
-            const uint32_t taddr = tmem + ((32 * warp) << 16) + (2 * q + half) * NCOL + 8 * c;
+            const uint32_t taddr = tmem + ((32 * warp) << 16) + (2 * q + half) * NACC + 8 * c;
             asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                          : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
                          : "r"(taddr)
