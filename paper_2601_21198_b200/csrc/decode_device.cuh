@@ -552,7 +552,9 @@ struct LaneDecoder {
 //             linear tensor.
 // Returns 0 on success, else a status code (warp-uniform); on
 // kStatusBadBitCount nothing has been written.
-template <bool STAGED, bool FAST, class Feed, class Sink>
+// SMALL: also an unrolled path for small full tiles (kept out of the instantiation that never sees any: it would
+// only lengthen its code).
+template <bool STAGED, bool FAST, bool SMALL, class Feed, class Sink>
 __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *rec_g, uint32_t rec_bytes,
                                                 uint32_t lut, uint32_t valid, uint32_t iters,
                                                 uint32_t lane, Feed &feed, Sink &sink) {
@@ -561,6 +563,23 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
   static_assert(kPieceIters % 2 == 0, "a piece holds whole pairs of iterations");
 
   const uint32_t pieces = (iters + kPieceIters - 1) / kPieceIters;
+  if (SMALL && valid == iters * 256u && iters < kPieceIters && (iters & 1u) == 0) {
+    // a small full tile (chunks of less than 2048 elements): one piece, a few pairs of iterations
+    const uint32_t sm_s = feed.begin(0);
+    if (sm_s == 0xFFFFFFFFu) return kStatusWaitTimeout;
+    const uint32_t sm_lane = sm_s + lane * 8;
+#pragma unroll
+    for (uint32_t k = 0; k < kPieceIters - 2; k += 2) {
+      if (k < iters) {
+        uint4 o0, o1;
+        dec.group2(lds_v2(sm_lane + k * 256), lds_v2(sm_lane + (k + 1) * 256), o0, o1);
+        sink.group(k, lane, o0);
+        sink.group(k + 1, lane, o1);
+      }
+    }
+    feed.end(0);
+    return 0;
+  }
   if (valid == iters * 256u && (iters % kPieceIters) == 0) {
     // every group exists and pieces are whole: unrolled iterations, addresses are immediates
     for (uint32_t p = 0; p < pieces; ++p) {

@@ -316,14 +316,14 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
           SmFeed feed{pipe, nxt, nxt_issued};
           GlobalSink sink{cur.out, cur.pitch};
           if (cur.staged) {
-            rc = fast ? decode_tile<true, true>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid,
+            rc = fast ? decode_tile<true, true, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid,
                                                   cur.iters, lane, feed, sink)
-                        : decode_tile<true, false>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid,
+                        : decode_tile<true, false, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid,
                                                    cur.iters, lane, feed, sink);
           } else {
-            rc = fast ? decode_tile<false, true>(0, cur.rec, cur.rec_bytes, lut, cur.valid,
+            rc = fast ? decode_tile<false, true, BATCHED>(0, cur.rec, cur.rec_bytes, lut, cur.valid,
                                                    cur.iters, lane, feed, sink)
-                        : decode_tile<false, false>(0, cur.rec, cur.rec_bytes, lut, cur.valid,
+                        : decode_tile<false, false, BATCHED>(0, cur.rec, cur.rec_bytes, lut, cur.valid,
                                                     cur.iters, lane, feed, sink);
           }
         }
