@@ -169,6 +169,11 @@ zipmoe_status zipmoe_blob_plan(const void *blob, uint64_t blob_bytes, uint64_t p
  *             only: when no record exceeds 2048 bytes (every tensor but near-incompressible ones) a kernel
  *             variant with smaller record stages and one more warp runs, about 3 % faster.  A wrong hint costs
  *             speed, never correctness.
+ * flags     : 0, or ZIPMOE_DECODE_SHORT_CODES: the caller promises that no table of the launch has a code longer
+ *             than 8 bits and that max_record_bytes is a true upper bound of at most 2048 (zipmoe_blob_plan's
+ *             descriptors and the blobs' tables say both).  The kernel variant chosen then carries only the common
+ *             path and is 2-3 % faster.  A tile that breaks the promise is not decoded: its output is left as it
+ *             was and status_word is set (code 5), so a false promise is loud, never silent.
  * Work distribution: launches of few large tensors (n_tiles >= 512 * n_tables) give every CTA an equal range of
  *             tiles; all others hand the tiles out dynamically through a 4-byte counter.  The counters are a
  *             ring of 1024 words in the library's own device memory (nothing is allocated); a launch zeroes
@@ -181,7 +186,8 @@ zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t n_chunks, 
                             const zipmoe_table *tables, uint32_t n_tables, const uint8_t *payload,
                             uint64_t payload_bytes, const uint8_t *sm, uint64_t sm_bytes, uint16_t *out_bf16,
                             uint64_t out_elems, uint32_t *status_word, zipmoe_stream stream,
-                            uint32_t max_record_bytes);
+                            uint32_t max_record_bytes, uint32_t flags);
+#define ZIPMOE_DECODE_SHORT_CODES 1u
 
 /* The recovery step alone (Section 3.3, "Memory-Coalesced Tensor Recovery Kernel"): exponent bytes that
  * are already decompressed and sign+mantissa bytes, both in element order, are merged into bf16:

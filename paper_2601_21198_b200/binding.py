@@ -23,6 +23,7 @@ if not os.path.exists(LIB_PATH):
 
 _lib = ctypes.CDLL(LIB_PATH)
 
+DECODE_SHORT_CODES = 1      # zipmoe_decode flag: no code above 8 bits, max_record_bytes exact and <= 2048
 OK = 0
 ERR_INVALID_ARG, ERR_BAD_FORMAT, ERR_BUFFER_TOO_SMALL, ERR_CUDA, ERR_DECODE_CORRUPT, ERR_UNSUPPORTED = -1, -2, -3, -4, -5, -6
 LAYOUT_LINEAR, LAYOUT_BLOCKED = 0, 1
@@ -64,7 +65,7 @@ _lib.zipmoe_encode.argtypes = [_vp, _u64, _u64, ctypes.POINTER(EncodeOpts), _vp,
 _lib.zipmoe_blob_info_get.argtypes = [_vp, _u64, ctypes.POINTER(BlobInfo)]
 _lib.zipmoe_blob_validate.argtypes = [_vp, _u64]
 _lib.zipmoe_blob_plan.argtypes = [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _u32, _vp, _vp]
-_lib.zipmoe_decode.argtypes = [_vp, _u32, _u32, _vp, _u32, _vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp, _u32]
+_lib.zipmoe_decode.argtypes = [_vp, _u32, _u32, _vp, _u32, _vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp, _u32, _u32]
 _lib.zipmoe_recover.argtypes = [_vp, _vp, _u64, _vp, _vp]
 _lib.zipmoe_recover.restype = _int
 _lib.zipmoe_ffn_workspace_bytes.argtypes = [_u32, _u32, ctypes.POINTER(CompressedExperts), ctypes.POINTER(_u64)]
@@ -159,11 +160,11 @@ def zipmoe_blob_plan(blob, payload_base, sm_base, out_base, table_id, chunk_base
 
 
 def zipmoe_decode(chunks, n_chunks, n_tiles, tables, n_tables, payload, payload_bytes, sm, sm_bytes, out_bf16,
-                  out_elems, status_word=None, stream=None, max_record_bytes=0):
+                  out_elems, status_word=None, stream=None, max_record_bytes=0, flags=0):
     """All pointer arguments are device tensors (or raw device addresses)."""
     _check("zipmoe_decode", _lib.zipmoe_decode(_ptr(chunks), n_chunks, n_tiles, _ptr(tables), n_tables, _ptr(payload),
                                                 payload_bytes, _ptr(sm), sm_bytes, _ptr(out_bf16), out_elems,
-                                                _ptr(status_word), _ptr(stream), int(max_record_bytes)))
+                                                _ptr(status_word), _ptr(stream), int(max_record_bytes), int(flags)))
 
 
 def zipmoe_recover(exp, sm, n_elems, out_bf16, stream=None):
@@ -302,6 +303,9 @@ class DecodePlan:
         self.tables = np.concatenate(tables) if tables else np.zeros(0, np.uint8)
         self.n_chunks, self.n_tiles, self.n_tables = chunk_base, tile_base, len(blobs)
         self.max_record_bytes = int(self.descs["max_record_bytes"].max()) if self.n_chunks else 0
+        # what the fastest kernel variant wants promised: no code longer than 8 bits, no record longer than 2048 bytes
+        self.max_code_len = int(self.tables.max()) if self.tables.size else 0
+        self.flags = DECODE_SHORT_CODES if (0 < self.max_record_bytes <= 2048 and self.max_code_len <= 8) else 0
 
     def algorithmic_bytes(self):
         """Bytes one decode must move: E-chunk section + SM bytes read, bf16 written."""
@@ -340,7 +344,7 @@ class DevicePlan:
         p = self.plan
         s = torch.cuda.current_stream(self.device) if stream is None else stream
         zipmoe_decode(self.descs, p.n_chunks, p.n_tiles, self.tables, p.n_tables, self.payload, p.payload_bytes,
-                      self.sm, p.sm_bytes, out, p.out_elems, self.status, s.cuda_stream, p.max_record_bytes)
+                      self.sm, p.sm_bytes, out, p.out_elems, self.status, s.cuda_stream, p.max_record_bytes, p.flags)
 
 
 def pad_expert_inter(w1, w3, w2, multiple=256):

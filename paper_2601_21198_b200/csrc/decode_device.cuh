@@ -31,6 +31,7 @@ constexpr uint32_t kStatusBadDescriptor = 1;  // a descriptor, offset or table p
 constexpr uint32_t kStatusBadBitCount = 2;    // a tile's lane bit counts overrun its record
 constexpr uint32_t kStatusWaitTimeout = 3;    // an asynchronous copy did not complete in time
 constexpr uint32_t kStatusBadTable = 4;       // code lengths do not form a complete prefix code
+constexpr uint32_t kStatusBrokenPromise = 5;  // ZIPMOE_DECODE_SHORT_CODES was given, yet a tile has longer codes or a longer record
 
 constexpr uint32_t kPieceIters = 8;           // iterations served by one piece of sign+mantissa bytes
 constexpr uint32_t kSmPieceBytes = kPieceIters * 256;

@@ -167,7 +167,10 @@ __device__ __forceinline__ TileWork fetch_tile(const LaunchArgs &a, const Packed
 // BATCHED: tiles are resolved 32 at a time, one per lane, instead of one by one by the whole warp.  That pays when
 // tiles are small or tensors many; with few large tensors of full tiles the one-by-one form keeps the hot loop leaner
 // and is 3 % faster.  The host picks by the launch's tiles per tensor.
-template <bool WIDE, bool BATCHED>
+// LEAN: only the common path is compiled in -- record staged in shared memory, codes of at most 8 bits -- on the
+// caller's promise (ZIPMOE_DECODE_SHORT_CODES) that the launch has nothing else; a tile that does is reported and
+// left undecoded.  The shorter code is worth 2-3 %.
+template <bool WIDE, bool BATCHED, bool LEAN = false>
 __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) decode_kernel(const LaunchArgs a) {
   constexpr int kWarps = Cfg<WIDE>::kWarps, kThreads = Cfg<WIDE>::kThreads, kWarpBytes = Cfg<WIDE>::kWarpBytes;
   constexpr uint32_t kBuf = Cfg<WIDE>::kBuf;
@@ -315,7 +318,11 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
           const uint32_t rec_s = pipe.pay_addr + stage * pipe.stage_bytes;
           SmFeed feed{pipe, nxt, nxt_issued};
           GlobalSink sink{cur.out, cur.pitch};
-          if (cur.staged) {
+          if (LEAN) {
+            rc = (cur.staged && fast) ? decode_tile<true, true, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid,
+                                                                        cur.iters, lane, feed, sink)
+                                      : kStatusBrokenPromise;
+          } else if (cur.staged) {
             rc = fast ? decode_tile<true, true, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid,
                                                   cur.iters, lane, feed, sink)
                         : decode_tile<true, false, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid,
@@ -333,7 +340,7 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
           dead = true;
           break;
         }
-        if (rc == kStatusBadBitCount) {
+        if (rc == kStatusBadBitCount || rc == kStatusBrokenPromise) {
           // nothing was decoded: take the tile's sign+mantissa pieces off the barriers
           report(a.status, rc);
           for (uint32_t p = 0; p < cur.pieces && !dead; ++p)
@@ -392,7 +399,9 @@ zipmoe_status prepare_device(int *sm_count, uint32_t **counters) {
     if (cudaFuncSetAttribute(decode_kernel<true, true>, at, Cfg<true>::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(decode_kernel<true, false>, at, Cfg<true>::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(decode_kernel<false, true>, at, Cfg<false>::kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(decode_kernel<false, false>, at, Cfg<false>::kSmemBytes) != cudaSuccess)
+        cudaFuncSetAttribute(decode_kernel<false, false>, at, Cfg<false>::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_kernel<false, true, true>, at, Cfg<false>::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_kernel<false, false, true>, at, Cfg<false>::kSmemBytes) != cudaSuccess)
       return ZIPMOE_ERR_CUDA;
     void *ptr = nullptr;   // (in host code the array's name is not a device address: ask for it)
     if (cudaGetSymbolAddress(&ptr, g_work_counters) != cudaSuccess || !ptr) return ZIPMOE_ERR_CUDA;
@@ -410,7 +419,7 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
                                        const zipmoe_table *tables, uint32_t n_tables, const uint8_t *payload,
                                        uint64_t payload_bytes, const uint8_t *sm, uint64_t sm_bytes,
                                        uint16_t *out_bf16, uint64_t out_elems, uint32_t *status_word,
-                                       zipmoe_stream stream, uint32_t max_record_bytes) {
+                                       zipmoe_stream stream, uint32_t max_record_bytes, uint32_t flags) {
   if (n_chunks == 0 || n_tiles == 0) return (n_chunks == 0 && n_tiles == 0) ? ZIPMOE_OK : ZIPMOE_ERR_INVALID_ARG;
   if (!chunks || !tables || n_tables == 0 || !payload || !sm || !out_bf16) return ZIPMOE_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(payload) | reinterpret_cast<uintptr_t>(sm) | reinterpret_cast<uintptr_t>(out_bf16) |
@@ -455,7 +464,10 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
     const uint32_t most = (n_tiles + 15 - 1) / 15;   // a tile per warp at least
     if (ctas > most) ctas = most;
   }
-  if (narrow && batched) zipmoe_dev::decode_kernel<false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
+  const bool lean = narrow && (flags & ZIPMOE_DECODE_SHORT_CODES);
+  if (lean && batched) zipmoe_dev::decode_kernel<false, true, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
+  else if (lean) zipmoe_dev::decode_kernel<false, false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
+  else if (narrow && batched) zipmoe_dev::decode_kernel<false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
   else if (narrow) zipmoe_dev::decode_kernel<false, false><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
   else if (batched) zipmoe_dev::decode_kernel<true, true><<<ctas, Wide::kThreads, Wide::kSmemBytes, st>>>(a);
   else zipmoe_dev::decode_kernel<true, false><<<ctas, Wide::kThreads, Wide::kSmemBytes, st>>>(a);

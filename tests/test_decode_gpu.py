@@ -157,6 +157,33 @@ def test_dynamic_distribution_many_launches_in_a_row(zb):
                 assert np.array_equal(got, want), it
 
 
+def test_short_codes_promise_kept_and_broken(zb):
+    """ZIPMOE_DECODE_SHORT_CODES selects the kernel variant that carries only the common path.  The plan gives the
+    promise exactly when it holds; a launch that gives it falsely must leave the offending tiles undecoded and say
+    so in the status word, never write wrong data."""
+    import torch
+    x = inputs.stress_tensor(1, max_elems=200000)[0]                 # heavy-tailed: needs codes above 8 bits at limit 12
+    short = zb.DecodePlan([zb.zipmoe_encode(x, chunk_elems=16384, max_code_len=8)])
+    long_ = zb.DecodePlan([zb.zipmoe_encode(x, chunk_elems=16384, max_code_len=12)])
+    assert short.flags == zb.DECODE_SHORT_CODES and short.max_code_len <= 8
+    assert long_.max_code_len > 8 and long_.flags == 0
+    for plan in (short, long_):                                     # both decode exactly with the plan's own flags
+        dev = plan.to_device()
+        out = dev.new_output()
+        dev.decode(out)
+        torch.cuda.synchronize()
+        assert int(dev.status.item()) == 0
+        assert np.array_equal(plan.tensor_slice(out.cpu().numpy().view(np.uint16), 0), x)
+    long_.flags = zb.DECODE_SHORT_CODES                             # the false promise
+    dev = long_.to_device()
+    out = dev.new_output()
+    out.fill_(0x5555)
+    dev.decode(out)
+    torch.cuda.synchronize()
+    assert int(dev.status.item()) == 5
+    assert bool((out == 0x5555).all())                              # nothing was written
+
+
 def test_empty_launch_and_bad_arguments(zb):
     import torch
     zb.zipmoe_decode(None, 0, 0, None, 0, None, 0, None, 0, None, 0)       # nothing to do: OK
