@@ -474,9 +474,9 @@ def run_ours(args):
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch, from the ncu capture summarised
 # under profiles/ (null until a capture of the current kernel exists)
 TRAFFIC_BYTES = {
-    # 410.5 MB measured on 16 of the 64 experts (profiles/decode_kernel_moe16_2048x1408.md), scaled by 4:
+    # 408.0 MB measured on 16 of the 64 experts (profiles/decode_kernel_moe16_2048x1408.md), scaled by 4:
     # traffic grows in proportion to the number of tiles
-    "moe64_2048x1408_chunk64K": 4 * 410_534_144,
+    "moe64_2048x1408_chunk64K": 4 * 407_956_992,
 }
 
 
