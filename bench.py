@@ -251,7 +251,10 @@ def bench_ffn(dev, iters=20, cpu_tokens=2, token_counts=(1, 16, 64), config="lar
         us_f, us_u = timed(fused), timed(unfused)
         nbytes = sum(expert_bytes[e] for e in active)
         out["T%d" % T] = {"us": us_f, "tokens_per_s": T / us_f * 1e6, "active_experts": len(active),
-                          "compressed_gbs": nbytes / us_f / 1e3, "decode_then_gemm_us": us_u,
+                          "compressed_gbs": nbytes / us_f / 1e3,
+                          # the fused call must at least read the routed experts' compressed bytes once
+                          "frac_of_hbm_roofline": nbytes / us_f / 1e3 / measured_peaks()[0]["hbm_gbs"],
+                          "decode_then_gemm_us": us_u,
                           "speedup_vs_decode_then_gemm": us_u / us_f, "max_abs_diff_vs_decode_then_gemm": diff,
                           "status": int(ex.dev.status.item())}
     out["config"] = label
