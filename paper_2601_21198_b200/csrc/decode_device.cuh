@@ -9,6 +9,7 @@
 #include <type_traits>
 
 #include "zipmoe.h"
+#include "tile_geometry.h"
 
 namespace zipmoe_dev {
 
@@ -32,10 +33,6 @@ constexpr uint32_t kStatusBadBitCount = 2;    // a tile's lane bit counts overru
 constexpr uint32_t kStatusWaitTimeout = 3;    // an asynchronous copy did not complete in time
 constexpr uint32_t kStatusBadTable = 4;       // code lengths do not form a complete prefix code
 constexpr uint32_t kStatusBrokenPromise = 5;  // ZIPMOE_DECODE_SHORT_CODES was given, yet a tile has longer codes or a longer record
-
-constexpr uint32_t kPieceIters = 8;           // iterations served by one piece of sign+mantissa bytes
-constexpr uint32_t kSmPieceBytes = kPieceIters * 256;
-constexpr uint32_t kSmPieces = 16 / kPieceIters;   // pieces of a full tile = sign+mantissa slots of a warp
 
 constexpr int kPayBuf = 2048;        // record bytes staged in shared memory; longer records are read from global
 constexpr int kPaySlack = 64;        // readable bytes after a staged record (a lane looks three words ahead)
@@ -279,8 +276,8 @@ __device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c
       rec_off + w.rec_bytes > a.payload_bytes)
     return w;
   w.iters = tile_elems >> 8;
-  w.pieces = (w.iters + kPieceIters - 1) / kPieceIters;
   w.valid = (t == m - 1) ? last : tile_elems;
+  w.pieces = sm_pieces_of_tile(w.valid);   // only the pieces that hold bytes of the tile are ever copied
   const uint32_t q = tile0 + t;
   uint64_t origin = out_off;
   if (tpr == 1) origin += (uint64_t)q * w.iters * pitch;   // linear layout: no division
@@ -566,7 +563,7 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
   if (!dec.init(rec_s, rec_g, rec_bytes, lut, lane)) return kStatusBadBitCount;
   static_assert(kPieceIters % 2 == 0, "a piece holds whole pairs of iterations");
 
-  const uint32_t pieces = (iters + kPieceIters - 1) / kPieceIters;
+  const uint32_t pieces = sm_pieces_of_tile(valid);   // pieces that exist: iterations past them hold no element
   if (SMALL && valid == iters * 256u && iters < kPieceIters && (iters & 1u) == 0) {
     // a small full tile (chunks of less than 2048 elements): one piece, a few pairs of iterations
     const uint32_t sm_s = feed.begin(0);

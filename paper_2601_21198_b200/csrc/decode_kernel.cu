@@ -80,8 +80,8 @@ struct WarpPipe {
     pending |= 1u << stage;
   }
   __device__ __forceinline__ void load_sm_piece(const TileWork &t, uint32_t p) {
-    const uint32_t all = (t.valid + 15u) & ~15u;
-    const uint32_t bytes = min(kSmPieceBytes, all - p * kSmPieceBytes);
+    const uint32_t bytes = sm_piece_bytes(t.valid, p);
+    if (bytes == 0) return;   // (callers ask for p < t.pieces only)
     if (lane == 0) bulk_load(sm_addr + p * kSmPieceBytes, t.sm + p * kSmPieceBytes, bytes, bar(kPayStages + p));
     pending |= 1u << (kPayStages + p);
   }
@@ -156,7 +156,7 @@ __device__ __forceinline__ TileWork fetch_tile(const LaunchArgs &a, const Packed
   w.staged = (bits >> 30) & 1u;
   w.valid = bits & 0x1FFFu;
   w.iters = (bits >> 13) & 31u;
-  w.pieces = (w.iters + kPieceIters - 1) / kPieceIters;
+  w.pieces = sm_pieces_of_tile(w.valid);
   w.rec_bytes = ((bits >> 18) & 0x3FFu) << 4;
   w.rec = a.payload + ((size_t)rec16 << 4);
   w.sm = a.sm + ((size_t)sm16 << 4);

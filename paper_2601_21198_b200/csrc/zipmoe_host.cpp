@@ -482,9 +482,10 @@ zipmoe_status zipmoe_blob_plan(const void *blob_v, uint64_t bytes, uint64_t payl
     const uint32_t m = g.chunk_tiles(k);
     if (at + 4ull * (m + 1) > info.payload_off + info.payload_bytes) return ZIPMOE_ERR_BAD_FORMAT;
     for (uint32_t t = 0; t < m; ++t) {
-      const uint32_t o0 = load_le<uint32_t>(blob + at + 4ull * t), o1 = load_le<uint32_t>(blob + at + 4ull * (t + 1));
-      if (o1 < o0) return ZIPMOE_ERR_BAD_FORMAT;
-      max_record = std::max(max_record, (o1 - o0) * 16u);
+      const uint64_t o0 = load_le<uint32_t>(blob + at + 4ull * t), o1 = load_le<uint32_t>(blob + at + 4ull * (t + 1));
+      // (a damaged tile table must not wrap this into a small hint that selects the narrow kernel)
+      if (o1 < o0 || (o1 - o0) * 16 > tile_record_max(g.tile_elems)) return ZIPMOE_ERR_BAD_FORMAT;
+      max_record = std::max(max_record, (uint32_t)((o1 - o0) * 16));
     }
   }
   for (uint32_t k = 0; k < g.n_chunks; ++k) {

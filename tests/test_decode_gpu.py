@@ -37,6 +37,9 @@ CASES = [
     (3, 1000, 0, 1024), (1, 4095, 0, 4096), (1, 4096, 0, 4096), (1, 4097, 0, 4096), (5, 4099, 0, 16384),
     (64, 1408, 0, 4096), (100, 1408, 0, 65536), (16, 256, 1, 4096), (48, 768, 1, 8192), (32, 4096, 1, 65536),
     (16, 14336, 1, 262144), (333, 1031, 0, 262144),
+    # a short last tile whose sign+mantissa bytes end in the first 2 KB piece, at its end, or just past it
+    (1, 2000, 0, 4096), (1, 2048, 0, 4096), (1, 4096 + 100, 0, 4096), (1, 4096 + 2048, 0, 4096), (3, 4096 + 1365, 0, 16384),
+    (1, 4096 + 2049, 0, 4096),
 ]
 
 
@@ -259,9 +262,10 @@ def test_small_expert_layer_config_full(zb):
     _check_full_workload(zb, workloads.small_layer(), 24)
 
 
-def test_large_expert_layer_config_full(zb):
+@pytest.mark.parametrize("max_code_len", [8, 12])
+def test_large_expert_layer_config_full(zb, max_code_len):
     from paper_2601_21198_b200 import workloads
-    _check_full_workload(zb, workloads.large_layer(max_code_len=12), 8)
+    _check_full_workload(zb, workloads.large_layer(max_code_len=max_code_len), 8)
 
 
 def test_large_expert_layer_blocked_layout(zb):

@@ -38,16 +38,30 @@ def oracle_out(ws_decoded, tok, ids, wts, rows):
     w1 = {e: ws_decoded[3 * e] for e in set(ids[rows].ravel().tolist())}
     w3 = {e: ws_decoded[3 * e + 1] for e in w1}
     w2 = {e: ws_decoded[3 * e + 2] for e in w1}
-    out, y = offn.expert_ffn(tok[rows], ids[rows], None if wts is None else wts[rows], w1, w3, w2)
-    return offn.bf16_to_f64(out), y
+    return offn.expert_ffn(tok[rows], ids[rows], None if wts is None else wts[rows], w1, w3, w2)
 
 
-def check(got_bits, want, label):
-    got = offn.bf16_to_f64(got_bits)
+def check(got_bits, want_bits, want_exact, label):
+    """want_bits: the oracle's bf16 output; want_exact: its fp64 value before the last rounding.  Every element
+    must lie within 1e-2 of the oracle's output -- except that an element of magnitude >= 1.28, whose bf16
+    neighbours are more than 1e-2 apart, may be the neighbouring bf16 value (one rounding flip of the final
+    conversion: fp32 against fp64 accumulation); such elements are counted, must be exactly one bf16 step away,
+    and must be rare."""
+    got, want = offn.bf16_to_f64(got_bits), offn.bf16_to_f64(want_bits)
     err = np.abs(got - want)
-    bound = np.maximum(MAX_ABS, np.abs(want) * 2.0 ** -7)      # one bf16 spacing is at most 2^-7 |x|
     rel = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30)
-    assert (err <= bound).all() and rel <= REL_FRO, (label, err.max(), rel)
+    assert rel <= REL_FRO, (label, rel)
+    wide = err > MAX_ABS
+    n_wide = int(wide.sum())
+    if n_wide:
+        g, w = got_bits[wide].astype(np.int64), want_bits[wide].astype(np.int64)
+        assert (np.abs(want[wide]) >= 1.28).all(), (label, "an error above 1e-2 on a small output", err.max())
+        assert (np.abs(g - w) == 1).all(), (label, "more than one bf16 step from the oracle")   # same sign, adjacent patterns
+        # a flip needs the exact value to sit near the midpoint of the two candidates
+        assert (np.abs(got[wide] - want_exact[wide]) <= 0.75 * err[wide]).all(), label
+        assert n_wide <= max(2, got.size // 500), (label, n_wide)
+    print("%s: %d of %d outputs one bf16 step from the oracle (|value| >= 1.28), max abs err %.3g, rel Frobenius %.3g"
+          % (label, n_wide, got.size, err.max(), rel))
 
 
 @pytest.mark.parametrize("T", [1, 5, 16, 64])
@@ -67,8 +81,8 @@ def test_small_experts_match_oracle(zb, T, max_code_len):
                      None if weights is None else torch.from_numpy(weights).cuda())
         torch.cuda.synchronize()
         assert int(ex.dev.status.item()) == 0
-        want, _ = oracle_out(decoded, tok, ids, weights, np.arange(T))
-        check(out.cpu().numpy().view(np.uint16), want, (T, max_code_len, weights is None))
+        want, y = oracle_out(decoded, tok, ids, weights, np.arange(T))
+        check(out.cpu().numpy().view(np.uint16), want, y, (T, max_code_len, weights is None))
 
 
 def test_single_expert_k1_and_unused_experts(zb):
@@ -81,8 +95,8 @@ def test_single_expert_k1_and_unused_experts(zb):
     out = ex.ffn(torch.from_numpy(tok.view(np.int16)).cuda(), torch.from_numpy(ids).cuda(), None)
     torch.cuda.synchronize()
     assert int(ex.dev.status.item()) == 0
-    want, _ = oracle_out(ws, tok, ids, None, np.arange(7))
-    check(out.cpu().numpy().view(np.uint16), want, "k1")
+    want, y = oracle_out(ws, tok, ids, None, np.arange(7))
+    check(out.cpu().numpy().view(np.uint16), want, y, "k1")
 
 
 def test_bad_arguments(zb):
@@ -103,7 +117,8 @@ def test_bad_arguments(zb):
 @pytest.mark.parametrize("T", [1, 16, 64])
 def test_large_experts_config(zb, T):
     """8 experts of 4096 -> 14336 -> 4096 (256K-element chunks), top-2 of 8 with Zipf(1.2) popularity.
-    The oracle FFN is evaluated on a sample of the tokens (tokens are independent)."""
+    Every token row is compared with the oracle for T = 1 and 16; for T = 64 (which also selects the kernel's
+    other shared-memory plan) 16 rows chosen so that every expert that has tokens is covered."""
     import torch
     from paper_2601_21198_b200 import workloads
     w = _large_layer(workloads)
@@ -114,9 +129,10 @@ def test_large_experts_config(zb, T):
                  torch.from_numpy(wts).cuda())
     torch.cuda.synchronize()
     assert int(ex.dev.status.item()) == 0
-    rows = np.arange(T) if T <= 4 else np.random.default_rng(T).choice(T, 4, replace=False)
-    want, _ = oracle_out(w.originals, tok, ids, wts, rows)
-    check(out.cpu().numpy().view(np.uint16)[rows], want, ("large", T))
+    rows = np.arange(T) if T <= 16 else _rows_covering_all_experts(ids, 16, seed=T)
+    assert set(ids[rows].ravel().tolist()) == set(ids.ravel().tolist())
+    want, y = oracle_out(w.originals, tok, ids, wts, rows)
+    check(out.cpu().numpy().view(np.uint16)[rows], want, y, ("large", T))
 
 
 @pytest.mark.parametrize("T", [1, 16])
@@ -135,9 +151,20 @@ def test_paper_shape_experts_with_padded_intermediate_size(zb, T):
     out = ex.ffn(torch.from_numpy(tok.view(np.int16)).cuda(), torch.from_numpy(ids).cuda(), torch.from_numpy(wts).cuda())
     torch.cuda.synchronize()
     assert int(ex.dev.status.item()) == 0
-    rows = np.arange(T) if T <= 4 else np.random.default_rng(T).choice(T, 4, replace=False)
-    want, _ = oracle_out(w.originals, tok, ids, wts, rows)
-    check(out.cpu().numpy().view(np.uint16)[rows], want, ("paper shape", T))
+    want, y = oracle_out(w.originals, tok, ids, wts, np.arange(T))
+    check(out.cpu().numpy().view(np.uint16), want, y, ("paper shape", T))
+
+
+def _rows_covering_all_experts(ids, n, seed):
+    """n token rows: first one row for every expert that appears in ids (the first token that names it), then
+    seeded random rows."""
+    rows = []
+    for e in sorted(set(ids.ravel().tolist())):
+        t = int(np.nonzero((ids == e).any(axis=1))[0][0])
+        if t not in rows:
+            rows.append(t)
+    rest = [int(t) for t in np.random.default_rng(seed).permutation(ids.shape[0]) if int(t) not in rows]
+    return np.array(sorted(rows + rest[: max(0, n - len(rows))]))
 
 
 _cache = {}

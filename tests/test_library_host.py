@@ -218,3 +218,18 @@ def test_plan_reports_the_largest_tile_record(zb):
     u = np.random.default_rng(0).integers(0, 1 << 16, 20000, dtype=np.uint16)
     plan = zb.DecodePlan([zb.zipmoe_encode(u, chunk_elems=4096)])
     assert plan.max_record_bytes == 64 + 4096 + 32 * 4   # 8-bit codes everywhere, one word of padding per lane
+
+
+def test_plan_rejects_a_damaged_tile_table(zb):
+    """The planner's record-size hint picks the kernel variant, so a tile table whose entries would wrap the 32-bit
+    size computation into a small number must be refused, not planned."""
+    x = inputs.gaussian((8, 4096), 0.02, 6)
+    blob = zb.zipmoe_encode(x, chunk_elems=16384)
+    info = zb.zipmoe_blob_info_get(blob)
+    assert zb.zipmoe_blob_plan(blob, 0, 0, 0, 0, 0, 0)[0]["max_record_bytes"][0] > 0
+    for entry, value in [(1, 0x10000001), (2, 0xFFFFFFF0), (1, 0)]:
+        b = blob.copy()
+        b[info.payload_off + 4 * entry: info.payload_off + 4 * entry + 4] = np.frombuffer(np.uint32(value).tobytes(), np.uint8)
+        with pytest.raises(zb.ZipMoEError) as err:
+            zb.zipmoe_blob_plan(b, 0, 0, 0, 0, 0, 0)
+        assert err.value.status == zb.ERR_BAD_FORMAT, (entry, value)
