@@ -21,18 +21,19 @@
  *     canonical Huffman code over exponent bytes, the quantity the paper's
  *     own entropy analysis measures (Fig. 2, Fig. 3).
  *
- * The container layout ("ZMOE v2") is this project's own; it is written out
+ * The container layout ("ZMOE v3") is this project's own; it is written out
  * in full below because the decoder is defined by it.  Every function that
  * has an independent pin (closed form, brute force, textbook special case)
  * is pinned in tests/test_oracle_*.py.  The one part that cannot be pinned
  * against anything but itself is the byte-exact blob layout produced by
- * zo_encode (tie-breaks between equally good codes are free): "parity
- * unpinned" for blob bytes; only decodability and size bounds bind.
+ * zo_encode (tie-breaks between equally good codes and the pairing of
+ * streams into columns are free): "parity unpinned" for blob bytes; only
+ * decodability and size bounds bind.
  *
  * ---------------------------------------------------------------------------
- * ZMOE v2 container (all integers little-endian)
+ * ZMOE v3 container (all integers little-endian)
  *
- *   offset  0  u32 magic 0x454F4D5A      4  u32 version (2)
+ *   offset  0  u32 magic 0x454F4D5A      4  u32 version (3)
  *           8  u64 n_elems              16  u32 rows     20 u32 cols
  *          24  u32 layout (0 linear, 1 blocked)          28 u32 chunk_elems
  *          32  u32 tile_elems           36  u32 max_code_len
@@ -59,24 +60,26 @@
  *                           in the chunk); tile_off[0] is the padded size of
  *                           this table, tile_off[m] the size of the chunk;
  *     zero padding to 16 bytes, then m tile records.
- *   Tile record:
- *     u16 sub_bits[32]      number of code bits of each lane (both of its
- *                           sub-streams together);
- *     the 32 lanes' bit ranges, lane 0 first, concatenated with no padding
- *     between them, stored as u32 words whose bits are consumed from bit 31
- *     down to bit 0; zero padding to a 16-byte boundary.
- *   A lane has two sub-streams inside its bit range [S, E):
- *     sub-stream 0 codes the lane's existing elements of the even iterations
- *       i = 0, 2, 4, ... < I (j = 0..7 inside each) and runs forwards from S:
- *       its k-th bit is bit S + k;
- *     sub-stream 1 codes those of the odd iterations i = 1, 3, 5, ... < I and
- *       runs backwards from E: its k-th bit is bit E - 1 - k.
- *   Bits of the range that belong to neither sub-stream lie between their ends:
- *   at most 63 of them, all zero (an encoder may insert them, e.g. to keep lanes
- *   of equal length from starting at the same word offset; this oracle's
- *   encoder inserts none).  (Two independent streams per lane let a decoder work
- *   on two codes at a time at no cost in size; the paper leaves the order of
- *   elements inside a shard open.)
+ *   Tile record of W rows (32 + 128*W bytes; W >= 1 follows from the record's size):
+ *     u8  bcol[32]          the column that holds lane L's backward stream:
+ *                           a permutation of 0..31;
+ *     u32 word[W][32]       row r, column c at byte 32 + (r*32 + c)*4.
+ *   Column c is a string of 32*W bits: its bit y is bit 31 - (y mod 32) of
+ *   word[y / 32][c].  Every lane has two code streams:
+ *     the forward stream codes the lane's existing elements of the even
+ *       iterations i = 0, 2, 4, ... < I (j = 0..7 inside each); its k-th bit is
+ *       bit k of column `lane`;
+ *     the backward stream codes those of the odd iterations i = 1, 3, 5, ... < I;
+ *       its k-th bit is bit 32*W - 1 - k of column bcol[lane].
+ *   The two streams that share a column must not overlap; the bits between
+ *   their ends are zero.  (Word r of all 32 columns is one contiguous 128-byte
+ *   row, so 32 readers that each follow one column touch 32 different
+ *   addresses modulo 128 bytes whatever their positions; pairing a long
+ *   forward stream with a short backward stream keeps W near the mean.  The
+ *   paper leaves the order of elements inside a shard open.)  An encoder may
+ *   choose any permutation and any W that fits; this oracle pairs the lanes in
+ *   descending order of forward bits with the lanes in ascending order of
+ *   backward bits and takes the smallest W.
  *
  *   Sign+mantissa section: byte q*tile_elems + pos holds
  *     (sign << 7) | mantissa  of the element at (q, pos); zero padded to 16.
@@ -101,20 +104,19 @@
 #define ZO_TABLE_OFF 64u
 #define ZO_CHUNKOFF_OFF 320u
 #define ZO_MAX_CODE_LEN 12
-#define ZO_VERSION 2u
-#define ZO_REC_HEAD 64u /* u16 sub_bits[32] */
+#define ZO_VERSION 3u
+#define ZO_REC_HEAD 32u /* u8 bcol[32] */
+#define ZO_MAX_ROWS 48u /* 128 codes of at most 12 bits in a column */
 
 /* ---- little-endian field access ---------------------------------------- */
 static uint32_t rd32(const uint8_t *p) {
   return (uint32_t)p[0] | ((uint32_t)p[1] << 8) | ((uint32_t)p[2] << 16) | ((uint32_t)p[3] << 24);
 }
 static uint64_t rd64(const uint8_t *p) { return (uint64_t)rd32(p) | ((uint64_t)rd32(p + 4) << 32); }
-static uint32_t rd16(const uint8_t *p) { return (uint32_t)p[0] | ((uint32_t)p[1] << 8); }
 static void wr32(uint8_t *p, uint32_t v) {
   p[0] = (uint8_t)v; p[1] = (uint8_t)(v >> 8); p[2] = (uint8_t)(v >> 16); p[3] = (uint8_t)(v >> 24);
 }
 static void wr64(uint8_t *p, uint64_t v) { wr32(p, (uint32_t)v); wr32(p + 4, (uint32_t)(v >> 32)); }
-static void wr16(uint8_t *p, uint32_t v) { p[0] = (uint8_t)v; p[1] = (uint8_t)(v >> 8); }
 static uint64_t round_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 
 /* ---- bit-field decomposition and re-assembly (Sections 2.2, 3.1, 3.3) -- */
@@ -308,23 +310,23 @@ static uint64_t elem_of(const zo_header *h, uint64_t q, uint32_t pos) {
 uint64_t zo_encode_bound(uint64_t rows, uint64_t cols, uint32_t layout, uint32_t chunk_elems) {
   zo_header h;
   if (geometry(rows, cols, layout, chunk_elems, &h) != ZO_OK) return 0;
-  uint64_t per_tile = ZO_REC_HEAD + (uint64_t)h.tile_elems * ZO_MAX_CODE_LEN / 8 + 16;
+  uint64_t per_tile = ZO_REC_HEAD + 128ull * ZO_MAX_ROWS;
   uint64_t tpc = h.chunk_elems / h.tile_elems;
   uint64_t per_chunk = round_up(4 * (tpc + 1), 16);
   return h.payload_off + h.n_tiles * per_tile + h.n_chunks * per_chunk + h.sm_bytes + 64;
 }
 
-/* ---- bit access: bits of a u32-word stream, bit 31 of each word first --- */
-static void put_bit(uint8_t *base, uint64_t p, uint32_t bit) {
-  uint8_t *w = base + 4 * (p >> 5);
-  uint32_t v = rd32(w);
-  uint32_t at = 31 - (uint32_t)(p & 31);
-  v = (v & ~((uint32_t)1 << at)) | ((bit & 1u) << at);
-  wr32(w, v);
+/* ---- bit access: bit y of column c of a tile record (see the layout above) -- */
+static uint8_t *column_word(const uint8_t *rec, uint32_t c, uint64_t y) {
+  return (uint8_t *)rec + ZO_REC_HEAD + ((y >> 5) * 32 + c) * 4;
 }
-static uint32_t get_bit(const uint8_t *base, uint64_t p) {
-  uint32_t v = rd32(base + 4 * (p >> 5));
-  return (v >> (31 - (uint32_t)(p & 31))) & 1u;
+static void put_bit(uint8_t *rec, uint32_t c, uint64_t y, uint32_t bit) {
+  uint8_t *w = column_word(rec, c, y);
+  uint32_t at = 31 - (uint32_t)(y & 31);
+  wr32(w, (rd32(w) & ~((uint32_t)1 << at)) | ((bit & 1u) << at));
+}
+static uint32_t get_bit(const uint8_t *rec, uint32_t c, uint64_t y) {
+  return (rd32(column_word(rec, c, y)) >> (31 - (uint32_t)(y & 31))) & 1u;
 }
 
 /* ---- encoder ------------------------------------------------------------ */
@@ -368,33 +370,51 @@ int zo_encode(const uint16_t *x, uint64_t rows, uint64_t cols, uint32_t layout, 
       uint64_t q = (uint64_t)q0 + t;
       wr32(chunk + 4ull * t, (uint32_t)(rel / 16));
       uint8_t *rec = chunk + rel;
-      uint64_t rec_max = ZO_REC_HEAD + (uint64_t)h.tile_elems * ZO_MAX_CODE_LEN / 8 + 16;
-      memset(rec, 0, rec_max);
-      uint64_t p = 0; /* bit position in the record's bit area */
+      /* code bits of every lane's forward stream (even iterations) and backward stream (odd iterations) */
+      uint64_t fbits[32], bbits[32];
       for (uint32_t lane = 0; lane < 32; ++lane) {
-        /* size of the lane's bit range first, then both sub-streams into it */
-        uint64_t lane_bits = 0;
-        for (uint32_t i = 0; i < I; ++i)
-          for (uint32_t j = 0; j < 8; ++j) {
-            uint64_t f = elem_of(&h, q, (i * 32 + lane) * 8 + j);
-            if (f != UINT64_MAX) lane_bits += len[exp[f]];
-          }
-        uint64_t fwd = p, bwd = p + lane_bits; /* next bit of sub-stream 0; one past the next bit of sub-stream 1 */
+        fbits[lane] = bbits[lane] = 0;
         for (uint32_t i = 0; i < I; ++i)
           for (uint32_t j = 0; j < 8; ++j) {
             uint64_t f = elem_of(&h, q, (i * 32 + lane) * 8 + j);
             if (f == UINT64_MAX) continue;
-            uint32_t s = exp[f];
-            for (int b = len[s] - 1; b >= 0; --b) {
-              if (i % 2 == 0) put_bit(rec + ZO_REC_HEAD, fwd++, (code[s] >> b) & 1u);
-              else put_bit(rec + ZO_REC_HEAD, --bwd, (code[s] >> b) & 1u);
+            if (i % 2 == 0) fbits[lane] += len[exp[f]];
+            else bbits[lane] += len[exp[f]];
+          }
+      }
+      /* pairing: the column with the k-th longest forward stream takes the k-th shortest backward stream
+       * (ties by lane number); any permutation would be valid, this one keeps the columns level */
+      uint32_t by_f[32], by_b[32], bcol[32];
+      for (uint32_t a = 0; a < 32; ++a) by_f[a] = by_b[a] = a;
+      for (uint32_t a = 1; a < 32; ++a)
+        for (uint32_t b = a; b > 0; --b) {
+          if (fbits[by_f[b]] > fbits[by_f[b - 1]]) { uint32_t t2 = by_f[b]; by_f[b] = by_f[b - 1]; by_f[b - 1] = t2; }
+          if (bbits[by_b[b]] < bbits[by_b[b - 1]]) { uint32_t t2 = by_b[b]; by_b[b] = by_b[b - 1]; by_b[b - 1] = t2; }
+        }
+      uint64_t W = 1;
+      for (uint32_t a = 0; a < 32; ++a) {
+        bcol[by_b[a]] = by_f[a];
+        uint64_t need = (fbits[by_f[a]] + bbits[by_b[a]] + 31) / 32;
+        if (need > W) W = need;
+      }
+      if (W > ZO_MAX_ROWS) { free(exp); free(sm); return ZO_ERR_ARG; }
+      uint64_t rec_bytes = ZO_REC_HEAD + 128 * W;
+      memset(rec, 0, rec_bytes);
+      for (uint32_t lane = 0; lane < 32; ++lane) rec[lane] = (uint8_t)bcol[lane];
+      for (uint32_t lane = 0; lane < 32; ++lane) {
+        uint64_t fwd = 0, bwd = 32 * W; /* next bit of the forward stream; one past the next bit of the backward stream */
+        for (uint32_t i = 0; i < I; ++i)
+          for (uint32_t j = 0; j < 8; ++j) {
+            uint64_t f = elem_of(&h, q, (i * 32 + lane) * 8 + j);
+            if (f == UINT64_MAX) continue;
+            uint32_t sy = exp[f];
+            for (int b = len[sy] - 1; b >= 0; --b) {
+              if (i % 2 == 0) put_bit(rec, lane, fwd++, (code[sy] >> b) & 1u);
+              else put_bit(rec, bcol[lane], --bwd, (code[sy] >> b) & 1u);
             }
           }
-        /* fwd == bwd here: the sub-streams meet */
-        wr16(rec + 2 * lane, (uint32_t)lane_bits);
-        p += lane_bits;
       }
-      rel += round_up(ZO_REC_HEAD + (p + 7) / 8, 16);
+      rel += rec_bytes;
     }
     wr32(chunk + 4ull * m, (uint32_t)(rel / 16));
     at += rel;
@@ -500,14 +520,22 @@ int zo_decode_chunk(const uint8_t *blob, uint64_t bytes, uint32_t k, uint16_t *o
   for (uint32_t t = 0; t < m; ++t) {
     uint64_t q = (uint64_t)q0 + t;
     uint64_t r0 = (uint64_t)rd32(chunk + 4ull * t) * 16, r1 = (uint64_t)rd32(chunk + 4ull * (t + 1)) * 16;
-    if (r1 < r0 + ZO_REC_HEAD || r1 > chunk_bytes) return ZO_ERR_CORRUPT;
+    if (r1 < r0 + ZO_REC_HEAD + 128 || r1 > chunk_bytes || (r1 - r0 - ZO_REC_HEAD) % 128) return ZO_ERR_CORRUPT;
     const uint8_t *rec = chunk + r0;
-    uint64_t area_bits = (r1 - r0 - ZO_REC_HEAD) * 8;
-    uint64_t p = 0;
+    uint64_t W = (r1 - r0 - ZO_REC_HEAD) / 128;
+    if (W > ZO_MAX_ROWS) return ZO_ERR_CORRUPT;
+    /* bcol must be a permutation: every column holds exactly one backward stream */
+    uint32_t owner[32]; /* the lane whose backward stream lives in column c */
+    for (uint32_t c = 0; c < 32; ++c) owner[c] = 32;
     for (uint32_t lane = 0; lane < 32; ++lane) {
-      uint64_t p_end = p + rd16(rec + 2 * lane);
-      if (p_end > area_bits) return ZO_ERR_CORRUPT;
-      uint64_t fwd = p, bwd = p_end;
+      uint32_t c = rec[lane];
+      if (c >= 32 || owner[c] != 32) return ZO_ERR_CORRUPT;
+      owner[c] = lane;
+    }
+    uint64_t fwd_end[32], bwd_end[32]; /* per lane: bits its forward stream used; first bit its backward stream used */
+    for (uint32_t lane = 0; lane < 32; ++lane) {
+      uint32_t bc = rec[lane];
+      uint64_t fwd = 0, bwd = 32 * W;
       for (uint32_t i = 0; i < I; ++i)
         for (uint32_t j = 0; j < 8; ++j) {
           uint32_t pos = (i * 32 + lane) * 8 + j;
@@ -516,22 +544,32 @@ int zo_decode_chunk(const uint8_t *blob, uint64_t bytes, uint32_t k, uint16_t *o
           uint32_t c = 0;
           int L = 0, found = 0;
           while (L < (int)h.max_code_len) {
-            if (fwd >= bwd) return ZO_ERR_CORRUPT; /* the lane's bits are used up */
-            uint32_t bit = (i % 2 == 0) ? get_bit(rec + ZO_REC_HEAD, fwd++) : get_bit(rec + ZO_REC_HEAD, --bwd);
+            uint32_t bit;
+            if (i % 2 == 0) {
+              if (fwd >= 32 * W) return ZO_ERR_CORRUPT; /* the column is used up */
+              bit = get_bit(rec, lane, fwd++);
+            } else {
+              if (bwd == 0) return ZO_ERR_CORRUPT;
+              bit = get_bit(rec, bc, --bwd);
+            }
             c = (c << 1) | bit;
             ++L;
             if (c >= first[L] && c - first[L] < count[L]) { found = 1; break; }
           }
           if (!found) return ZO_ERR_CORRUPT;
           uint8_t e = order[base[L] + (c - first[L])];
-          uint8_t s = smsec[q * h.tile_elems + pos];
-          zo_merge(&e, &s, 1, &out[f]);
+          uint8_t sb = smsec[q * h.tile_elems + pos];
+          zo_merge(&e, &sb, 1, &out[f]);
         }
-      /* what is left between the sub-streams is padding: short and zero */
-      if (bwd - fwd > 63) return ZO_ERR_CORRUPT;
-      for (uint64_t g = fwd; g < bwd; ++g)
-        if (get_bit(rec + ZO_REC_HEAD, g)) return ZO_ERR_CORRUPT;
-      p = p_end;
+      fwd_end[lane] = fwd;
+      bwd_end[lane] = bwd;
+    }
+    /* the two streams of a column must not overlap, and what lies between them is zero */
+    for (uint32_t c = 0; c < 32; ++c) {
+      uint64_t lo = fwd_end[c], hi = bwd_end[owner[c]];
+      if (lo > hi) return ZO_ERR_CORRUPT;
+      for (uint64_t g = lo; g < hi; ++g)
+        if (get_bit(rec, c, g)) return ZO_ERR_CORRUPT;
     }
   }
   return ZO_OK;

@@ -200,18 +200,34 @@ def _bits_of_bytes(values):
     return [(v >> b) & 1 for v in values for b in range(7, -1, -1)]
 
 
-def _pack_words(bits):
-    """Bits -> bytes of a u32 word stream consumed from bit 31 down, little-endian in memory."""
-    bits = list(bits) + [0] * (-len(bits) % 32)
-    by = np.packbits(np.array(bits, dtype=np.uint8)).reshape(-1, 4)[:, ::-1]
-    return by.ravel()
+def _record_of_columns(bcol, columns):
+    """A tile record written out from the format's definition: 32 bytes naming the column of each lane's backward
+    stream, then W rows of 32 words; bit y of column c is bit 31 - y % 32 of the word in row y // 32, column c."""
+    W = len(columns[0]) // 32
+    words = np.zeros((W, 32), np.uint32)
+    for c, bits in enumerate(columns):
+        assert len(bits) == 32 * W
+        for y, bit in enumerate(bits):
+            if bit:
+                words[y // 32, c] |= np.uint32(1 << (31 - y % 32))
+    return np.concatenate([np.array(bcol, np.uint8), words.astype("<u4").ravel().view(np.uint8)])
+
+
+def _column(forward_bits, backward_bits, W):
+    """Forward stream from bit 0 upwards, backward stream from bit 32 W - 1 downwards, zeros between."""
+    col = [0] * (32 * W)
+    assert len(forward_bits) + len(backward_bits) <= 32 * W
+    col[:len(forward_bits)] = forward_bits
+    for k, bit in enumerate(backward_bits):
+        col[32 * W - 1 - k] = bit
+    return col
 
 
 def test_uniform_exponents_store_the_raw_exponent_bytes():
-    """All 256 exponents equally frequent -> every code is the 8-bit symbol itself, so a
-    lane's bit range is: the exponent bytes of its even iterations, forwards, then those
-    of its odd iterations written backwards from the end of the range (the last byte of
-    the range is the bit-reversed first odd-iteration exponent).  Needs no Huffman."""
+    """All 256 exponents equally frequent -> every code is the 8-bit symbol itself, so column c of a tile's
+    record is: the exponent bytes of lane c's even iterations from the top, and those of its odd iterations
+    written upwards from the bottom (all streams are equally long, so every lane keeps its own column).
+    Needs no Huffman."""
     rng = np.random.default_rng(11)
     e = np.tile(np.arange(256, dtype=np.uint16), 32)
     rng.shuffle(e)
@@ -223,20 +239,15 @@ def test_uniform_exponents_store_the_raw_exponent_bytes():
     assert hdr["n_chunks"] == 2 and hdr["n_tiles"] == 2 and hdr["tile_elems"] == 4096
     pay = hdr["payload_off"]
     offs = blob[320:320 + 8 * 3].view(np.uint64)
-    rec_bytes = 64 + 4096
+    rec_bytes = 32 + 32 * 128          # 128 codes of 8 bits per column: 32 rows
     assert offs.tolist() == [0, (16 + rec_bytes) * 8, 2 * (16 + rec_bytes) * 8]
     for q in range(2):
         chunk = blob[pay + q * (16 + rec_bytes): pay + (q + 1) * (16 + rec_bytes)]
         assert chunk[:8].view(np.uint32).tolist() == [1, 1 + rec_bytes // 16]
-        rec = chunk[16:]
-        assert (rec[:64].view(np.uint16) == 128 * 8).all()
         tile = e[q * 4096:(q + 1) * 4096].astype(np.uint8).reshape(16, 32, 8)   # [i, lane, j]
-        bits = []
-        for lane in range(32):
-            even = tile[0::2, lane, :].ravel().tolist()
-            odd = tile[1::2, lane, :].ravel().tolist()
-            bits += _bits_of_bytes(even) + _bits_of_bytes(odd)[::-1]
-        assert np.array_equal(rec[64:], _pack_words(bits))
+        cols = [_column(_bits_of_bytes(tile[0::2, lane, :].ravel().tolist()),
+                        _bits_of_bytes(tile[1::2, lane, :].ravel().tolist()), 32) for lane in range(32)]
+        assert np.array_equal(chunk[16:], _record_of_columns(range(32), cols))
     # sign+mantissa section: raw bytes in element order for the linear layout
     smsec = blob[pay + hdr["payload_bytes"]:]
     assert np.array_equal(smsec, ((x >> 8) & 0x80 | x & 0x7F).astype(np.uint8))
@@ -244,9 +255,9 @@ def test_uniform_exponents_store_the_raw_exponent_bytes():
 
 
 def test_uniform_exponents_odd_iteration_count_and_ragged_tail():
-    """Three iterations per tile (chunk of 768 elements) and a tensor that ends in the
-    middle of a lane's group: sub-stream 0 holds iterations 0 and 2, sub-stream 1
-    iteration 1, and elements past the end are not coded."""
+    """Three iterations per tile (chunk of 768 elements) and a tensor that ends in the middle of a lane's
+    group: the forward stream holds iterations 0 and 2, the backward stream iteration 1, and elements past
+    the end are not coded.  The longest column needs 16 + 8 codes of 8 bits: six rows."""
     n = 256 * 5 + 13
     rng = np.random.default_rng(5)
     e = np.concatenate([np.tile(np.arange(256, dtype=np.uint16), 5), np.arange(13, dtype=np.uint16)])
@@ -262,17 +273,50 @@ def test_uniform_exponents_odd_iteration_count_and_ragged_tail():
         chunk = blob[pay + offs[q]: pay + offs[q + 1]]
         first, end = chunk[:8].view(np.uint32).tolist()
         rec = chunk[16 * first: 16 * end]
-        counts, bits = [], []
+        assert rec.size == 32 + 6 * 128
+        cols = []
         for lane in range(32):
             sub = [[int(e[f]) for i in range(h, 3, 2) for j in range(8)
                     for f in [q * 768 + (i * 32 + lane) * 8 + j] if f < n] for h in range(2)]
-            counts.append(8 * (len(sub[0]) + len(sub[1])))
-            bits += _bits_of_bytes(sub[0]) + _bits_of_bytes(sub[1])[::-1]
-        assert rec[:64].view(np.uint16).tolist() == counts
-        body = _pack_words(bits)
-        assert np.array_equal(rec[64:64 + body.size], body)
-        assert not rec[64 + body.size:].any() and rec.size == -(-(64 + len(bits) // 8) // 16) * 16
+            cols.append(_column(_bits_of_bytes(sub[0]), _bits_of_bytes(sub[1]), 6))
+        # the lanes with the longest forward streams come first already (tile 1: lanes 0 and 1), every
+        # backward stream is equally long: each lane keeps its own column
+        assert np.array_equal(rec, _record_of_columns(range(32), cols))
     assert np.array_equal(codec.decode(blob), x)
+
+
+def test_streams_are_paired_into_columns_longest_forward_with_shortest_backward():
+    """Three exponents A, B, C with codes 0, 10, 11 (A far more frequent).  One tile of two iterations: the
+    forward streams code iteration 0, the backward streams iteration 1.  Lane 3 has the longest forward stream
+    (four B), lane 7 the shortest backward stream (no C; every other lane has one), so lane 7's backward stream
+    goes to column 3, and the lanes between move up by one column.  One row holds everything."""
+    A, B, C = 120, 121, 122
+    e = np.full((2, 32, 8), A, np.uint16)
+    e[0, 3, [1, 2, 5, 6]] = B
+    for lane in range(32):
+        if lane != 7:
+            e[1, lane, lane % 8] = C
+    x = (e.ravel() << 7 | 0x0011).astype(np.uint16)
+    blob = codec.encode(x, chunk_elems=512)
+    L = blob[64:320]
+    assert (L[A], L[B], L[C]) == (1, 2, 2) and L.sum() == 5
+    code = {A: [0], B: [1, 0], C: [1, 1]}
+    hdr = codec.info(blob)
+    assert hdr["n_tiles"] == 1 and hdr["payload_bytes"] == 16 + 32 + 128
+    rec = blob[hdr["payload_off"] + 16: hdr["payload_off"] + hdr["payload_bytes"]]
+    bcol = [0, 1, 2, 4, 5, 6, 7, 3] + list(range(8, 32))
+    assert rec[:32].tolist() == bcol
+    fwd = [[b for s in e[0, lane] for b in code[int(s)]] for lane in range(32)]
+    bwd = [[b for s in e[1, lane] for b in code[int(s)]] for lane in range(32)]
+    assert len(fwd[3]) == 12 and len(bwd[7]) == 8 and len(bwd[0]) == 9
+    cols = [_column(fwd[c], bwd[bcol.index(c)], 1) for c in range(32)]
+    assert np.array_equal(rec, _record_of_columns(bcol, cols))
+    assert np.array_equal(codec.decode(blob), x)
+    # column 0 uses bits 0..7 (forward) and 23..31 (backward); a set bit between them is damage
+    bad = blob.copy()
+    bad[hdr["payload_off"] + 16 + 32 + 2] |= 1          # bit 15 of column 0 = bit 16 of its word
+    with pytest.raises(ValueError):
+        codec.decode(bad)
 
 
 def test_round_trip_brute_force_tiny():
@@ -318,8 +362,9 @@ def test_empty_and_single_symbol_tensors():
     x = np.full(1000, 0x3C12, np.uint16)
     blob = codec.encode(x, chunk_elems=1024)
     assert np.array_equal(codec.decode(blob), x)
-    rec = blob[codec.info(blob)["payload_off"] + 16:]
-    assert int(rec[:64].view(np.uint16).sum()) == 1000     # one bit per element
+    hdr = codec.info(blob)
+    rec = blob[hdr["payload_off"] + 16: hdr["payload_off"] + hdr["payload_bytes"]]
+    assert rec.size == 32 + 128 and not rec[32:].any()     # one bit per element (the code 0): at most 16 + 16 in a column
 
 
 def test_chunks_decode_independently_and_in_any_order():
@@ -404,6 +449,7 @@ def test_corrupt_blobs_are_rejected_not_decoded():
     broken(lambda b: b.__setitem__(64 + int(np.flatnonzero(b[64:320])[0]), 0))   # incomplete code
     broken(lambda b: b.__setitem__(328, b[328] ^ 0x10))                    # chunk offset not 128-bit aligned
     broken(lambda b: b.__setitem__(pay + 4, b[pay + 4] + 1))               # tile table end != chunk size
-    broken(lambda b: b.__setitem__(pay + 16, b[pay + 16] ^ 1))             # a lane's bit count
+    broken(lambda b: b.__setitem__(pay + 16, b[pay + 16] ^ 1))             # two backward streams in one column
+    broken(lambda b: b.__setitem__(pay + 17, 32))                          # a column that does not exist
     with pytest.raises(ValueError):
         codec.decode(blob[:-16])                                           # truncated
