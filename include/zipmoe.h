@@ -106,7 +106,7 @@ zipmoe_status zipmoe_blob_info_get(const void *blob, uint64_t blob_bytes, zipmoe
 
 /* Full structural check of a blob on the host: header, complete prefix code
  * (Kraft sum exactly 1, lengths <= max_code_len), monotone 128-bit-aligned
- * chunk offsets, tile tables and per-lane bit counts inside their records.
+ * chunk offsets, tile tables, record sizes and the records' column tables (a permutation each).
  * A blob that passes can be handed to the device decoder safely. */
 zipmoe_status zipmoe_blob_validate(const void *blob, uint64_t blob_bytes);
 
@@ -166,19 +166,22 @@ zipmoe_status zipmoe_blob_plan(const void *blob, uint64_t blob_bytes, uint64_t p
  *             the kernel skips the offending tile and always terminates.
  * n_tiles   : total tiles of the launch (sum of chunks[].n_tiles).
  * max_record_bytes : the largest chunks[].max_record_bytes of the launch, or 0 if unknown.  A host-side hint
- *             only: when no record exceeds 2048 bytes (every tensor but near-incompressible ones) a kernel
- *             variant with smaller record stages and one more warp runs, about 3 % faster.  A wrong hint costs
- *             speed, never correctness.
+ *             only: when no record exceeds ZIPMOE_NARROW_RECORD_BYTES (16 rows: every tensor but
+ *             near-incompressible ones) a kernel variant with smaller record stages and one more warp runs, about
+ *             3 % faster.  A wrong hint costs speed, never correctness.
  * flags     : 0, or ZIPMOE_DECODE_SHORT_CODES: the caller promises that no table of the launch has a code longer
- *             than 8 bits and that max_record_bytes is a true upper bound of at most 2048 (zipmoe_blob_plan's
+ *             than 8 bits and that max_record_bytes is a true upper bound of at most ZIPMOE_NARROW_RECORD_BYTES (zipmoe_blob_plan's
  *             descriptors and the blobs' tables say both).  The kernel variant chosen then carries only the common
  *             path and is 2-3 % faster.  A tile that breaks the promise is not decoded: its output is left as it
  *             was and status_word is set (code 5), so a false promise is loud, never silent.
  * Work distribution: launches of few large tensors (n_tiles >= 512 * n_tables) give every CTA an equal range of
- *             tiles; all others hand the tiles out dynamically through a 4-byte counter.  The counters are a
- *             ring of 1024 words in the library's own device memory (nothing is allocated); a launch zeroes
- *             its word on `stream` before the kernel (one cudaMemsetAsync).  More than 1024 such launches in
- *             flight at once on one device would share counters: do not queue that many without synchronising.
+ *             tiles; all others hand the tiles out dynamically through an 8-byte counter.  The counters are a
+ *             ring of 1024 in the library's own device memory (nothing is allocated); a launch zeroes its
+ *             counter on `stream` before the kernel (one cudaMemsetAsync) and tags it as its own with the first
+ *             range of tiles it takes.  More than 1024 such launches in flight at once on one device would share
+ *             counters: the launch that finds another launch's tag stops taking tiles and sets status_word
+ *             (code 6), the other one is not disturbed -- incomplete output is never silent.  The same holds for
+ *             a captured graph that replays such a launch while a later launch owns its counter.
  * All device pointers 16-byte aligned.  Errors found on the host (null or
  * misaligned pointers, zero table count with non-zero chunks) are returned
  * before anything is launched. */
@@ -188,6 +191,7 @@ zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t n_chunks, 
                             uint64_t out_elems, uint32_t *status_word, zipmoe_stream stream,
                             uint32_t max_record_bytes, uint32_t flags);
 #define ZIPMOE_DECODE_SHORT_CODES 1u
+#define ZIPMOE_NARROW_RECORD_BYTES 2080u /* a tile record of 16 rows: 32 + 16 * 128 bytes */
 
 /* The recovery step alone (Section 3.3, "Memory-Coalesced Tensor Recovery Kernel"): exponent bytes that
  * are already decompressed and sign+mantissa bytes, both in element order, are merged into bf16:

@@ -23,7 +23,8 @@ if not os.path.exists(LIB_PATH):
 
 _lib = ctypes.CDLL(LIB_PATH)
 
-DECODE_SHORT_CODES = 1      # zipmoe_decode flag: no code above 8 bits, max_record_bytes exact and <= 2048
+DECODE_SHORT_CODES = 1      # zipmoe_decode flag: no code above 8 bits, max_record_bytes exact and <= NARROW_RECORD_BYTES
+NARROW_RECORD_BYTES = 2080  # a tile record of 16 rows
 OK = 0
 ERR_INVALID_ARG, ERR_BAD_FORMAT, ERR_BUFFER_TOO_SMALL, ERR_CUDA, ERR_DECODE_CORRUPT, ERR_UNSUPPORTED = -1, -2, -3, -4, -5, -6
 LAYOUT_LINEAR, LAYOUT_BLOCKED = 0, 1
@@ -303,9 +304,9 @@ class DecodePlan:
         self.tables = np.concatenate(tables) if tables else np.zeros(0, np.uint8)
         self.n_chunks, self.n_tiles, self.n_tables = chunk_base, tile_base, len(blobs)
         self.max_record_bytes = int(self.descs["max_record_bytes"].max()) if self.n_chunks else 0
-        # what the fastest kernel variant wants promised: no code longer than 8 bits, no record longer than 2048 bytes
+        # what the fastest kernel variant wants promised: no code longer than 8 bits, no record higher than 16 rows
         self.max_code_len = int(self.tables.max()) if self.tables.size else 0
-        self.flags = DECODE_SHORT_CODES if (0 < self.max_record_bytes <= 2048 and self.max_code_len <= 8) else 0
+        self.flags = DECODE_SHORT_CODES if (0 < self.max_record_bytes <= NARROW_RECORD_BYTES and self.max_code_len <= 8) else 0
 
     def algorithmic_bytes(self):
         """Bytes one decode must move: E-chunk section + SM bytes read, bf16 written."""

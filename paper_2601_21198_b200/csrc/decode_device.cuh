@@ -18,24 +18,33 @@ namespace zipmoe_dev {
 //    by the next 8 code bits and replicated for each of the 32 lanes, entry
 //    (v, lane) at word v*32 + lane, so that lane l only ever touches bank l and
 //    the data-dependent lookups of a warp are free of bank conflicts;
-//  * any other code gets the wide table: u16 entries indexed by the next 12 bits.
-// Entry = (symbol << 7) | length in both.
+//  * any other code gets the wide table: one copy, indexed by the next 12 bits.
+// Entry = (symbol << 23) | length in both: the symbol sits where the exponent
+// field of the upper bf16 of a pair goes, the length in the low bits, and the
+// bits between are zero, so that sums of entries carry the sum of the lengths
+// in their low 23 bits whatever the symbols are.
 constexpr int kLaneLutBits = 8;
 constexpr int kLaneLutBytes = (1 << kLaneLutBits) * 32 * 4;   // 32 KB
 constexpr int kWideLutBits = ZIPMOE_MAX_CODE_LEN;
 constexpr int kWideLutEntries = 1 << kWideLutBits;
-constexpr int kWideLutBytes = kWideLutEntries * 2;            // 8 KB
+constexpr int kWideLutBytes = kWideLutEntries * 4;            // 16 KB
 constexpr int kLutBytes = kLaneLutBytes;                      // the wide table overlays the lane table
 constexpr int kLutScratchBytes = 256 + 16 * 4 + 8 * 16 * 4 + 256 * 2 + 256 * 4 + 16;
+constexpr uint32_t kEntrySymShift = 23;
+constexpr uint32_t kPosMask = (1u << kEntrySymShift) - 1;     // the bits of a sum of entries that count code bits
 
 constexpr uint32_t kStatusBadDescriptor = 1;  // a descriptor, offset or table points outside the buffers
-constexpr uint32_t kStatusBadBitCount = 2;    // a tile's lane bit counts overrun its record
+constexpr uint32_t kStatusBadRecord = 2;      // a tile record is not a column table and whole rows, or too high
 constexpr uint32_t kStatusWaitTimeout = 3;    // an asynchronous copy did not complete in time
 constexpr uint32_t kStatusBadTable = 4;       // code lengths do not form a complete prefix code
 constexpr uint32_t kStatusBrokenPromise = 5;  // ZIPMOE_DECODE_SHORT_CODES was given, yet a tile has longer codes or a longer record
+constexpr uint32_t kStatusCounterShared = 6;  // the work counter of a dynamically distributed launch is in use by another launch
 
-constexpr int kPayBuf = 2048;        // record bytes staged in shared memory; longer records are read from global
-constexpr int kPaySlack = 64;        // readable bytes after a staged record (a lane looks three words ahead)
+constexpr uint32_t kRecHead = 32;    // a record starts with the column of each lane's backward stream
+constexpr uint32_t kRowBytes = 128;  // then rows of one word per column
+constexpr uint32_t kMaxRows = 48;    // 128 codes of at most 12 bits per column
+constexpr int kPayBuf = kRecHead + 16 * kRowBytes;   // record bytes staged in shared memory by the narrow kernels (16 rows)
+constexpr int kPaySlack = kRowBytes; // readable bytes after a staged record (a lane reads the word under its position and the next)
 constexpr int kPayStage = kPayBuf + kPaySlack;
 
 __device__ __forceinline__ void report(uint32_t *status, uint32_t code) {
@@ -96,6 +105,11 @@ __device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
   asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
   return v;
 }
+__device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
 __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
   uint32_t v;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
@@ -116,10 +130,9 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
 // Returns the longest code length (0 for an invalid table).  An incomplete or
 // over-full code is reported and leaves zero entries in the holes: decoding
 // then yields garbage but stays in bounds.
-// lut_raw holds the lane table (u32 entries, or u16 entries when lane16) when the result is <= 8, the wide
-// table otherwise.
+// lut_raw holds the lane table when the result is <= 8, the wide table otherwise.
 __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint8_t *code_len, uint8_t *lut_raw,
-                                              uint8_t *scratch, uint32_t *status, const bool lane16 = false) {
+                                              uint8_t *scratch, uint32_t *status) {
   uint8_t *s_len = scratch;                                           // [256]
   uint32_t *s_first = reinterpret_cast<uint32_t *>(scratch + 256);    // [16] left-aligned 12-bit start of each length
   uint32_t *s_wcnt = s_first + 16;                                    // [8][16] per-warp symbol counts by length
@@ -127,7 +140,7 @@ __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint
   uint32_t *s_short = reinterpret_cast<uint32_t *>(s_start + 256);    // [256] lane-table entry of each 8-bit prefix
   uint32_t *s_max = s_short + 256;                                    // [1] longest length
   uint32_t *lane_lut = reinterpret_cast<uint32_t *>(lut_raw);
-  uint16_t *wide_lut = reinterpret_cast<uint16_t *>(lut_raw);
+  uint32_t *wide_lut = reinterpret_cast<uint32_t *>(lut_raw);
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   uint32_t len = 0;
@@ -170,10 +183,8 @@ __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint
     uint32_t start = s_first[len] + (rank << (kWideLutBits - len));
     s_start[tid] = (uint16_t)(start < (uint32_t)kWideLutEntries ? start : 0xFFFF);
   }
-  if (longest > (uint32_t)kLaneLutBits) {
-    uint32_t *w32 = reinterpret_cast<uint32_t *>(wide_lut);
-    for (uint32_t k = tid; k < (uint32_t)kWideLutEntries / 2; k += THREADS) w32[k] = 0;
-  }
+  if (longest > (uint32_t)kLaneLutBits)
+    for (uint32_t k = tid; k < (uint32_t)kWideLutEntries; k += THREADS) wide_lut[k] = 0;
   __syncthreads();
   // every symbol fills the range of windows its code is a prefix of
   for (uint32_t s = warp; s < 256; s += THREADS / 32) {
@@ -181,24 +192,18 @@ __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint
     if (!L) continue;
     const uint32_t start = s_start[s], n = 1u << (kWideLutBits - L);
     if (start == 0xFFFF || start + n > (uint32_t)kWideLutEntries) continue;
-    const uint32_t entry = (s << 7) | L;
+    const uint32_t entry = (s << kEntrySymShift) | L;
     if (L <= (uint32_t)kLaneLutBits) {
       const uint32_t n8 = n >> (kWideLutBits - kLaneLutBits), s8 = start >> (kWideLutBits - kLaneLutBits);
       for (uint32_t k = lane; k < n8; k += 32) s_short[s8 + k] = entry;
     }
     if (longest > (uint32_t)kLaneLutBits)
-      for (uint32_t k = lane; k < n; k += 32) wide_lut[start + k] = (uint16_t)entry;
+      for (uint32_t k = lane; k < n; k += 32) wide_lut[start + k] = entry;
   }
   __syncthreads();
   // replicate the 8-bit table once per lane
-  if (longest <= (uint32_t)kLaneLutBits) {
-    if (lane16) {
-      uint16_t *lane_lut16 = reinterpret_cast<uint16_t *>(lut_raw);
-      for (uint32_t k = tid; k < (1u << kLaneLutBits) * 32; k += THREADS) lane_lut16[k] = (uint16_t)s_short[k >> 5];
-    } else {
-      for (uint32_t k = tid; k < (1u << kLaneLutBits) * 32; k += THREADS) lane_lut[k] = s_short[k >> 5];
-    }
-  }
+  if (longest <= (uint32_t)kLaneLutBits)
+    for (uint32_t k = tid; k < (1u << kLaneLutBits) * 32; k += THREADS) lane_lut[k] = s_short[k >> 5];
   __syncthreads();
   return longest;
 }
@@ -221,7 +226,9 @@ struct LaunchArgs {
   uint32_t *status;
   uint64_t payload_bytes, sm_bytes, out_elems;
   uint32_t n_chunks, n_tiles, n_tables, tiles_per_cta;
-  uint32_t *work_counter;   // zeroed before the launch: next tile not yet handed to a CTA (dynamic distribution only)
+  uint32_t *work_counter;   // two words zeroed before the launch (dynamic distribution only): the next tile not yet
+                            // handed to a CTA, and the tag of the launch that uses the counter
+  uint32_t work_tag;
 };
 
 // Which descriptor holds global tile g: exact guess for launches whose chunks all hold the same number of tiles,
@@ -272,8 +279,9 @@ __device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c
   const uint64_t rec_off = pay_off + 16ull * o0;
   if (o1 <= o0) return w;
   w.rec_bytes = (o1 - o0) * 16u;
-  if (w.rec_bytes < 64 || w.rec_bytes > 64 + tile_elems / 8 * ZIPMOE_MAX_CODE_LEN + 32 * 8 + 16 ||   // codes, padding
-      rec_off + w.rec_bytes > a.payload_bytes)
+  // a record is the column table and 1..kMaxRows whole rows
+  if (w.rec_bytes < kRecHead + kRowBytes || w.rec_bytes > kRecHead + kMaxRows * kRowBytes ||
+      ((w.rec_bytes - kRecHead) & (kRowBytes - 1)) || rec_off + w.rec_bytes > a.payload_bytes)
     return w;
   w.iters = tile_elems >> 8;
   w.valid = (t == m - 1) ? last : tile_elems;
@@ -304,169 +312,100 @@ __device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) 
   return d;
 }
 
-// One sub-stream of a lane: a stream of u32 words of which the lane keeps two in
-// registers (`cur` holds the next code bit, `nxt` the bits after it) plus a third,
-// loaded one word early so that its latency is off the decode chain, and the
-// number `pos` of bits of `cur` already consumed (pos mod 64 < 32 between batches).
-//   DIR = +1 (forward sub-stream): words in ascending address order, each consumed
-//         from bit 31 down;
-//   DIR = -1 (backward sub-stream): words in descending address order, each consumed
-//         from bit 0 up.
-// window() returns the next 32 code bits with the first one in bit 31.
-template <bool STAGED, int DIR>
-struct SubStream {
-  uint32_t pos, cur, nxt, ahead;
-  uint32_t at_s;             // shared address of the next word to load (STAGED)
-  const uint32_t *at_g;      // global address of the next word to load (!STAGED)
-  const uint32_t *floor_g;   // the record's first word: a backward stream of a corrupt record stops here (!STAGED)
-
-  __device__ __forceinline__ uint32_t pop() {
-    if (STAGED) {
-      const uint32_t v = lds_u32(at_s);
-      at_s += (uint32_t)(4 * DIR);
-      return v;
-    }
-    const uint32_t v = __ldg(at_g);
-    at_g += DIR;
-    if (DIR < 0 && at_g < floor_g) at_g = floor_g;
-    return v;
-  }
-  // word = index of the word that holds the next code bit, counted from `words_s` / `words_g`
-  // (may be -1 for an empty backward stream at the very start of the bit area: the word before it exists)
-  __device__ __forceinline__ void start(uint32_t words_s, const uint32_t *words_g, const uint32_t *floor, int32_t word,
-                                        uint32_t consumed) {
-    at_s = words_s + 4 * word;
-    at_g = words_g + word;
-    floor_g = floor;
-    if (!STAGED && DIR < 0 && at_g < floor_g) at_g = floor_g;
-    pos = consumed;
-    cur = pop();
-    nxt = pop();
-    ahead = pop();
-  }
-  __device__ __forceinline__ uint32_t window() const {
-    if (DIR > 0) return __funnelshift_l(nxt, cur, pos);
-    return __brev(__funnelshift_r(cur, nxt, pos));
-  }
-  // If bit 5 of pos is set (a whole word has been consumed): cur <- nxt, nxt <- ahead, ahead <- the
-  // following word, clear the bit.  Predicated, no branch.
-  __device__ __forceinline__ void advance() {
-    if (STAGED) {
-      if (DIR > 0)
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
-            "and.b32 t, %0, 32;\n\t"
-            "setp.ne.u32 p, t, 0;\n\t"
-            "@p mov.b32 %1, %2;\n\t"
-            "@p mov.b32 %2, %3;\n\t"
-            "@p ld.shared.u32 %3, [%4];\n\t"
-            "@p add.u32 %4, %4, 4;\n\t"
-            "@p xor.b32 %0, %0, 32;\n\t}"
-            : "+r"(pos), "+r"(cur), "+r"(nxt), "+r"(ahead), "+r"(at_s));
-      else
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
-            "and.b32 t, %0, 32;\n\t"
-            "setp.ne.u32 p, t, 0;\n\t"
-            "@p mov.b32 %1, %2;\n\t"
-            "@p mov.b32 %2, %3;\n\t"
-            "@p ld.shared.u32 %3, [%4];\n\t"
-            "@p add.u32 %4, %4, -4;\n\t"
-            "@p xor.b32 %0, %0, 32;\n\t}"
-            : "+r"(pos), "+r"(cur), "+r"(nxt), "+r"(ahead), "+r"(at_s));
-    } else if (pos & 32u) {
-      cur = nxt;
-      nxt = ahead;
-      ahead = pop();
-      pos ^= 32u;
-    }
-  }
-};
-
-// One lane's view of a tile record: its two sub-streams of code bits and the
-// lookup table.  The record's bit area is a stream of u32 words; bit y of it is
-// bit 31 - (y mod 32) of word y / 32.  The lane's codes occupy the bit range
-// [S, E) (S = sum of the bit counts of the lanes before, E = S + the lane's own):
-//   sub-stream 0 (the lane's elements of even iterations) runs forwards from S,
-//   sub-stream 1 (odd iterations) runs backwards from E: its k-th bit is bit E-1-k.
-// The two are independent, so the lane decodes one code of each at a time and the
-// two lookup chains overlap.  A batch takes a stream's next 32 bits into one
-// register and decodes from its top:
-//   FAST  (no code longer than 8 bits): four codes per batch, looked up in the
-//         lane table with the top 8 bits;
-//   !FAST (codes up to 12 bits): two codes per batch, looked up in the wide
-//         table with the top 12 bits.
-// Whole table entries, (symbol << 7) | length, are added to a stream's pos: their
-// low 4 bits are the code length and bits 4..6 are zero, so the low 7 bits of pos
-// stay exact and the rest is ignored (the funnel shifts take the amount mod 32).
-// KIND: kLutWide (12-bit shared table), kLutLane32 (8-bit table, one u32 copy per lane: no bank conflicts, 32 KB) or
-// kLutLane16 (8-bit table, one u16 copy per lane: two lanes share a bank, 16 KB).
-constexpr int kLutWide = 0, kLutLane32 = 1, kLutLane16 = 2;
-
-template <bool STAGED, int KIND>
+// One lane's view of a tile record: the record is `rows` rows of 32 words (after a 32-byte column table); the
+// lane's forward stream is column `lane` read downwards from row 0, its backward stream the column the table names
+// read upwards from the last row.  Bit y of a column is bit 31 - y % 32 of its word in row y / 32; the forward
+// stream's k-th bit is column bit k, the backward stream's k-th bit is column bit 32 * rows - 1 - k.
+// A stream's whole state is the number of bits it has consumed.  For every batch of codes the lane loads the word
+// under its position and the one after it afresh: word r of all columns is one 128-byte row, so these loads of a
+// warp touch 32 different banks wherever the lanes are.  A batch takes the stream's next 32 bits into one register
+// and decodes from its top:
+//   FAST  (no code longer than 8 bits): four codes per batch, looked up in the lane table with the top 8 bits;
+//   !FAST (codes up to 12 bits): two codes per batch, looked up in the wide table with the top 12 bits.
+// Whole table entries, (symbol << 23) | length, are added to a position: the low 23 bits of the sum are the code
+// bits consumed, the rest is masked off.
+// STAGED: the record is in shared memory at rec_s; else it is read from global memory at rec_g (a record too
+// high for the kernel's record stages: correct, slow).
+template <bool STAGED, bool FAST>
 struct LaneDecoder {
-  static constexpr bool FAST = KIND != kLutWide;
-  SubStream<STAGED, +1> s0;
-  SubStream<STAGED, -1> s1;
+  uint32_t pos0, pos1;       // code bits consumed from the forward / backward stream
+  uint32_t col0, top1;       // STAGED: shared address of the forward column's row 0 / of the backward column's last row
+  const uint32_t *words_g;   // !STAGED: the record's rows in global memory
+  uint32_t lane_g, bcol_g, last_row;
   uint32_t lut, my_lut;
 
-  // record in shared memory at rec_s (STAGED) or in global memory at rec_g; lut =
-  // shared address of the lane table (FAST) or the wide table (!FAST).  Turns the
-  // record's 32 bit counts into this lane's range by a warp-shuffle prefix sum.
-  // Returns false (warp-uniform) if the counts overrun the record.
-  __device__ __forceinline__ bool init(uint32_t rec_s, const uint8_t *rec_g, uint32_t rec_bytes, uint32_t lut_addr,
+  __device__ __forceinline__ void init(uint32_t rec_s, const uint8_t *rec_g, uint32_t rec_bytes, uint32_t lut_addr,
                                        uint32_t lane) {
-    uint32_t my_bits;
-    if (STAGED) my_bits = lds_u16(rec_s + 2 * lane);
-    else my_bits = __ldg(reinterpret_cast<const uint16_t *>(rec_g) + lane);
-    uint32_t incl = my_bits;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-      if (lane >= (uint32_t)d) incl += t;
-    }
-    const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-    if (64u * 8u + total > rec_bytes * 8u) return false;
-    const uint32_t *floor = reinterpret_cast<const uint32_t *>(rec_g);
-    const uint32_t *words_g = floor + 16;
-    const uint32_t words_s = rec_s + 64;
-    const uint32_t S = incl - my_bits;
-    s0.start(words_s, words_g, floor, (int32_t)(S >> 5), S & 31u);
-    // the backward stream's next bit is bit incl - 1 (bit -1, in the word before the bit area, if the
-    // range is empty and starts at 0: nothing is decoded from it then)
-    const uint32_t y = incl + 31u;   // that bit, plus one word
-    s1.start(words_s, words_g, floor, (int32_t)(y >> 5) - 1, 31u - (y & 31u));
+    const uint32_t rows = (rec_bytes - kRecHead) / kRowBytes;
+    uint32_t bcol;
+    if (STAGED) bcol = lds_u8(rec_s + lane) & 31u;
+    else bcol = __ldg(rec_g + lane) & 31u;
+    col0 = rec_s + kRecHead + 4 * lane;
+    top1 = rec_s + kRecHead + (rows - 1) * kRowBytes + 4 * bcol;
+    words_g = reinterpret_cast<const uint32_t *>(rec_g + kRecHead);
+    lane_g = lane;
+    bcol_g = bcol;
+    last_row = rows - 1;
+    pos0 = pos1 = 0;
     lut = lut_addr;
-    my_lut = lut_addr + (KIND == kLutLane16 ? 2 : 4) * lane;
-    return true;
+    my_lut = lut_addr + 4 * lane;
   }
-  __device__ __forceinline__ uint32_t lookup(uint32_t w) const {   // (symbol << 7) | length of the code at the top of w
-    if (KIND == kLutLane32) return lds_u32(mad_u32(w >> (32 - kLaneLutBits), 128u, my_lut));
-    if (KIND == kLutLane16) return lds_u16(mad_u32(w >> (32 - kLaneLutBits), 64u, my_lut));
-    return lds_u16(mad_u32(w >> (32 - kWideLutBits), 2u, lut));
+  // the next 32 bits of the forward stream, the first one in bit 31
+  __device__ __forceinline__ uint32_t window0() const {
+    const uint32_t r = pos0 >> 5;
+    uint32_t c, n;
+    if (STAGED) {
+      const uint32_t a = mad_u32(r, kRowBytes, col0);
+      c = lds_u32(a);
+      n = lds_u32(a + kRowBytes);
+    } else {
+      c = __ldg(words_g + min(r, last_row) * 32 + lane_g);
+      n = __ldg(words_g + min(r + 1, last_row) * 32 + lane_g);
+    }
+    return __funnelshift_l(n, c, pos0);
+  }
+  // the next 32 bits of the backward stream, the first one in bit 31
+  __device__ __forceinline__ uint32_t window1() const {
+    const uint32_t r = pos1 >> 5;
+    uint32_t c, n;
+    if (STAGED) {
+      const uint32_t a = top1 - r * kRowBytes;
+      c = lds_u32(a);
+      n = lds_u32(a - kRowBytes);
+    } else {
+      c = __ldg(words_g + (last_row - min(r, last_row)) * 32 + bcol_g);
+      n = __ldg(words_g + (last_row - min(r + 1, last_row)) * 32 + bcol_g);
+    }
+    return __brev(__funnelshift_r(c, n, pos1));
+  }
+  __device__ __forceinline__ uint32_t lookup(uint32_t w) const {   // (symbol << 23) | length of the code at the top of w
+    if (FAST) return lds_u32(mad_u32(w >> (32 - kLaneLutBits), 128u, my_lut));
+    return lds_u32(mad_u32(w >> (32 - kWideLutBits), 4u, lut));
   }
   __device__ static __forceinline__ uint32_t next(uint32_t w, uint32_t entry) {   // drop the code just decoded
     return __funnelshift_l(0u, w, entry);
   }
-  // 8 exponent entries and 8 sign+mantissa bytes -> 8 bf16
+  // 8 table entries and 8 sign+mantissa bytes -> 8 bf16.  Bytes 2 and 3 of an entry are the symbol at the place
+  // of a bf16's exponent; two entries are packed by one byte permutation, the sign+mantissa bytes are spread to
+  // their places by another, and one logic operation joins them.
   __device__ static __forceinline__ uint4 merge(const uint2 smv, const uint32_t (&e)[8]) {
     constexpr uint32_t kKeep = 0x807F807Fu;   // sign and mantissa bits of two bf16
     uint4 o;
-    o.x = (__byte_perm(smv.x, 0, 0x1100) & kKeep) | (mad_u32(e[1], 65536u, e[0]) & ~kKeep);
-    o.y = (__byte_perm(smv.x, 0, 0x3322) & kKeep) | (mad_u32(e[3], 65536u, e[2]) & ~kKeep);
-    o.z = (__byte_perm(smv.y, 0, 0x1100) & kKeep) | (mad_u32(e[5], 65536u, e[4]) & ~kKeep);
-    o.w = (__byte_perm(smv.y, 0, 0x3322) & kKeep) | (mad_u32(e[7], 65536u, e[6]) & ~kKeep);
+    o.x = (__byte_perm(smv.x, 0, 0x1100) & kKeep) | __byte_perm(e[0], e[1], 0x7632);
+    o.y = (__byte_perm(smv.x, 0, 0x3322) & kKeep) | __byte_perm(e[2], e[3], 0x7632);
+    o.z = (__byte_perm(smv.y, 0, 0x1100) & kKeep) | __byte_perm(e[4], e[5], 0x7632);
+    o.w = (__byte_perm(smv.y, 0, 0x3322) & kKeep) | __byte_perm(e[6], e[7], 0x7632);
     return o;
   }
-  // The next 8 elements of both sub-streams (one group of an even iteration and one of the
-  // following odd iteration) merged with their sign+mantissa bytes.  The two decode chains are
-  // written interleaved so that each one's lookup latency is covered by the other's work.
+  // The next 8 elements of both streams (one group of an even iteration and one of the following odd
+  // iteration) merged with their sign+mantissa bytes.  The two decode chains are written interleaved so that
+  // each one's lookup latency is covered by the other's work.
   __device__ __forceinline__ void group2(const uint2 sm0, const uint2 sm1, uint4 &o0, uint4 &o1) {
     uint32_t e[8], f[8];
     if (FAST) {
 #pragma unroll
       for (int h = 0; h < 8; h += 4) {
-        uint32_t w = s0.window(), x = s1.window();
+        uint32_t w = window0(), x = window1();
         e[h] = lookup(w);
         f[h] = lookup(x);
         w = next(w, e[h]);
@@ -481,62 +420,51 @@ struct LaneDecoder {
         x = next(x, f[h + 2]);
         e[h + 3] = lookup(w);
         f[h + 3] = lookup(x);
-        s0.pos += (e[h] + e[h + 1]) + (e[h + 2] + e[h + 3]);
-        s1.pos += (f[h] + f[h + 1]) + (f[h + 2] + f[h + 3]);
-        s0.advance();
-        s1.advance();
+        pos0 = (pos0 + (e[h] + e[h + 1]) + (e[h + 2] + e[h + 3])) & kPosMask;
+        pos1 = (pos1 + (f[h] + f[h + 1]) + (f[h + 2] + f[h + 3])) & kPosMask;
       }
     } else {
 #pragma unroll
       for (int h = 0; h < 8; h += 2) {
-        uint32_t w = s0.window(), x = s1.window();
+        uint32_t w = window0(), x = window1();
         e[h] = lookup(w);
         f[h] = lookup(x);
         w = next(w, e[h]);
         x = next(x, f[h]);
         e[h + 1] = lookup(w);
         f[h + 1] = lookup(x);
-        s0.pos += e[h] + e[h + 1];
-        s1.pos += f[h] + f[h + 1];
-        s0.advance();
-        s1.advance();
+        pos0 = (pos0 + e[h] + e[h + 1]) & kPosMask;
+        pos1 = (pos1 + f[h] + f[h + 1]) & kPosMask;
       }
     }
     o0 = merge(sm0, e);
     o1 = merge(sm1, f);
   }
-  // one code of sub-stream WHICH
+  // one code of stream WHICH
   template <int WHICH>
   __device__ __forceinline__ uint32_t single() {
     uint32_t e;
     if (WHICH == 0) {
-      e = lookup(s0.window());
-      s0.pos += e;
-      s0.advance();
+      e = lookup(window0());
+      pos0 = (pos0 + e) & kPosMask;
     } else {
-      e = lookup(s1.window());
-      s1.pos += e;
-      s1.advance();
+      e = lookup(window1());
+      pos1 = (pos1 + e) & kPosMask;
     }
     return e;
   }
-  // the next 8 elements of sub-stream WHICH alone (the ragged end of a tensor)
+  // the next 8 elements of stream WHICH alone (the ragged end of a tensor)
   template <int WHICH>
   __device__ __forceinline__ uint4 group1(const uint2 smv) {
     uint32_t e[8];
 #pragma unroll
     for (int h = 0; h < 8; h += 2) {
-      uint32_t w = WHICH == 0 ? s0.window() : s1.window();
+      uint32_t w = WHICH == 0 ? window0() : window1();
       e[h] = lookup(w);
       w = next(w, e[h]);
       e[h + 1] = lookup(w);
-      if (WHICH == 0) {
-        s0.pos += e[h] + e[h + 1];
-        s0.advance();
-      } else {
-        s1.pos += e[h] + e[h + 1];
-        s1.advance();
-      }
+      if (WHICH == 0) pos0 = (pos0 + e[h] + e[h + 1]) & kPosMask;
+      else pos1 = (pos1 + e[h] + e[h + 1]) & kPosMask;
     }
     return merge(smv, e);
   }
@@ -551,16 +479,15 @@ struct LaneDecoder {
 //   output  : sink.group(i, lane, v) takes the 8 bf16 of iteration i, lane;
 //             sink.elem(i, lane, j, v) one bf16 of the short last group of a
 //             linear tensor.
-// Returns 0 on success, else a status code (warp-uniform); on
-// kStatusBadBitCount nothing has been written.
+// Returns 0 on success, else a status code (warp-uniform).
 // SMALL: also an unrolled path for small full tiles (kept out of the instantiation that never sees any: it would
 // only lengthen its code).
 template <bool STAGED, bool FAST, bool SMALL, class Feed, class Sink>
 __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *rec_g, uint32_t rec_bytes,
                                                 uint32_t lut, uint32_t valid, uint32_t iters,
                                                 uint32_t lane, Feed &feed, Sink &sink) {
-  LaneDecoder<STAGED, FAST ? kLutLane32 : kLutWide> dec;
-  if (!dec.init(rec_s, rec_g, rec_bytes, lut, lane)) return kStatusBadBitCount;
+  LaneDecoder<STAGED, FAST> dec;
+  dec.init(rec_s, rec_g, rec_bytes, lut, lane);
   static_assert(kPieceIters % 2 == 0, "a piece holds whole pairs of iterations");
 
   const uint32_t pieces = sm_pieces_of_tile(valid);   // pieces that exist: iterations past them hold no element
@@ -611,7 +538,7 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
         const uint32_t e = dec.template single<WHICH>();
         const uint32_t at = sm_at + j;
         const uint32_t smb = (lds_u32(at & ~3u) >> (8 * (at & 3u))) & 0xFFu;
-        sink.elem(i, lane, j, (uint16_t)(((smb & 0x80u) << 8) | (e & 0x7F80u) | (smb & 0x7Fu)));
+        sink.elem(i, lane, j, (uint16_t)(((smb & 0x80u) << 8) | ((e >> 16) & 0x7F80u) | (smb & 0x7Fu)));
       }
     }
   };

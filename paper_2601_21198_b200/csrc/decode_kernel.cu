@@ -7,7 +7,7 @@
 // decompressed exponents never reach global memory.
 //
 // Data movement per tile (256*I elements):
-//   global -> shared : the tile record (sub-stream bit counts + code bits) by
+//   global -> shared : the tile record (column table + rows of code words) by
 //                      one bulk asynchronous copy (cp.async.bulk, completion
 //                      on an mbarrier), one tile ahead of the decode; the
 //                      tile's sign+mantissa bytes as two 2 KB pieces through
@@ -34,12 +34,11 @@ constexpr int kPayStages = 2;
 constexpr int kBarsPerWarp = kPayStages + kSmPieces;   // two record stages, one barrier per sign+mantissa slot
 
 // Two instantiations of the kernel, chosen by the host from the launch's largest tile record:
-//   WIDE = false: record stages of kPayStage bytes (records of up to 2048 bytes: every tensor whose codes average
-//                 less than ~3.9 bits), 16 warps per CTA;
-//   WIDE = true : record stages of 4352 bytes (records of up to 4288 bytes: 8-bit codes everywhere plus the word of
-//                 padding per lane that the encoder gives such tiles, e.g. tensors with near-uniform exponents),
-//                 one warp fewer so that the stages still fit.
-// A record longer than its stage is read from global memory word by word (correct, slow).
+//   WIDE = false: record stages of kPayStage bytes (records of up to 16 rows: every tensor whose codes average
+//                 less than ~4 bits), 16 warps per CTA;
+//   WIDE = true : record stages for records of up to 32 rows (8-bit codes everywhere, e.g. tensors with
+//                 near-uniform exponents), one warp fewer so that the stages still fit.
+// A record higher than its stage is read from global memory word by word (correct, slow).
 template <bool WIDE>
 struct Cfg {
 #ifndef ZIPMOE_CTAS_PER_SM
@@ -48,7 +47,7 @@ struct Cfg {
   static constexpr int kCtasPerSm = WIDE ? 1 : ZIPMOE_CTAS_PER_SM;
   static constexpr int kWarps = WIDE ? ZIPMOE_WARPS - 1 : ZIPMOE_WARPS / kCtasPerSm;   // warps per CTA
   static constexpr int kThreads = kWarps * 32;
-  static constexpr int kStage = WIDE ? 64 + 4096 + 32 * 4 + kPaySlack : kPayStage;   // bytes of a record stage
+  static constexpr int kStage = WIDE ? (int)(kRecHead + 32 * kRowBytes) + kPaySlack : kPayStage;   // bytes of a record stage
   static constexpr int kBuf = kStage - kPaySlack;                         // longest staged record
   static constexpr int kWarpBytes = kPayStages * kStage + kSmPieces * kSmPieceBytes;
   static constexpr int kSmemBytes = kLutBytes + kWarps * kWarpBytes + kWarps * kBarsPerWarp * 8 + kLutScratchBytes;
@@ -217,12 +216,33 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
   if (BATCHED) {
     __syncthreads();   // s_grab of the previous round has been read by every thread
     if (tid == 0) {
-      const uint32_t seen = *reinterpret_cast<volatile uint32_t *>(a.work_counter);
-      uint32_t take = seen < a.n_tiles ? (a.n_tiles - seen) / (ZIPMOE_GRAB_DIV * gridDim.x) : 0;
-      take = max(take, max(1u, min(kMinGrab, a.n_tiles / gridDim.x)));   // small launches: spread over all CTAs
-      const uint32_t first = atomicAdd(a.work_counter, take);
+      // The counter is one 64-bit word: the tag of the launch that owns it above the next tile not yet handed out.
+      // It was zeroed on the stream before this kernel; the first range taken installs the tag in the same atomic
+      // step.  Should two launches ever be given the same counter while both are in flight (more of them queued
+      // than the ring has slots), one of them finds the other's tag: it reports that and takes no more tiles,
+      // and the other is not disturbed -- nothing is skipped silently.
+      unsigned long long *ctr = reinterpret_cast<unsigned long long *>(a.work_counter);
+      uint32_t first = a.n_tiles, take = 0;
+      for (uint32_t tries = 0; tries < (1u << 16); ++tries) {
+        const unsigned long long old = *reinterpret_cast<volatile unsigned long long *>(ctr);
+        const uint32_t tag = (uint32_t)(old >> 32), seen = (uint32_t)old;
+        if (tag != 0u && tag != a.work_tag) {
+          report(a.status, kStatusCounterShared);
+          break;
+        }
+        if (seen >= a.n_tiles) break;   // all handed out
+        uint32_t want = (a.n_tiles - seen) / (ZIPMOE_GRAB_DIV * gridDim.x);
+        want = max(want, max(1u, min(kMinGrab, a.n_tiles / gridDim.x)));   // small launches: spread over all CTAs
+        want = min(want, a.n_tiles - seen);
+        const unsigned long long next = ((unsigned long long)a.work_tag << 32) | (seen + want);
+        if (atomicCAS(ctr, old, next) == old) {
+          first = seen;
+          take = want;
+          break;
+        }
+      }
       s_grab[0] = first;
-      s_grab[1] = first < a.n_tiles ? min(a.n_tiles - first, take) + first : first;
+      s_grab[1] = first + take;
     }
     __syncthreads();
     g0 = s_grab[0];
@@ -340,7 +360,7 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
           dead = true;
           break;
         }
-        if (rc == kStatusBadBitCount || rc == kStatusBrokenPromise) {
+        if (rc == kStatusBrokenPromise) {
           // nothing was decoded: take the tile's sign+mantissa pieces off the barriers
           report(a.status, rc);
           for (uint32_t p = 0; p < cur.pieces && !dead; ++p)
@@ -376,7 +396,7 @@ namespace {
 // word per launch, zeroed on the launch's stream right before the kernel.  A slot comes round again after
 // kCounterSlots launches of that kind; by then the launch that had it has long finished.
 constexpr uint32_t kCounterSlots = 1024;
-static __device__ uint32_t g_work_counters[kCounterSlots];
+static __device__ unsigned long long g_work_counters[kCounterSlots];   // per slot: tag of the owning launch << 32 | next tile
 std::atomic<uint32_t> g_next_slot{0};
 
 struct DeviceInfo {
@@ -457,9 +477,12 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
   // CTA; else tiles resolved 32 at a time and handed to the CTAs dynamically (one CTA per SM either way)
   const bool batched = (uint64_t)n_tiles < 512ull * n_tables;
   a.work_counter = nullptr;
+  a.work_tag = 0;
   if (batched) {
-    a.work_counter = counters + (g_next_slot.fetch_add(1) % kCounterSlots);
-    if (cudaMemsetAsync(a.work_counter, 0, sizeof(uint32_t), st) != cudaSuccess) return ZIPMOE_ERR_CUDA;
+    const uint32_t seq = g_next_slot.fetch_add(1);
+    a.work_counter = counters + 2 * (seq % kCounterSlots);
+    a.work_tag = seq | 0x80000000u;   // never zero; differs between any two launches that can meet on a slot
+    if (cudaMemsetAsync(a.work_counter, 0, 8, st) != cudaSuccess) return ZIPMOE_ERR_CUDA;
     ctas = (uint32_t)sms * (narrow ? zipmoe_dev::Cfg<false>::kCtasPerSm : 1u);
     const uint32_t most = (n_tiles + 15 - 1) / 15;   // a tile per warp at least
     if (ctas > most) ctas = most;

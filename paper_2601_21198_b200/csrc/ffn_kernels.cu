@@ -24,8 +24,8 @@
 //   * one MMA warp per group waits for the group's half to be complete and
 //     issues its 16 MMAs (K = 16 each; B = the activations, N = token rows);
 //     accumulators live in tensor memory, one [64 x N] fp32 block per group and half;
-//   * one loader warp stages the activations of the current K step (token rows
-//     x 256 bf16) in a two-stage ring shared by all groups;
+//   * one loader warp stages the activations in half K steps (token rows x 128
+//     bf16) in a three-stage ring shared by all groups;
 //   * at the end four warps read the accumulators back (tcgen05.ld) and store Y.
 // The host wrapper runs it for W1 and W3 (gate, up), applies SiLU(g)*u, runs it
 // for W2, and combines the experts of every token.
@@ -56,10 +56,9 @@ constexpr int kFfnMaxThreads = (kFfnMaxWarps + kFfnGroups + 1) * 32;            
 constexpr uint32_t kBLbo = 144;                          // bytes between the 8x8 cores of a half-tile along K: 128 + 16 of
                                                          // padding, so that the 32 lanes' 16-byte stores spread over all banks
 constexpr uint32_t kBBufBytes = 32 * kBLbo;              // one half-tile: 8 rows x 256 columns
-constexpr uint32_t kXGroupBytes = 4096;                  // 8 token rows x 256 columns of bf16, cores 128 bytes apart
+constexpr uint32_t kXGroupBytes = 2048;                  // 8 token rows x 128 columns of bf16, cores 128 bytes apart
+constexpr uint32_t kXStages = 3;                         // half K steps in the activation ring: one whole step and half of the next
 constexpr uint32_t kFfnWarpBytes = 2 * kPayStage + kBBufBytes;   // two record stages, one half-tile buffer
-constexpr uint32_t kFfnLutBytes = kLaneLutBytes / 2;     // u16 lane table (two lanes per bank): the fused kernel spends its
-                                                         // shared memory on decode warps rather than on the table
 constexpr uint32_t kFfnShortTries = 1u << 10;            // wait limit once something has already gone wrong
 
 struct FfnArgs {
@@ -101,11 +100,11 @@ __host__ __device__ inline void ffn_job_parts(uint64_t job, uint32_t steps, uint
 
 // shared-memory layout: [X stages][per-warp buffers][tables][table scratch][barriers][tmem slot]
 __host__ __device__ inline uint32_t ffn_bar_count(uint32_t n_warps) {
-  return 2 * n_warps + 2 * ((n_warps + kGroupWarps - 1) / kGroupWarps) + 4;   // the word after them is the CTA's give-up flag
+  return 2 * n_warps + 2 * ((n_warps + kGroupWarps - 1) / kGroupWarps) + 2 * kXStages;   // the word after them is the CTA's give-up flag
 }
-__host__ __device__ inline uint32_t ffn_smem_bytes(uint32_t n_warps, uint32_t groups, bool lane16) {
-  const uint32_t after_warps = (lane16 ? kFfnLutBytes : (uint32_t)kLutBytes) + kLutScratchBytes + ffn_bar_count(n_warps) * 8 + 16;
-  return 2 * groups * kXGroupBytes + n_warps * kFfnWarpBytes + after_warps;
+__host__ __device__ inline uint32_t ffn_smem_bytes(uint32_t n_warps, uint32_t groups) {
+  const uint32_t after_warps = (uint32_t)kLutBytes + kLutScratchBytes + ffn_bar_count(n_warps) * 8 + 16;
+  return kXStages * groups * kXGroupBytes + n_warps * kFfnWarpBytes + after_warps;
 }
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -144,9 +143,8 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-template <bool LANE16>
 __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const FfnArgs a) {
-  constexpr uint32_t kMyLutBytes = LANE16 ? kFfnLutBytes : kLutBytes;
+  constexpr uint32_t kMyLutBytes = kLutBytes;
   extern __shared__ __align__(128) uint8_t smem[];
   const uint32_t NW = a.n_warps, G = a.groups, Q = (NW + kGroupWarps - 1) / kGroupWarps, NCOL = 8 * G;
   // accumulator columns per group and half = N of the MMAs: with M = 128, N is a multiple of 16 (for up to 8 token
@@ -165,17 +163,17 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   uint32_t u = (uint32_t)ffn_first_unit(blockIdx.x, U, P);
   const uint32_t u_end = (uint32_t)ffn_first_unit(blockIdx.x + 1, U, P);
 
-  uint8_t *x_raw = smem;                                   // [2][G][4096]
-  uint8_t *warp_raw = x_raw + 2 * G * kXGroupBytes;        // [NW][2 record stages | half-tile buffer]
+  uint8_t *x_raw = smem;                                   // [kXStages][G][2048]
+  uint8_t *warp_raw = x_raw + kXStages * G * kXGroupBytes; // [NW][2 record stages | half-tile buffer]
   uint8_t *lut_raw = warp_raw + NW * kFfnWarpBytes;
   uint8_t *lut_scratch = lut_raw + kMyLutBytes;
   uint64_t *bars = reinterpret_cast<uint64_t *>(lut_scratch + kLutScratchBytes);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + ffn_bar_count(NW));
   volatile uint32_t *give_up = tmem_slot + 1;              // set once a wait ran out: the CTA stops after the piece
-  // barriers: [NW][2] record stages, [Q] group's half written, [Q] group's MMAs done, [2] X full, [2] X empty
+  // barriers: [NW][2] record stages, [Q] group's half written, [Q] group's MMAs done, [3] X full, [3] X empty
   const uint32_t bar0 = smem_addr(bars);
   const uint32_t quad_full = bar0 + 8 * (2 * NW), quad_done = quad_full + 8 * Q;
-  const uint32_t x_full = quad_done + 8 * Q, x_empty = x_full + 16;
+  const uint32_t x_full = quad_done + 8 * Q, x_empty = x_full + 8 * kXStages;
   const uint32_t x_addr = smem_addr(x_raw), lut = smem_addr(lut_raw);
   const bool is_decode = warp < NW, is_mma = warp >= NW && warp < NW + Q, is_loader = warp == NW + Q;
 
@@ -187,10 +185,10 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
       mbar_init(quad_full + 8 * q, min((uint32_t)kGroupWarps, NW - q * kGroupWarps));   // the group's decode warps
       mbar_init(quad_done + 8 * q, 1);
     }
-    mbar_init(x_full, 1);
-    mbar_init(x_full + 8, 1);
-    mbar_init(x_empty, Q);
-    mbar_init(x_empty + 8, Q);
+    for (uint32_t b = 0; b < kXStages; ++b) {
+      mbar_init(x_full + 8 * b, 1);
+      mbar_init(x_empty + 8 * b, Q);
+    }
     *give_up = 0;
   }
   fence_barrier_init();
@@ -217,7 +215,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   const uint32_t rec_bar = bar0 + 8 * (2 * (is_decode ? warp : 0));
   uint32_t rec_phase = 0, stage = 0;   // decode warp: parity of its two record stages, the stage of its next tile
   uint32_t hn = 0;                     // decode and MMA warps: halves the group has handed over so far
-  uint32_t xs = 0;                     // loader and MMA warps: K steps staged / consumed so far
+  uint32_t xst = 0, xround = 0;        // loader and MMA warps: ring stage of the next half K step, times the ring has gone round
   uint32_t lut_tensor = 0xFFFFFFFFu;   // the tensor whose table is in shared memory
   bool fast = true;
 
@@ -285,7 +283,8 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
         }
         const uint32_t *tab = reinterpret_cast<const uint32_t *>(a.la.payload + pay_off);
         const uint32_t o0 = __ldg(tab + t), o1 = __ldg(tab + t + 1);
-        if (o1 <= o0 || o1 - o0 < 4 || o1 - o0 > (64 + ZIPMOE_TILE_ELEMS_MAX / 8 * ZIPMOE_MAX_CODE_LEN + 32 * 8) / 16 + 1 ||
+        // a record is the column table (2 units of 16 bytes) and 1..kMaxRows rows (8 units each)
+        if (o1 <= o0 || o1 - o0 < 10 || o1 - o0 > 2 + 8 * kMaxRows || ((o1 - o0 - 2) & 7u) ||
             pay_off + 16ull * o1 > a.la.payload_bytes) {
           bad = true;
           continue;
@@ -326,32 +325,31 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
     }
 
     if (tensor != lut_tensor) {   // (every warp is done with the previous table: a piece ends with CTA barriers)
-      fast = build_lut(blockDim.x, a.la.tables[table_id].code_len, lut_raw, lut_scratch, a.la.status, LANE16) <=
+      fast = build_lut(blockDim.x, a.la.tables[table_id].code_len, lut_raw, lut_scratch, a.la.status) <=
              (uint32_t)kLaneLutBits;
       lut_tensor = tensor;
     }
 
     if (is_loader) {
-      // ---- activations: one K step (8G token rows x 256 columns) per stage ----
-      for (uint32_t s = 0; s < n_steps; ++s, ++xs) {
-        const uint32_t b = xs & 1, n = xs >> 1;
-        if (n > 0 && !mbar_wait_bounded(x_empty + 8 * b, (n - 1) & 1)) {
+      // ---- activations: half a K step (8G token rows x 128 columns) per stage ----
+      for (uint32_t hs = 0; hs < 2 * n_steps; ++hs) {
+        if (xround > 0 && !mbar_wait_bounded(x_empty + 8 * xst, (xround - 1) & 1)) {
           report(a.la.status, kStatusWaitTimeout);
           *give_up = 1;
           break;
         }
-        const uint32_t xstage = x_addr + b * G * kXGroupBytes;
+        const uint32_t xstage = x_addr + xst * G * kXGroupBytes;
         for (uint32_t row = lane; row < NCOL; row += 32) {
           const uint16_t *src = a.x;
           uint32_t src_bytes = 0;   // rows past the expert's last slot are filled with zeros
           if (row < Te) {
             const uint32_t xr = a.slot_token ? __ldg(a.slot_token + off + row) : off + row;
-            src = a.x + (size_t)xr * a.K + (size_t)(s0 + s) * 256;
+            src = a.x + (size_t)xr * a.K + (size_t)(2 * s0 + hs) * 128;
             src_bytes = 16;
           }
           const uint32_t dst = xstage + (row >> 3) * kXGroupBytes + (row & 7) * 16;
 #pragma unroll 8
-          for (uint32_t k8 = 0; k8 < 32; ++k8)
+          for (uint32_t k8 = 0; k8 < 16; ++k8)
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + k8 * 128),
                          "l"(src + (src_bytes ? k8 * 8 : 0)), "r"(src_bytes)
                          : "memory");
@@ -359,7 +357,11 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
         asm volatile("cp.async.wait_all;" ::: "memory");
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(x_full + 8 * b);
+        if (lane == 0) mbar_arrive(x_full + 8 * xst);
+        if (++xst == kXStages) {
+          xst = 0;
+          ++xround;
+        }
       }
     } else if (is_mma) {
       // ---- one MMA warp per group; one lane issues, per half-tile: D[64 x N] (+)= A[64 x 256] * X[N x 256]^T ----
@@ -368,10 +370,15 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
       const uint32_t abuf = smem_addr(warp_raw) + 2 * kPayStage + kGroupWarps * q * kFfnWarpBytes;
       const uint64_t a_desc0 = smem_desc(abuf, kBLbo, kFfnWarpBytes);
       bool alive = true;
-      for (uint32_t s = 0; s < n_steps && alive; ++s, ++xs) {
-        const uint32_t xb = xs & 1;
-        const uint64_t b_desc0 = smem_desc(x_addr + xb * G * kXGroupBytes, 128, kXGroupBytes);
-        if (!mbar_wait_bounded(x_full + 8 * xb, (xs >> 1) & 1)) alive = false;
+      for (uint32_t s = 0; s < n_steps && alive; ++s) {
+        // the step's two half steps of activations: ring stages xst and the one after it
+        const uint32_t st0 = xst, rd0 = xround;
+        const uint32_t st1 = st0 + 1 == kXStages ? 0 : st0 + 1, rd1 = st0 + 1 == kXStages ? rd0 + 1 : rd0;
+        xst = st1 + 1 == kXStages ? 0 : st1 + 1;
+        xround = st1 + 1 == kXStages ? rd1 + 1 : rd1;
+        const uint64_t b_desc0 = smem_desc(x_addr + st0 * G * kXGroupBytes, 128, kXGroupBytes);
+        const uint64_t b_desc1 = smem_desc(x_addr + st1 * G * kXGroupBytes, 128, kXGroupBytes);
+        if (!mbar_wait_bounded(x_full + 8 * st0, rd0 & 1) || !mbar_wait_bounded(x_full + 8 * st1, rd1 & 1)) alive = false;
         for (uint32_t half = 0; half < 2 && alive; ++half, ++hn) {
           if (!mbar_wait_bounded(quad_full + 8 * q, hn & 1)) {
             alive = false;
@@ -383,9 +390,13 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
             // the K slice j of an operand starts 2 cores further: the start-address field counts 16-byte units
 #pragma unroll
             for (uint32_t j = 0; j < 16; ++j)
-              mma_bf16(d_tmem, a_desc0 + j * (2 * kBLbo / 16), b_desc0 + j * (256 / 16), idesc, (s > 0 || j > 0) ? 1u : 0u);
+              mma_bf16(d_tmem, a_desc0 + j * (2 * kBLbo / 16), (j < 8 ? b_desc0 : b_desc1) + (j & 7) * (256 / 16), idesc,
+                       (s > 0 || j > 0) ? 1u : 0u);
             mma_commit(quad_done + 8 * q);
-            if (half == 1) mma_commit(x_empty + 8 * xb);   // this group is done with the X stage
+            if (half == 1) {   // this group is done with the step's two X stages
+              mma_commit(x_empty + 8 * st0);
+              mma_commit(x_empty + 8 * st1);
+            }
           }
           __syncwarp();
         }
@@ -431,15 +442,8 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
           }
           // both halves of the tile, for every combination of record location and table kind
           auto run = [&](auto staged_c, auto fast_c) -> bool {
-            LaneDecoder<decltype(staged_c)::value, !decltype(fast_c)::value ? kLutWide : LANE16 ? kLutLane16 : kLutLane32> dec;
-            if (!dec.init(my + stage * kPayStage, cur.rec, cur.rec_bytes, lut, lane)) {
-              report(a.la.status, kStatusBadBitCount);
-              buffer_free();
-              publish();   // keep the count of halves
-              buffer_free();
-              publish();
-              return false;
-            }
+            LaneDecoder<decltype(staged_c)::value, decltype(fast_c)::value> dec;
+            dec.init(my + stage * kPayStage, cur.rec, cur.rec_bytes, lut, lane);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
               // Sign+mantissa bytes: sm[k] holds row k of the half being decoded; as soon as a row has been
@@ -672,7 +676,6 @@ struct FfnPlan {
   uint32_t groups_gu, groups_dn;     // strip groups per matrix
   uint32_t min_gu, min_dn;           // smallest share of a CTA, in K steps
   uint32_t parts_gu, parts_dn;       // bound on the partial sums of a job
-  bool lane16;
   uint64_t off_offsets, off_active, off_slot_token, off_slot_of, off_slot_active, off_gu, off_h, off_y, total;
 };
 
@@ -696,14 +699,13 @@ zipmoe_status make_plan(uint32_t T, uint32_t k, const zipmoe_compressed_experts 
   p->S = T * k;
   p->groups = (T + 7) / 8;
   p->grid = grid;
-  // as many decode warps as fit; the 32 KB conflict-free table if it still fits beside them, else the 16 KB one
+  // as many decode warps as fit beside the activation ring and the lookup table
   uint32_t nw = zipmoe_dev::kFfnMaxWarps;
-  p->lane16 = zipmoe_dev::ffn_smem_bytes(nw, p->groups, false) > 227u * 1024u;
-  while (nw > (uint32_t)zipmoe_dev::kGroupWarps && zipmoe_dev::ffn_smem_bytes(nw, p->groups, p->lane16) > 227u * 1024u)
+  while (nw > (uint32_t)zipmoe_dev::kGroupWarps && zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u)
     nw -= zipmoe_dev::kGroupWarps;
-  if (zipmoe_dev::ffn_smem_bytes(nw, p->groups, p->lane16) > 227u * 1024u) return ZIPMOE_ERR_UNSUPPORTED;
+  if (zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) return ZIPMOE_ERR_UNSUPPORTED;
   p->n_warps = nw;
-  p->smem = zipmoe_dev::ffn_smem_bytes(nw, p->groups, p->lane16);
+  p->smem = zipmoe_dev::ffn_smem_bytes(nw, p->groups);
   const uint32_t steps_gu = ex->hidden / 256, steps_dn = ex->inter / 256;
   p->groups_gu = (ex->inter / 16 + nw - 1) / nw;
   p->groups_dn = (ex->hidden / 16 + nw - 1) / nw;
@@ -779,10 +781,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
     int major = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ZIPMOE_ERR_CUDA;
     if (major != 10) return ZIPMOE_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(ffn_matmul_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-            cudaSuccess ||
-        cudaFuncSetAttribute(ffn_matmul_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-            cudaSuccess)
+    if (cudaFuncSetAttribute(ffn_matmul_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return ZIPMOE_ERR_CUDA;
     g_ffn_ready[dev] = true;
   }
@@ -816,6 +815,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.la.n_tables = ex->n_tables;
   a.la.tiles_per_cta = 0;
   a.la.work_counter = nullptr;
+  a.la.work_tag = 0;
   a.tensor_first_chunk = ex->tensor_first_chunk;
   a.expert_offset = expert_offset;
   a.active = active;
@@ -841,8 +841,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.n_groups = p.groups_gu;
   a.min_units = p.min_gu;
   a.max_parts = p.parts_gu;
-  if (p.lane16) ffn_matmul_kernel<true><<<p.grid, threads, p.smem, stream>>>(a);
-  else ffn_matmul_kernel<false><<<p.grid, threads, p.smem, stream>>>(a);
+  ffn_matmul_kernel<<<p.grid, threads, p.smem, stream>>>(a);
 
   po.n_mats = 2;
   po.n_groups = p.groups_gu;
@@ -862,8 +861,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.n_groups = p.groups_dn;
   a.min_units = p.min_dn;
   a.max_parts = p.parts_dn;
-  if (p.lane16) ffn_matmul_kernel<true><<<p.grid, threads, p.smem, stream>>>(a);
-  else ffn_matmul_kernel<false><<<p.grid, threads, p.smem, stream>>>(a);
+  ffn_matmul_kernel<<<p.grid, threads, p.smem, stream>>>(a);
 
   po.n_mats = 1;
   po.n_groups = p.groups_dn;

@@ -1,4 +1,4 @@
-// Internal view of the ZMOE v2 container shared by the library's host code
+// Internal view of the ZMOE v3 container shared by the library's host code
 // (encoder, validator, planner).  Device code does not include this file: the
 // kernels see only zipmoe_chunk_desc / zipmoe_table from the public header.
 #pragma once
@@ -10,14 +10,16 @@
 namespace zipmoe {
 
 constexpr uint32_t kMagic = 0x454F4D5Au;
-constexpr uint32_t kVersion = 2;
+constexpr uint32_t kVersion = 3;
 constexpr uint64_t kHeaderBytes = 64;
 constexpr uint64_t kTableOff = 64;
 constexpr uint64_t kChunkOffOff = 320;
 constexpr uint32_t kLanes = 32;
 constexpr uint32_t kGroup = 8;          // elements per lane per iteration
 constexpr uint32_t kIterElems = 256;    // kLanes * kGroup
-constexpr uint32_t kRecordHeadBytes = 64;  // u16 sub_bits[32]: code bits of each lane (both sub-streams together)
+constexpr uint32_t kRecordHeadBytes = 32;  // u8 bcol[32]: the column that holds each lane's backward stream
+constexpr uint32_t kRowBytes = 128;        // one word of each of the 32 columns
+constexpr uint32_t kMaxRows = 48;          // a column holds at most 128 codes of at most 12 bits
 
 inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 

@@ -61,9 +61,7 @@ zipmoe_status resolve_opts(const zipmoe_encode_opts *o, Opts *r) {
   return ZIPMOE_OK;
 }
 
-uint64_t tile_record_max(uint32_t tile_elems) {
-  return align_up(kRecordHeadBytes + (uint64_t)tile_elems * ZIPMOE_MAX_CODE_LEN / 8 + kLanes * 8, 16);   // codes + padding
-}
+uint64_t tile_record_max(uint32_t) { return kRecordHeadBytes + (uint64_t)kMaxRows * kRowBytes; }
 
 // Huffman code lengths by the usual greedy merge on a min-heap.  When the tree
 // is deeper than `limit` the rare symbols' counts are flattened (halved,
@@ -122,38 +120,33 @@ void canonical_codes(const uint8_t *len, uint32_t *code) {
   for (int s = 0; s < 256; ++s) code[s] = len[s] ? next[len[s]]++ : 0;
 }
 
-// the low n bits of v in reverse order
-inline uint32_t reverse_bits(uint32_t v, uint32_t n) {
-  uint32_t r = 0;
-  for (uint32_t b = 0; b < n; ++b) r |= ((v >> b) & 1u) << (n - 1 - b);
-  return r;
-}
-
-// Appends codes to a u32 word stream, most significant bit of each word first.
+// Appends codes to a word stream, most significant bit of each word first.
 struct BitWriter {
-  uint8_t *dst;
+  uint32_t *dst;
   uint64_t acc = 0;   // pending bits, right-aligned
   uint32_t fill = 0;  // number of pending bits (< 32 between calls)
-  uint64_t total = 0;
-  explicit BitWriter(uint8_t *p) : dst(p) {}
+  explicit BitWriter(uint32_t *p) : dst(p) {}
   void put(uint32_t code, uint32_t nbits) {
     acc = (acc << nbits) | code;
     fill += nbits;
-    total += nbits;
     if (fill >= 32) {
       fill -= 32;
-      store_le<uint32_t>(dst, (uint32_t)(acc >> fill));
-      dst += 4;
+      *dst++ = (uint32_t)(acc >> fill);
     }
   }
   void flush() {
-    if (fill) {
-      store_le<uint32_t>(dst, (uint32_t)(acc << (32 - fill)));
-      dst += 4;
-      fill = 0;
-    }
+    if (fill) *dst++ = (uint32_t)(acc << (32 - fill));
+    fill = 0;
   }
 };
+
+inline uint32_t reverse32(uint32_t v) {
+  v = ((v >> 1) & 0x55555555u) | ((v & 0x55555555u) << 1);
+  v = ((v >> 2) & 0x33333333u) | ((v & 0x33333333u) << 2);
+  v = ((v >> 4) & 0x0F0F0F0Fu) | ((v & 0x0F0F0F0Fu) << 4);
+  v = ((v >> 8) & 0x00FF00FFu) | ((v & 0x00FF00FFu) << 8);
+  return (v >> 16) | (v << 16);
+}
 
 template <typename F>
 void parallel_for(uint32_t n, uint32_t n_threads, F body) {
@@ -170,35 +163,39 @@ void parallel_for(uint32_t n, uint32_t n_threads, F body) {
   for (auto &th : pool) th.join();
 }
 
-// Zero bits the encoder leaves between a lane's two sub-streams (the format allows up to 63).  When every lane
-// of a tile has the same number of code bits and that number is a multiple of 256 -- a fixed-length code, as
-// near-uniform exponents give -- the lanes' words would all start at the same offsets modulo 8 words, and a decoder
-// that keeps the record in banked shared memory would serialise its word loads.  One word of padding per lane
-// staggers them.
-uint32_t lane_padding_bits(const uint32_t *lane_bits) {
-  for (uint32_t lane = 1; lane < kLanes; ++lane)
-    if (lane_bits[lane] != lane_bits[0]) return 0;
-  return (lane_bits[0] != 0 && lane_bits[0] % 256 == 0) ? 32u : 0u;
-}
-
-// bits of every lane's sub-stream of tile q; returns their sum
-uint64_t tile_lane_bits(const Geometry &g, const uint16_t *x, const uint8_t *len, uint32_t q, uint32_t *lane_bits) {
+// Code bits of every lane's forward stream (even iterations) and backward stream (odd iterations) of tile q.
+void tile_stream_bits(const Geometry &g, const uint16_t *x, const uint8_t *len, uint32_t q, uint32_t *fbits,
+                      uint32_t *bbits) {
   const uint32_t valid = g.tile_valid(q);
   const uint64_t origin = g.tile_origin(q), pitch = g.row_pitch();
-  uint64_t sum = 0;
   for (uint32_t lane = 0; lane < kLanes; ++lane) {
-    uint32_t bits = 0;
+    uint32_t bits[2] = {0, 0};
     for (uint32_t i = 0; i < g.iters; ++i) {
       uint32_t pos = (i * kLanes + lane) * kGroup;
       if (pos >= valid) break;
       uint32_t cnt = std::min(kGroup, valid - pos);
       const uint16_t *p = x + origin + i * pitch + lane * kGroup;
-      for (uint32_t j = 0; j < cnt; ++j) bits += len[(p[j] >> 7) & 0xFF];
+      for (uint32_t j = 0; j < cnt; ++j) bits[i & 1] += len[(p[j] >> 7) & 0xFF];
     }
-    lane_bits[lane] = bits;
-    sum += bits;
+    fbits[lane] = bits[0];
+    bbits[lane] = bits[1];
   }
-  return sum;
+}
+
+// Which column takes which backward stream, and how many rows the record needs.  All columns of a record are
+// equally high, so the record is as high as its fullest column: the lane with the k-th longest forward stream
+// shares its column with the k-th shortest backward stream, which keeps the fullest column close to the mean.
+uint32_t pair_streams(const uint32_t *fbits, const uint32_t *bbits, uint8_t *bcol) {
+  uint8_t by_f[kLanes], by_b[kLanes];
+  for (uint32_t a = 0; a < kLanes; ++a) by_f[a] = by_b[a] = (uint8_t)a;
+  std::stable_sort(by_f, by_f + kLanes, [&](uint8_t a, uint8_t b) { return fbits[a] > fbits[b]; });
+  std::stable_sort(by_b, by_b + kLanes, [&](uint8_t a, uint8_t b) { return bbits[a] < bbits[b]; });
+  uint32_t rows = 1;
+  for (uint32_t a = 0; a < kLanes; ++a) {
+    bcol[by_b[a]] = by_f[a];
+    rows = std::max(rows, (fbits[by_f[a]] + bbits[by_b[a]] + 31) / 32);
+  }
+  return rows;
 }
 
 }  // namespace
@@ -267,11 +264,11 @@ zipmoe_status zipmoe_encode(const uint16_t *bf16, uint64_t rows, uint64_t cols, 
   // pass 1: size of every tile record, then of every chunk
   std::vector<uint32_t> rec_units(g.n_tiles);  // record size in 16-byte units
   parallel_for(g.n_chunks, o.n_threads, [&](uint32_t k) {
-    uint32_t q0 = k * g.tiles_per_chunk, m = g.chunk_tiles(k), lane_bits[kLanes];
+    uint32_t q0 = k * g.tiles_per_chunk, m = g.chunk_tiles(k), fbits[kLanes], bbits[kLanes];
+    uint8_t bcol[kLanes];
     for (uint32_t t = 0; t < m; ++t) {
-      uint64_t bits = tile_lane_bits(g, bf16, len, q0 + t, lane_bits);
-      bits += (uint64_t)kLanes * lane_padding_bits(lane_bits);
-      rec_units[q0 + t] = (uint32_t)(align_up(kRecordHeadBytes + (bits + 7) / 8, 16) / 16);
+      tile_stream_bits(g, bf16, len, q0 + t, fbits, bbits);
+      rec_units[q0 + t] = (kRecordHeadBytes + pair_streams(fbits, bbits, bcol) * kRowBytes) / 16;
     }
   });
   std::vector<uint64_t> chunk_byte(g.n_chunks + 1, 0);
@@ -320,19 +317,19 @@ zipmoe_status zipmoe_encode(const uint16_t *bf16, uint64_t rows, uint64_t cols, 
       store_le<uint32_t>(chunk + 4ull * t, unit);
       uint8_t *rec = chunk + (uint64_t)unit * 16;
       const uint64_t rec_bytes = (uint64_t)rec_units[q] * 16;
-      std::memset(rec + rec_bytes - 16, 0, 16);  // padding of the last unit
+      std::memset(rec, 0, rec_bytes);
+      const uint32_t rows = (uint32_t)((rec_bytes - kRecordHeadBytes) / kRowBytes);
       const uint32_t valid = g.tile_valid(q);
       const uint64_t origin = g.tile_origin(q), pitch = g.row_pitch();
-      BitWriter bw(rec + kRecordHeadBytes);
-      uint32_t lane_bits[kLanes];
-      tile_lane_bits(g, bf16, len, q, lane_bits);
-      const uint32_t pad_bits = lane_padding_bits(lane_bits);
+      uint32_t fbits[kLanes], bbits[kLanes];
+      tile_stream_bits(g, bf16, len, q, fbits, bbits);
+      pair_streams(fbits, bbits, rec);   // rec[lane] = the column of the lane's backward stream
+      uint32_t words[kMaxRows * kLanes];   // [rows][32], copied into the record once complete
+      std::memset(words, 0, (size_t)rows * kRowBytes);
       for (uint32_t lane = 0; lane < kLanes; ++lane) {
-        const uint64_t before = bw.total;
-        // sub-stream 0 (even iterations) forwards; sub-stream 1 (odd iterations) is read backwards from the
-        // end of the lane's bit range, so it is appended last code first, every code with its bits reversed
-        uint8_t odd[ZIPMOE_TILE_ELEMS_MAX / kIterElems / 2 * kGroup];
-        uint32_t n_odd = 0;
+        // both streams are first written as plain word streams (first bit = bit 31 of word 0) ...
+        uint32_t fw[kMaxRows + 1] = {0}, bw[kMaxRows + 1] = {0};
+        BitWriter f(fw), b(bw);
         for (uint32_t i = 0; i < g.iters; ++i) {
           uint32_t pos = (i * kLanes + lane) * kGroup;
           if (pos >= valid) break;
@@ -340,18 +337,20 @@ zipmoe_status zipmoe_encode(const uint16_t *bf16, uint64_t rows, uint64_t cols, 
           const uint16_t *p = bf16 + origin + i * pitch + lane * kGroup;
           for (uint32_t j = 0; j < cnt; ++j) {
             uint32_t s = (p[j] >> 7) & 0xFF;
-            if (i & 1) odd[n_odd++] = (uint8_t)s;
-            else bw.put(code[s], len[s]);
+            if (i & 1) b.put(code[s], len[s]);
+            else f.put(code[s], len[s]);
           }
         }
-        if (pad_bits) bw.put(0, pad_bits);
-        while (n_odd) {
-          const uint32_t s = odd[--n_odd];
-          bw.put(reverse_bits(code[s], len[s]), len[s]);
-        }
-        store_le<uint16_t>(rec + 2 * lane, (uint16_t)(bw.total - before));
+        f.flush();
+        b.flush();
+        // ... then the forward stream goes down its own column from row 0, and the backward stream up the
+        // column it was paired with from the last row, bit-reversed as a whole (its k-th bit is the column's
+        // bit 32 * rows - 1 - k).  The two never share a bit, so or-ing them into the rows is safe.
+        const uint32_t fwords = (fbits[lane] + 31) / 32, bwords = (bbits[lane] + 31) / 32, bc = rec[lane];
+        for (uint32_t r = 0; r < fwords; ++r) words[r * kLanes + lane] |= fw[r];
+        for (uint32_t r = 0; r < bwords; ++r) words[(rows - 1 - r) * kLanes + bc] |= reverse32(bw[r]);
       }
-      bw.flush();
+      std::memcpy(rec + kRecordHeadBytes, words, (size_t)rows * kRowBytes);   // (little-endian host)
       // sign+mantissa bytes of the tile, in tile order
       uint8_t *smt = smsec + (uint64_t)q * g.tile_elems;
       for (uint32_t i = 0; i < g.iters; ++i) {
@@ -440,22 +439,30 @@ zipmoe_status zipmoe_blob_validate(const void *blob_v, uint64_t bytes) {
     for (uint32_t t = 0; t < m; ++t) {
       uint64_t r0 = (uint64_t)load_le<uint32_t>(chunk + 4ull * t) * 16;
       uint64_t r1 = (uint64_t)load_le<uint32_t>(chunk + 4ull * (t + 1)) * 16;
-      if (r1 < r0 + kRecordHeadBytes || r1 > chunk_bytes) return ZIPMOE_ERR_BAD_FORMAT;
+      // a record is the column table and at least one whole row of 32 words
+      if (r1 < r0 + kRecordHeadBytes + kRowBytes || r1 > chunk_bytes || (r1 - r0 - kRecordHeadBytes) % kRowBytes)
+        return ZIPMOE_ERR_BAD_FORMAT;
       if (r1 - r0 > tile_record_max(g.tile_elems)) return ZIPMOE_ERR_BAD_FORMAT;
-      uint64_t bits = 0;
-      const uint32_t valid = g.tile_valid(q0 + t);
+      // every column holds exactly one backward stream
+      uint32_t seen = 0;
       for (uint32_t lane = 0; lane < kLanes; ++lane) {
-        uint32_t b = load_le<uint16_t>(chunk + r0 + 2 * lane);
-        // a lane holds at most 8*iters codes of at most max_code_len bits, and at least one bit per element
-        uint32_t elems = 0;
+        const uint32_t c = chunk[r0 + lane];
+        if (c >= kLanes || (seen >> c) & 1u) return ZIPMOE_ERR_BAD_FORMAT;
+        seen |= 1u << c;
+      }
+      // a column has room for at least one bit per element of its two streams
+      const uint32_t valid = g.tile_valid(q0 + t);
+      const uint64_t col_bits = (r1 - r0 - kRecordHeadBytes) / kRowBytes * 32;
+      uint32_t felems[kLanes], belems[kLanes];
+      for (uint32_t lane = 0; lane < kLanes; ++lane) {
+        felems[lane] = belems[lane] = 0;
         for (uint32_t i = 0; i < g.iters; ++i) {
           uint32_t pos = (i * kLanes + lane) * kGroup;
-          if (pos < valid) elems += std::min(kGroup, valid - pos);
+          if (pos < valid) ((i & 1) ? belems : felems)[lane] += std::min(kGroup, valid - pos);
         }
-        if (b < elems || b > elems * info.max_code_len + 63) return ZIPMOE_ERR_BAD_FORMAT;   // up to 63 padding bits
-        bits += b;
       }
-      if (kRecordHeadBytes * 8 + bits > (r1 - r0) * 8) return ZIPMOE_ERR_BAD_FORMAT;
+      for (uint32_t lane = 0; lane < kLanes; ++lane)
+        if (felems[chunk[r0 + lane]] + belems[lane] > col_bits) return ZIPMOE_ERR_BAD_FORMAT;
     }
     prev = next;
   }

@@ -110,8 +110,8 @@ def test_every_bit_pattern_and_special_values(zb):
 
 
 def test_long_records_of_near_uniform_exponents(zb):
-    """Near-uniform exponents: 8-bit codes, tile records of 4288 bytes (the encoder pads lanes of equal
-    length), decoded by the kernel instantiation with the larger record stages."""
+    """Near-uniform exponents: 8-bit codes, tile records of 32 rows, decoded by the kernel instantiation with
+    the larger record stages."""
     x = np.random.default_rng(2).integers(0, 1 << 16, 50021, dtype=np.uint16)
     blob = zb.zipmoe_encode(x, chunk_elems=16384)
     assert blob[64:320].min() >= 7

@@ -113,7 +113,8 @@ def test_bad_arguments_and_corrupt_blobs(zb):
     info = zb.zipmoe_blob_info_get(blob)
     for at, val in [(0, 0), (36, 13), (64 + int(np.flatnonzero(blob[64:320])[0]), 0), (328, blob[328] ^ 0x10),
                     (info.payload_off + 4, blob[info.payload_off + 4] + 1),
-                    (info.payload_off + 17, 0xFF)]:            # a lane's bit count beyond 8*I*max_len
+                    (info.payload_off + 17, 0xFF),             # a column that does not exist
+                    (info.payload_off + 18, blob[info.payload_off + 19])]:   # two backward streams in one column
         b = blob.copy()
         b[at] = val
         assert zb.zipmoe_blob_validate(b) == zb.ERR_BAD_FORMAT, at
@@ -187,10 +188,11 @@ def test_ffn_planning_on_the_host(zb):
     assert ctypes.sizeof(zb.CompressedExperts) == 80
 
 
-def test_equal_length_lanes_are_padded_and_still_decode(zb):
-    """Fixed-length codes (all 256 exponents equally frequent) give every lane of a tile the same number of code
-    bits; the encoder then leaves one zero word between each lane's two sub-streams.  The oracle, which inserts
-    no padding itself, must accept and decode such a blob."""
+def test_records_are_level_columns(zb):
+    """A record is as high as its fullest column.  Fixed-length codes (all 256 exponents equally frequent) give 32
+    rows and leave every lane in its own column; on Gaussian weights the library pairs long forward streams with
+    short backward streams, so that the record is within a row of the mean need of its columns -- and the oracle,
+    which reads the pairing from the record, decodes it."""
     from oracle import codec
     rng = np.random.default_rng(3)
     e = np.tile(np.arange(256, dtype=np.uint16), 40)
@@ -199,16 +201,23 @@ def test_equal_length_lanes_are_padded_and_still_decode(zb):
     blob = zb.zipmoe_encode(x, chunk_elems=4096)
     assert (blob[64:320] == 8).all() and zb.zipmoe_blob_validate(blob) == zb.OK
     info = zb.zipmoe_blob_info_get(blob)
-    rec = blob[info.payload_off + 16:]
-    assert (rec[:64].view(np.uint16) == 128 * 8 + 32).all()   # first tile: 128 codes of 8 bits and the padding
+    table = blob[info.payload_off: info.payload_off + 8].view(np.uint32)
+    assert (int(table[1]) - int(table[0])) * 16 == 32 + 32 * 128
+    assert blob[info.payload_off + 16: info.payload_off + 48].tolist() == list(range(32))
     assert np.array_equal(codec.decode(blob), x)
-    bad = blob.copy()
-    bad[info.payload_off + 16 + 64 + 16 * 4] = 1              # lane 0: 16 words forwards, then the padding word
-    with pytest.raises(ValueError):
-        codec.decode(bad)                                     # padding must be zero
-    y = x.copy()
-    y[5] = (7 << 7) | 0x33                                    # no longer a fixed-length code?  still decodes
-    assert np.array_equal(codec.decode(zb.zipmoe_encode(y, chunk_elems=4096)), y)
+
+    g = inputs.gaussian((64, 4096), 0.02, 12)
+    blob = zb.zipmoe_encode(g, chunk_elems=65536, max_code_len=12)
+    info = zb.zipmoe_blob_info_get(blob)
+    L = blob[64:320].astype(np.int64)
+    mean_rows = L[(g.ravel() >> 7) & 0xFF].sum() / 64 / 32 / 32   # code bits per column, in rows of 32 bits
+    offs = blob[info.payload_off: info.payload_off + 4 * 17].view(np.uint32).astype(np.int64)   # 16 tiles in the chunk
+    rows = ((offs[1:] - offs[:-1]) * 16 - 32) / 128
+    assert (rows == rows.astype(np.int64)).all() and rows.min() >= mean_rows - 0.5 and rows.max() <= mean_rows + 2
+    assert np.median(rows) <= mean_rows + 1
+    assert any(blob[info.payload_off + int(offs[0]) * 16: info.payload_off + int(offs[0]) * 16 + 32].tolist()[k] != k
+               for k in range(32))                            # a real pairing, not the identity
+    assert np.array_equal(codec.decode(blob), g.ravel())
 
 
 def test_plan_reports_the_largest_tile_record(zb):
@@ -217,7 +226,7 @@ def test_plan_reports_the_largest_tile_record(zb):
     assert 1300 < plan.max_record_bytes < 1700
     u = np.random.default_rng(0).integers(0, 1 << 16, 20000, dtype=np.uint16)
     plan = zb.DecodePlan([zb.zipmoe_encode(u, chunk_elems=4096)])
-    assert plan.max_record_bytes == 64 + 4096 + 32 * 4   # 8-bit codes everywhere, one word of padding per lane
+    assert plan.max_record_bytes == 32 + 32 * 128        # 8-bit codes everywhere: 128 codes per column, 32 rows
 
 
 def test_plan_rejects_a_damaged_tile_table(zb):
