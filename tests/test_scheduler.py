@@ -1,0 +1,97 @@
+"""Pins of the cache-affinity scheduling oracle (oracle/scheduler.py; paper Section 3.3, Appendix Algorithm
+"Cache-Affinity Scheduling", Theorem 1) and the library's zipmoe_plan_schedule / zipmoe_plan_simulate against it."""
+import numpy as np
+import pytest
+
+from oracle import scheduler as osch
+
+
+def test_single_task_makespan_is_the_printed_critical_path_when_workers_cover_the_chunks():
+    """Definition "Critical-Path": z_j = rho u [M, S] + max(K c / min(K, L), u [M, E]) + p_j.  With L >= K every
+    E-chunk is decompressed as it arrives, and the simulated schedule of one task takes exactly z_j."""
+    for state in "MCSE":
+        for (c, u, rho, K, L, p) in [(1.0, 4.0, 0.5, 2, 2, 3.0), (0.3, 2.0, 0.35, 4, 6, 0.7), (5.0, 1.0, 0.4, 3, 3, 0.1)]:
+            inst = osch.Instance([(0, state)], {0: p}, c, u, rho, K, L)
+            got = osch.simulate(inst, [[0]])["makespan"]
+            assert abs(got - osch.critical_path_as_printed(inst, 0)) < 1e-12, (state, c, u, rho, K, L)
+    # fewer workers than chunks: the reads and the decompressions pipeline, and the task beats the printed sum
+    inst = osch.Instance([(0, "S")], {0: 1.0}, 1.0, 4.0, 0.5, 4, 1)     # E-chunks arrive at .5, 1, 1.5, 2
+    assert osch.simulate(inst, [[0]])["makespan"] == 0.5 + 4 * 1.0 + 1.0
+    assert osch.critical_path_as_printed(inst, 0) == 2.0 + 4.0 + 1.0
+
+
+def test_block_construction_worked_by_hand_one_block():
+    """K = 2, L = 1, c = 1, u = 4, rho = 0.5 (an E-chunk reads in 1).  Task 0: expert 0 missed (Type-I, p = 3);
+    task 1: expert 1 compressed in memory (Type-II, p = 2).  Block [0] alone: reads end at 6, the worker at 3: not
+    compute-dominant.  Task 1 in front costs no idle time (the worker starts at 0 instead of waiting for the first
+    E-chunk), so the block is [1, 0]: worker 0-2 on task 1, 2-4 on task 0; SM-chunk of task 0 at 6; GPU 2-4, 6-9."""
+    inst = osch.Instance([(0, "M"), (1, "C")], {0: 3.0, 1: 2.0}, 1.0, 4.0, 0.5, 2, 1)
+    alone = osch.simulate(inst, [[0]])
+    assert alone["io_end"] == [6.0] and alone["worker_end"] == [[3.0]] and alone["charge"] == 1.0
+    assert not osch.compute_dominant(inst, [[0]])
+    blocks = osch.cache_affinity_blocks(inst)
+    assert blocks == [[1, 0]]
+    s = osch.simulate(inst, blocks)
+    assert s["charge"] == 0.0 and s["ready"] == {1: 2.0, 0: 6.0} and s["makespan"] == 9.0
+    assert osch.lower_bound(inst) == 9.0                                  # here the schedule is optimal
+
+
+def test_block_construction_worked_by_hand_three_blocks():
+    """K = 1, L = 1, c = 5, u = 1, rho = 0.5.  Two missed experts and one compressed one.  The decompression is so
+    slow that [task 0] alone is compute-dominant (worker ends at 5.5, reads at 1.5, lag 4 >= 0.5), likewise
+    [task 1]; the Type-II task is left for a last block -- and, being ready at time 0, its decompression is what
+    the work-conserving worker runs first."""
+    inst = osch.Instance([(0, "M"), (1, "M"), (2, "C")], {0: 1.0, 1: 1.0, 2: 0.5}, 5.0, 1.0, 0.5, 1, 1)
+    blocks = osch.cache_affinity_blocks(inst)
+    assert blocks == [[0], [1], [2]]
+    s = osch.simulate(inst, blocks)
+    assert s["io_end"] == [1.5, 3.0, 3.0] and s["ready"] == {0: 10.0, 1: 15.0, 2: 5.0} and s["makespan"] == 16.0
+    assert osch.lower_bound(inst) == 15.0
+
+
+def random_instance(rng, n_experts, tensors):
+    tasks = []
+    for n in range(n_experts):
+        state = "MCSE"[int(rng.integers(4))]
+        tasks += [(n, state)] * tensors
+    p = {n: float(rng.uniform(0.1, 3.0)) for n in range(n_experts)}
+    return osch.Instance(tasks, p, c=float(rng.uniform(0.1, 2.0)), u=float(rng.uniform(0.5, 4.0)),
+                         rho=float(rng.uniform(0.3, 0.7)), K=int(rng.integers(1, 4)), L=int(rng.integers(1, 4)))
+
+
+def test_theorem_1_against_brute_force_on_tiny_instances():
+    """ALG <= (3 - 1/L) OPT.  OPT is taken over every priority order and every cut into blocks (brute force, at
+    most five tasks), which can only over-estimate the true optimum, and no schedule beats Lemma 1's bound."""
+    rng = np.random.default_rng(0)
+    worst = 0.0
+    for trial in range(40):
+        n_experts = int(rng.integers(1, 6))
+        inst = random_instance(rng, n_experts, tensors=1)
+        blocks = osch.cache_affinity_blocks(inst)
+        assert sorted(j for B in blocks for j in B) == list(range(len(inst.tasks)))
+        alg = osch.simulate(inst, blocks)["makespan"]
+        opt, _ = osch.best_blocks(inst)
+        lb = osch.lower_bound(inst)
+        assert lb <= opt + 1e-9 and opt <= alg + 1e-9
+        assert alg <= (3.0 - 1.0 / inst.L) * opt + 1e-9, (trial, alg, opt)
+        worst = max(worst, alg / opt)
+    print("worst ALG / OPT over 40 tiny instances: %.3f" % worst)
+
+
+def test_theorem_1_against_the_lower_bound_on_larger_instances():
+    """Where brute force is out of reach, Lemma 1's bound stands in for OPT from below: every schedule is at least
+    the bound, and the algorithm's stays within (3 - 1/L) of it on these instances (a stronger statement than
+    the theorem, recorded because it holds)."""
+    rng = np.random.default_rng(1)
+    for trial in range(60):
+        inst = random_instance(rng, int(rng.integers(2, 9)), tensors=int(rng.integers(1, 4)))
+        blocks = osch.cache_affinity_blocks(inst)
+        assert sorted(j for B in blocks for j in B) == list(range(len(inst.tasks)))
+        # tasks of an expert stay together and the bases come in non-increasing expert time
+        bases = [B[0] for B in blocks if inst.type_one(B[0])]
+        assert all(inst.p_of(a) >= inst.p_of(b) for a, b in zip(bases, bases[1:]))
+        alg = osch.simulate(inst, blocks)["makespan"]
+        lb = osch.lower_bound(inst)
+        order = list(rng.permutation(len(inst.tasks)))
+        assert osch.simulate(inst, [[int(j) for j in order]])["makespan"] >= lb - 1e-9
+        assert lb - 1e-9 <= alg <= (3.0 - 1.0 / inst.L) * lb + 1e-9, (trial, alg, lb)
