@@ -378,6 +378,47 @@ struct LaneDecoder {
     }
     return __brev(__funnelshift_r(c, n, pos1));
   }
+  // The next 64 bits of a stream as two registers (hi = the next 32 bits, first one in bit 31; lo = the 32 after
+  // them), from three words loaded at once: enough for two batches, so that only every other batch waits for
+  // shared memory.  second(hi, lo, used) is the window after `used` (0..32) of hi's bits have been consumed.
+  __device__ __forceinline__ void pair0(uint32_t &hi, uint32_t &lo) const {
+    const uint32_t r = pos0 >> 5;
+    uint32_t c, n, m;
+    if (STAGED) {
+      const uint32_t a = mad_u32(r, kRowBytes, col0);
+      c = lds_u32(a);
+      n = lds_u32(a + kRowBytes);
+      m = lds_u32(a + 2 * kRowBytes);
+    } else {
+      c = __ldg(words_g + min(r, last_row) * 32 + lane_g);
+      n = __ldg(words_g + min(r + 1, last_row) * 32 + lane_g);
+      m = __ldg(words_g + min(r + 2, last_row) * 32 + lane_g);
+    }
+    hi = __funnelshift_l(n, c, pos0);
+    lo = __funnelshift_l(m, n, pos0);
+  }
+  __device__ __forceinline__ void pair1(uint32_t &hi, uint32_t &lo) const {   // (bit-reversed: first bit in bit 0)
+    const uint32_t r = pos1 >> 5;
+    uint32_t c, n, m;
+    if (STAGED) {
+      const uint32_t a = top1 - r * kRowBytes;
+      c = lds_u32(a);
+      n = lds_u32(a - kRowBytes);
+      m = lds_u32(a - 2 * kRowBytes);
+    } else {
+      c = __ldg(words_g + (last_row - min(r, last_row)) * 32 + bcol_g);
+      n = __ldg(words_g + (last_row - min(r + 1, last_row)) * 32 + bcol_g);
+      m = __ldg(words_g + (last_row - min(r + 2, last_row)) * 32 + bcol_g);
+    }
+    hi = __funnelshift_r(c, n, pos1);
+    lo = __funnelshift_r(n, m, pos1);
+  }
+  __device__ static __forceinline__ uint32_t second0(uint32_t hi, uint32_t lo, uint32_t used) {
+    return __funnelshift_lc(lo, hi, used);
+  }
+  __device__ static __forceinline__ uint32_t second1(uint32_t hi, uint32_t lo, uint32_t used) {
+    return __brev(__funnelshift_rc(hi, lo, used));
+  }
   __device__ __forceinline__ uint32_t lookup(uint32_t w) const {   // (symbol << 23) | length of the code at the top of w
     if (FAST) return lds_u32(mad_u32(w >> (32 - kLaneLutBits), 128u, my_lut));
     return lds_u32(mad_u32(w >> (32 - kWideLutBits), 4u, lut));
@@ -403,9 +444,17 @@ struct LaneDecoder {
   __device__ __forceinline__ void group2(const uint2 sm0, const uint2 sm1, uint4 &o0, uint4 &o1) {
     uint32_t e[8], f[8];
     if (FAST) {
+      // two batches of four codes per stream from one pair of windows
+      uint32_t whi, wlo, xhi, xlo;
+      pair0(whi, wlo);
+      pair1(xhi, xlo);
+      uint32_t w = whi, x = __brev(xhi), used0 = 0, used1 = 0;
 #pragma unroll
       for (int h = 0; h < 8; h += 4) {
-        uint32_t w = window0(), x = window1();
+        if (h) {
+          w = second0(whi, wlo, used0);
+          x = second1(xhi, xlo, used1);
+        }
         e[h] = lookup(w);
         f[h] = lookup(x);
         w = next(w, e[h]);
@@ -420,21 +469,36 @@ struct LaneDecoder {
         x = next(x, f[h + 2]);
         e[h + 3] = lookup(w);
         f[h + 3] = lookup(x);
-        pos0 = (pos0 + (e[h] + e[h + 1]) + (e[h + 2] + e[h + 3])) & kPosMask;
-        pos1 = (pos1 + (f[h] + f[h + 1]) + (f[h + 2] + f[h + 3])) & kPosMask;
+        used0 = ((e[h] + e[h + 1]) + (e[h + 2] + e[h + 3])) & kPosMask;
+        used1 = ((f[h] + f[h + 1]) + (f[h + 2] + f[h + 3])) & kPosMask;
+        pos0 += used0;
+        pos1 += used1;
       }
     } else {
+      // two batches of two codes per stream from one pair of windows, twice
 #pragma unroll
-      for (int h = 0; h < 8; h += 2) {
-        uint32_t w = window0(), x = window1();
+      for (int h = 0; h < 8; h += 4) {
+        uint32_t whi, wlo, xhi, xlo;
+        pair0(whi, wlo);
+        pair1(xhi, xlo);
+        uint32_t w = whi, x = __brev(xhi);
         e[h] = lookup(w);
         f[h] = lookup(x);
         w = next(w, e[h]);
         x = next(x, f[h]);
         e[h + 1] = lookup(w);
         f[h + 1] = lookup(x);
-        pos0 = (pos0 + e[h] + e[h + 1]) & kPosMask;
-        pos1 = (pos1 + f[h] + f[h + 1]) & kPosMask;
+        const uint32_t used0 = (e[h] + e[h + 1]) & kPosMask, used1 = (f[h] + f[h + 1]) & kPosMask;
+        w = second0(whi, wlo, used0);
+        x = second1(xhi, xlo, used1);
+        e[h + 2] = lookup(w);
+        f[h + 2] = lookup(x);
+        w = next(w, e[h + 2]);
+        x = next(x, f[h + 2]);
+        e[h + 3] = lookup(w);
+        f[h + 3] = lookup(x);
+        pos0 = (pos0 + used0 + e[h + 2] + e[h + 3]) & kPosMask;
+        pos1 = (pos1 + used1 + f[h + 2] + f[h + 3]) & kPosMask;
       }
     }
     o0 = merge(sm0, e);
