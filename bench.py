@@ -522,7 +522,8 @@ def run_ours(args):
     from paper_2601_21198_b200 import binding, build
     build.build()
     if args.ffn_only:      # profiling captures of the fused kernels on one token count
-        res = bench_ffn(dev, iters=args.ffn_iters, cpu_tokens=0, token_counts=(args.ffn_only,), config=args.ffn_config)
+        res = bench_ffn(dev, iters=args.ffn_iters, cpu_tokens=0, token_counts=tuple(int(t) for t in args.ffn_only.split(",")),
+                        config=args.ffn_config)
         print(json.dumps({"ffn": res}))
         return
     profiling = args.experts is not None or args.quick     # a small case for a profiler: no side sections
@@ -683,7 +684,7 @@ def main():
                     help="the configuration of the headline figure (default: the 8-expert 14336x4096 layer)")
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="device time the timed loops of the headline configuration must add up to")
-    ap.add_argument("--ffn-only", type=int, default=0, metavar="T",
+    ap.add_argument("--ffn-only", default="", metavar="T[,T...]",
                     help="run only the fused expert-FFN section for T tokens (profiling captures)")
     ap.add_argument("--ffn-iters", type=int, default=20)
     ap.add_argument("--e2e-slices", type=int, default=8,

@@ -339,6 +339,44 @@ zipmoe_status zipmoe_plan_cache_pools(const double *f, uint32_t n, uint32_t k, u
                                       const double expert_size[4], const zipmoe_plan_costs *costs, double step,
                                       double ratios[4], uint32_t capacity[4], double *expected);
 
+/* ---- cache-affinity scheduling (host only, no CUDA) ---------------------------
+ * The paper's scheduler (Section 3.3 "Cache-Affinity Scheduler"; appendix, Algorithm "Cache-Affinity
+ * Scheduling") as a simulator.  One reconstruction task per tensor of every selected expert; a task's
+ * compression state says what has to be read: 0 = M missed (E-chunks and SM-chunk), 1 = C compressed in memory
+ * (nothing), 2 = S SM-chunk in memory (E-chunks), 3 = E E-chunks in memory (SM-chunk).  Costs: u = read of one
+ * SM-chunk, rho * u / K = read of one of a tensor's K E-chunks, c = its decompression; p[n] = GPU time of the
+ * tokens routed to expert n.  One I/O thread, L decompression workers, one GPU stream, all work-conserving:
+ * the I/O thread reads, block by block, the E-chunks of the block's tasks and then their SM-chunks; a free
+ * worker takes the first decompression in priority order whose E-chunk has arrived; the GPU runs an expert
+ * once all its tensors are recovered.  Makespan = completion of the last expert. */
+typedef struct {
+  uint32_t expert; /* index into p                                   */
+  uint32_t state;  /* 0 M, 1 C, 2 S, 3 E                             */
+} zipmoe_sched_task;
+
+typedef struct {
+  double c, u, rho; /* delays as above; rho = compressed size of the exponent bits relative to their raw size */
+  uint32_t K, L;    /* E-chunks per tensor; decompression workers                                             */
+} zipmoe_sched_costs;
+
+/* Makespan, and total idle time of the workers directly before their operations (the appendix's "charge"), of
+ * the priority order order[0 .. n_tasks) cut into blocks: block_of[i] = block of order[i], non-decreasing.
+ * host in: tasks, p[n_experts], costs, order (a permutation), block_of; host out: *makespan, *charge (may be NULL). */
+zipmoe_status zipmoe_plan_simulate(const zipmoe_sched_task *tasks, uint32_t n_tasks, const double *p, uint32_t n_experts,
+                                   const zipmoe_sched_costs *costs, const uint32_t *order, const uint32_t *block_of,
+                                   double *makespan, double *charge);
+
+/* Algorithm "Cache-Affinity Scheduling": tasks that must read an SM-chunk (Type-I) and the others (Type-II) are
+ * sorted by non-increasing expert time; every block starts from the first unscheduled Type-I task and takes
+ * candidates (Type-II first) at the earliest position that adds no worker idle time -- else after the last task
+ * of its kind with at least its expert time -- until the block is compute-dominant: the l-th earliest worker
+ * completes at least l * rho * u / K after the block's reads, for l = 1 .. min(L, K) (Eq. "compute_dominate").
+ * Type-II tasks that no block took form a last block.
+ * host out: order[n_tasks], block_of[n_tasks], *n_blocks and *makespan (either may be NULL). */
+zipmoe_status zipmoe_plan_schedule(const zipmoe_sched_task *tasks, uint32_t n_tasks, const double *p, uint32_t n_experts,
+                                   const zipmoe_sched_costs *costs, uint32_t *order, uint32_t *block_of,
+                                   uint32_t *n_blocks, double *makespan);
+
 /* Name of a status code (static string). */
 const char *zipmoe_status_string(zipmoe_status s);
 

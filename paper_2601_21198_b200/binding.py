@@ -245,6 +245,58 @@ def zipmoe_plan_cache_pools(f, k, pool_mask, budget, expert_size, costs, step):
     return ratios, [int(c) for c in cap], out.value
 
 
+# ---- cache-affinity scheduling (host only) --------------------------------------------------------
+class SchedTask(ctypes.Structure):
+    _fields_ = [("expert", _u32), ("state", _u32)]
+
+
+class SchedCosts(ctypes.Structure):
+    _fields_ = [("c", ctypes.c_double), ("u", ctypes.c_double), ("rho", ctypes.c_double), ("K", _u32), ("L", _u32)]
+
+
+SCHED_STATES = {"M": 0, "C": 1, "S": 2, "E": 3}
+_lib.zipmoe_plan_simulate.argtypes = [ctypes.POINTER(SchedTask), _u32, _dp, _u32, ctypes.POINTER(SchedCosts),
+                                      ctypes.POINTER(_u32), ctypes.POINTER(_u32), _dp, _dp]
+_lib.zipmoe_plan_schedule.argtypes = [ctypes.POINTER(SchedTask), _u32, _dp, _u32, ctypes.POINTER(SchedCosts),
+                                      ctypes.POINTER(_u32), ctypes.POINTER(_u32), ctypes.POINTER(_u32), _dp]
+_lib.zipmoe_plan_simulate.restype = _int
+_lib.zipmoe_plan_schedule.restype = _int
+
+
+def _sched_args(tasks, p, costs):
+    arr = (SchedTask * len(tasks))(*[SchedTask(int(n), SCHED_STATES[s] if isinstance(s, str) else int(s)) for n, s in tasks])
+    pv, pp = _dbl(p)
+    return arr, pv, pp, SchedCosts(*costs)
+
+
+def zipmoe_plan_simulate(tasks, p, costs, blocks):
+    """tasks: [(expert, state)], p: expert times, costs: (c, u, rho, K, L), blocks: lists of task indices.
+    Returns (makespan, charge)."""
+    arr, pv, pp, cs = _sched_args(tasks, p, costs)
+    order = [j for B in blocks for j in B]
+    block_of = [b for b, B in enumerate(blocks) for _ in B]
+    n = len(tasks)
+    mk, ch = ctypes.c_double(0), ctypes.c_double(0)
+    _check("zipmoe_plan_simulate",
+           _lib.zipmoe_plan_simulate(arr, n, pp, pv.size, ctypes.byref(cs), (_u32 * n)(*order), (_u32 * n)(*block_of),
+                                     ctypes.byref(mk), ctypes.byref(ch)))
+    return mk.value, ch.value
+
+
+def zipmoe_plan_schedule(tasks, p, costs):
+    """Returns (blocks: lists of task indices in priority order, makespan)."""
+    arr, pv, pp, cs = _sched_args(tasks, p, costs)
+    n = len(tasks)
+    order, block_of, nb, mk = (_u32 * n)(), (_u32 * n)(), _u32(0), ctypes.c_double(0)
+    _check("zipmoe_plan_schedule",
+           _lib.zipmoe_plan_schedule(arr, n, pp, pv.size, ctypes.byref(cs), order, block_of, ctypes.byref(nb),
+                                     ctypes.byref(mk)))
+    blocks = [[] for _ in range(nb.value)]
+    for j, b in zip(order, block_of):
+        blocks[b].append(int(j))
+    return blocks, mk.value
+
+
 def zipmoe_ffn_workspace_bytes(T, k, experts):
     out = _u64(0)
     _check("zipmoe_ffn_workspace_bytes", _lib.zipmoe_ffn_workspace_bytes(T, k, ctypes.byref(experts), ctypes.byref(out)))

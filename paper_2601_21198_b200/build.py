@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libzipmoe.so")
-SOURCES = ["zipmoe_host.cpp", "planner.cpp", "decode_kernel.cu", "ffn_kernels.cu", "recover_kernel.cu"]
+SOURCES = ["zipmoe_host.cpp", "planner.cpp", "scheduler.cpp", "decode_kernel.cu", "ffn_kernels.cu", "recover_kernel.cu"]
 HEADERS = ["zipmoe_format.h", "decode_device.cuh", "tile_geometry.h", os.path.join(ROOT, "include", "zipmoe.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--use_fast_math",
               "-Xcompiler", "-fPIC,-O3,-Wall", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC]

@@ -77,11 +77,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return done != 0;
 }
-// Wait with an iteration limit (each try blocks for a short, hardware-defined
-// time): returns false instead of spinning forever if the copy never lands.
+// Wait with an iteration limit: returns false instead of spinning forever if the copy never lands.  A try that
+// fails is followed by a short sleep (growing to a quarter of a microsecond), so that a warp that waits -- the
+// helper warps of the fused kernel wait most of the time -- leaves its scheduler's issue slots to the warps
+// that decode.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t tries = 1u << 20) {
-  for (uint32_t it = 0; it < tries; ++it)
+  if (mbar_try_wait(bar, parity)) return true;
+  uint32_t ns = 32;
+  for (uint32_t it = 0; it < tries; ++it) {
+    __nanosleep(ns);
     if (mbar_try_wait(bar, parity)) return true;
+    if (ns < 256) ns += ns;
+  }
   return false;
 }
 // global -> shared, bytes a multiple of 16, both addresses 16-byte aligned

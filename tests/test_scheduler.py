@@ -95,3 +95,49 @@ def test_theorem_1_against_the_lower_bound_on_larger_instances():
         order = list(rng.permutation(len(inst.tasks)))
         assert osch.simulate(inst, [[int(j) for j in order]])["makespan"] >= lb - 1e-9
         assert lb - 1e-9 <= alg <= (3.0 - 1.0 / inst.L) * lb + 1e-9, (trial, alg, lb)
+
+
+# ---------------------------------------------------------------- the library against the oracle
+@pytest.fixture(scope="module")
+def zb():
+    from paper_2601_21198_b200 import build
+    build.build()
+    from paper_2601_21198_b200 import binding
+    return binding
+
+
+def _as_args(inst):
+    n_experts = max(n for n, _ in inst.tasks) + 1
+    return inst.tasks, [inst.p.get(n, 0.0) for n in range(n_experts)], (inst.c, inst.u, inst.rho, inst.K, inst.L)
+
+
+def test_library_scheduler_matches_the_oracle(zb):
+    rng = np.random.default_rng(7)
+    for trial in range(80):
+        inst = random_instance(rng, int(rng.integers(1, 9)), tensors=int(rng.integers(1, 4)))
+        tasks, p, costs = _as_args(inst)
+        want = osch.cache_affinity_blocks(inst)
+        got, makespan = zb.zipmoe_plan_schedule(tasks, p, costs)
+        assert got == want, trial
+        s = osch.simulate(inst, want)
+        assert abs(makespan - s["makespan"]) < 1e-9
+        # any order: the two simulators agree on makespan and charge
+        order = [int(j) for j in rng.permutation(len(tasks))]
+        cut = int(rng.integers(0, len(order) + 1))
+        blocks = [b for b in (order[:cut], order[cut:]) if b]
+        mk, ch = zb.zipmoe_plan_simulate(tasks, p, costs, blocks)
+        s = osch.simulate(inst, blocks)
+        assert abs(mk - s["makespan"]) < 1e-9 and abs(ch - s["charge"]) < 1e-9, trial
+
+
+def test_library_scheduler_worked_examples_and_bad_arguments(zb):
+    blocks, mk = zb.zipmoe_plan_schedule([(0, "M"), (1, "C")], [3.0, 2.0], (1.0, 4.0, 0.5, 2, 1))
+    assert blocks == [[1, 0]] and mk == 9.0
+    blocks, mk = zb.zipmoe_plan_schedule([(0, "M"), (1, "M"), (2, "C")], [1.0, 1.0, 0.5], (5.0, 1.0, 0.5, 1, 1))
+    assert blocks == [[0], [1], [2]] and mk == 16.0
+    for tasks, p, costs in [([(3, "M")], [1.0], (1, 1, 0.5, 1, 1)), ([(0, 7)], [1.0], (1, 1, 0.5, 1, 1)),
+                            ([(0, "M")], [1.0], (1, 1, 0.5, 0, 1)), ([(0, "M")], [1.0], (1, 1, 0.5, 1, 0))]:
+        with pytest.raises(zb.ZipMoEError):
+            zb.zipmoe_plan_schedule(tasks, p, costs)
+    with pytest.raises(zb.ZipMoEError):
+        zb.zipmoe_plan_simulate([(0, "M"), (0, "C")], [1.0], (1, 1, 0.5, 1, 1), [[0, 0]])   # not a permutation
