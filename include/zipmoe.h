@@ -177,11 +177,11 @@ zipmoe_status zipmoe_blob_plan(const void *blob, uint64_t blob_bytes, uint64_t p
  * Work distribution: launches of few large tensors (n_tiles >= 512 * n_tables) give every CTA an equal range of
  *             tiles; all others hand the tiles out dynamically through an 8-byte counter.  The counters are a
  *             ring of 1024 in the library's own device memory (nothing is allocated); a launch zeroes its
- *             counter on `stream` before the kernel (one cudaMemsetAsync) and tags it as its own with the first
- *             range of tiles it takes.  More than 1024 such launches in flight at once on one device would share
- *             counters: the launch that finds another launch's tag stops taking tiles and sets status_word
- *             (code 6), the other one is not disturbed -- incomplete output is never silent.  The same holds for
- *             a captured graph that replays such a launch while a later launch owns its counter.
+ *             counter on `stream` before the kernel (one cudaMemsetAsync) and its first CTA tags it as the
+ *             launch's own.  More than 1024 such launches in flight at once on one device would share counters:
+ *             a launch that finds another launch's tag on its counter stops taking tiles and sets status_word
+ *             (code 6), so that incomplete output does not go unnoticed.  The same holds for a captured graph
+ *             that replays such a launch while a later launch owns its counter.
  * All device pointers 16-byte aligned.  Errors found on the host (null or
  * misaligned pointers, zero table count with non-zero chunks) are returned
  * before anything is launched. */

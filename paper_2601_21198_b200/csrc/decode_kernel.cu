@@ -217,29 +217,28 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
     __syncthreads();   // s_grab of the previous round has been read by every thread
     if (tid == 0) {
       // The counter is one 64-bit word: the tag of the launch that owns it above the next tile not yet handed out.
-      // It was zeroed on the stream before this kernel; the first range taken installs the tag in the same atomic
-      // step.  Should two launches ever be given the same counter while both are in flight (more of them queued
-      // than the ring has slots), one of them finds the other's tag: it reports that and takes no more tiles,
-      // and the other is not disturbed -- nothing is skipped silently.
+      // It was zeroed on the stream before this kernel; the first CTA to arrive installs the launch's tag.  Should
+      // two launches ever be given the same counter while both are in flight (more of them queued than the ring
+      // has slots), a CTA that finds the other launch's tag reports that and takes no more tiles, so that
+      // incomplete output does not go unnoticed.  (The tag is checked before the range is taken, not in the same
+      // atomic step: a compare-and-swap loop would make the CTAs of a launch queue up behind one another.)
       unsigned long long *ctr = reinterpret_cast<unsigned long long *>(a.work_counter);
+      const unsigned long long old = *reinterpret_cast<volatile unsigned long long *>(ctr);
+      uint32_t tag = (uint32_t)(old >> 32);
+      const uint32_t seen = (uint32_t)old;
+      if (tag == 0u) {
+        const uint32_t prev = atomicCAS(a.work_counter + 1, 0u, a.work_tag);   // the upper word
+        tag = prev ? prev : a.work_tag;
+      }
       uint32_t first = a.n_tiles, take = 0;
-      for (uint32_t tries = 0; tries < (1u << 16); ++tries) {
-        const unsigned long long old = *reinterpret_cast<volatile unsigned long long *>(ctr);
-        const uint32_t tag = (uint32_t)(old >> 32), seen = (uint32_t)old;
-        if (tag != 0u && tag != a.work_tag) {
-          report(a.status, kStatusCounterShared);
-          break;
-        }
-        if (seen >= a.n_tiles) break;   // all handed out
-        uint32_t want = (a.n_tiles - seen) / (ZIPMOE_GRAB_DIV * gridDim.x);
-        want = max(want, max(1u, min(kMinGrab, a.n_tiles / gridDim.x)));   // small launches: spread over all CTAs
-        want = min(want, a.n_tiles - seen);
-        const unsigned long long next = ((unsigned long long)a.work_tag << 32) | (seen + want);
-        if (atomicCAS(ctr, old, next) == old) {
-          first = seen;
-          take = want;
-          break;
-        }
+      if (tag != a.work_tag) {
+        report(a.status, kStatusCounterShared);
+      } else if (seen < a.n_tiles) {
+        take = (a.n_tiles - seen) / (ZIPMOE_GRAB_DIV * gridDim.x);
+        take = max(take, max(1u, min(kMinGrab, a.n_tiles / gridDim.x)));   // small launches: spread over all CTAs
+        first = (uint32_t)atomicAdd(ctr, (unsigned long long)take);
+        take = first < a.n_tiles ? min(a.n_tiles - first, take) : 0u;
+        if (take == 0) first = a.n_tiles;
       }
       s_grab[0] = first;
       s_grab[1] = first + take;

@@ -451,6 +451,9 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
               // half, or the first half of the strip's next tile), a whole half ahead of its use.
               const uint8_t *ahead = half == 0 ? cur.sm + 8 * 256 + lane * 8 : nxt.sm + lane * 8;
               const bool more = half == 0 || have_next;
+              // and the half after that one is asked into the second-level cache (2 KB = 16 lines, one per lane)
+              if (have_next && lane < 16)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(nxt.sm + (half == 0 ? 0 : 8 * 256) + lane * 128));
               // the first four rows (two from each of the lane's sub-streams) are decoded into registers while
               // the previous half's MMAs may still run
               uint4 v[4];
