@@ -151,6 +151,37 @@ zipmoe_status zipmoe_blob_plan(const void *blob, uint64_t blob_bytes, uint64_t p
                                uint64_t out_base, uint32_t table_id, uint32_t chunk_base, uint32_t tile_base,
                                zipmoe_chunk_desc *descs, zipmoe_table *table);
 
+/* One decode launch over several blobs: where every blob's E-chunk section, SM section and tensor sit in the
+ * launch's three buffers, and what zipmoe_decode / zipmoe_decode_expert_ffn need to know about the whole. */
+typedef struct {
+  uint64_t payload_bytes;    /* E-chunk sections of all blobs, back to back                                   */
+  uint64_t sm_bytes;         /* their SM sections, each rounded up to 16 bytes                                */
+  uint64_t out_elems;        /* their tensors, each rounded up to 8 elements                                  */
+  uint32_t n_chunks, n_tiles, n_tables;
+  uint32_t max_record_bytes; /* largest tile record of the launch: zipmoe_decode's argument of that name      */
+  uint32_t max_code_len;     /* longest code of any table of the launch                                       */
+  uint32_t flags;            /* ZIPMOE_DECODE_SHORT_CODES if the launch may promise it, else 0                */
+} zipmoe_launch_info;
+
+/* Sizes only (the first call of the two-call pattern).  host in: blobs[n_blobs], blob_bytes[n_blobs];
+ * host out: *info with the three sizes and the counts (max_record_bytes, max_code_len and flags are zero). */
+zipmoe_status zipmoe_launch_plan_size(const void *const *blobs, const uint64_t *blob_bytes, uint32_t n_blobs,
+                                      zipmoe_launch_info *info);
+
+/* Lays the blobs out for one launch (Section 3.1: what "Real-time Inference" finds in memory -- E-chunks,
+ * SM-chunks and metadata -- arranged for the decoder): copies every blob's E-chunk section into `payload` and
+ * its SM section into `sm`, one after the other, zero-fills the ZIPMOE_DEVICE_PAD_BYTES after each, and writes
+ * the chunk descriptors (zipmoe_blob_plan with table_id = index of the blob) and tables.  The caller copies the
+ * four arrays to the device as they are.
+ * host in : blobs, blob_bytes
+ * host out: payload[info.payload_bytes + PAD], sm[info.sm_bytes + PAD], descs[info.n_chunks], tables[n_blobs],
+ *           tensor_first_chunk[n_blobs] (may be NULL: first descriptor of each blob, as
+ *           zipmoe_compressed_experts wants it), out_base[n_blobs] (may be NULL: element offset of each tensor
+ *           in the output buffer of info.out_elems elements), *info (complete). */
+zipmoe_status zipmoe_launch_plan(const void *const *blobs, const uint64_t *blob_bytes, uint32_t n_blobs, uint8_t *payload,
+                                 uint8_t *sm, zipmoe_chunk_desc *descs, zipmoe_table *tables, uint32_t *tensor_first_chunk,
+                                 uint64_t *out_base, zipmoe_launch_info *info);
+
 /* Real-time reconstruction (Section 3.1 "Real-time Inference", steps 6-7;
  * Section 3.3 "Memory-Coalesced Tensor Recovery Kernel"): decode every
  * chunk's exponent bytes from its E-chunk and merge them with the SM bytes
@@ -376,6 +407,14 @@ zipmoe_status zipmoe_plan_simulate(const zipmoe_sched_task *tasks, uint32_t n_ta
 zipmoe_status zipmoe_plan_schedule(const zipmoe_sched_task *tasks, uint32_t n_tasks, const double *p, uint32_t n_experts,
                                    const zipmoe_sched_costs *costs, uint32_t *order, uint32_t *block_of,
                                    uint32_t *n_blocks, double *makespan);
+
+/* For the library's own tests (the paper has no counterpart).  Every wait of a kernel on an asynchronous copy is
+ * bounded: when it runs out the kernel sets status_word (code 3), skips the work that depended on the copy, and
+ * still terminates.  That path cannot be reached with sound inputs, so this switch provokes it without a fault:
+ * from now on zipmoe_decode and zipmoe_decode_expert_ffn arm the barrier of every tile-record copy for
+ * extra_tx_bytes more than the copy delivers (so that the barrier never completes although the copy does) and give
+ * up after `tries` tries.  (0, 0) restores normal operation.  Process-wide; not for concurrent use. */
+void zipmoe_test_wait_fault(uint32_t extra_tx_bytes, uint32_t tries);
 
 /* Name of a status code (static string). */
 const char *zipmoe_status_string(zipmoe_status s);

@@ -2,8 +2,8 @@
 
 Every function here has the name of the C entry point it forwards to and does
 argument marshalling only (numpy arrays / torch tensors -> pointers and sizes).
-`DecodePlan` lays several blobs out in contiguous host buffers and collects the
-descriptors zipmoe_blob_plan writes; it computes nothing of the codec.
+`DecodePlan` holds what zipmoe_launch_plan wrote for several blobs (buffers,
+descriptors, tables); it computes nothing of the codec or of the layout.
 
 There is no fallback: if the CUDA library has not been built, importing this
 module raises.
@@ -101,6 +101,15 @@ def _ptr(a):
     if isinstance(a, np.ndarray):
         return a.ctypes.data
     return a.data_ptr()
+
+
+_lib.zipmoe_test_wait_fault.argtypes = [_u32, _u32]
+_lib.zipmoe_test_wait_fault.restype = None
+
+
+def zipmoe_test_wait_fault(extra_tx_bytes, tries):
+    """Test switch: record barriers armed for extra_tx_bytes too many, waits limited to `tries`; (0, 0) = normal."""
+    _lib.zipmoe_test_wait_fault(int(extra_tx_bytes), int(tries))
 
 
 def zipmoe_version():
@@ -320,45 +329,47 @@ def zipmoe_decode_expert_ffn_noalloc(tokens, T, topk_ids, topk_weights, k, exper
                                                  ctypes.byref(experts), _ptr(out), _ptr(status_word), _ptr(stream)))
 
 
+class LaunchInfo(ctypes.Structure):
+    _fields_ = [("payload_bytes", _u64), ("sm_bytes", _u64), ("out_elems", _u64), ("n_chunks", _u32), ("n_tiles", _u32),
+                ("n_tables", _u32), ("max_record_bytes", _u32), ("max_code_len", _u32), ("flags", _u32)]
+
+
+_lib.zipmoe_launch_plan_size.argtypes = [ctypes.POINTER(_vp), ctypes.POINTER(_u64), _u32, ctypes.POINTER(LaunchInfo)]
+_lib.zipmoe_launch_plan.argtypes = [ctypes.POINTER(_vp), ctypes.POINTER(_u64), _u32, _vp, _vp, _vp, _vp, _vp, _vp,
+                                    ctypes.POINTER(LaunchInfo)]
+_lib.zipmoe_launch_plan_size.restype = _int
+_lib.zipmoe_launch_plan.restype = _int
+
+
 class DecodePlan:
-    """Host-side layout of one decode launch over several blobs: where each
-    blob's E-chunk section, SM section and output tensor sit in three contiguous
-    buffers, plus the chunk descriptors and tables from zipmoe_blob_plan."""
+    """One decode launch over several blobs, as zipmoe_launch_plan lays it out: the three contiguous host
+    buffers, the chunk descriptors and the tables.  Marshalling only: the layout is the library's."""
 
     def __init__(self, blobs):
+        blobs = [np.ascontiguousarray(b, dtype=np.uint8) for b in blobs]
+        n = len(blobs)
+        ptrs = (_vp * max(n, 1))(*[b.ctypes.data for b in blobs])
+        sizes = (_u64 * max(n, 1))(*[b.size for b in blobs])
+        info = LaunchInfo()
+        _check("zipmoe_launch_plan_size", _lib.zipmoe_launch_plan_size(ptrs, sizes, n, ctypes.byref(info)))
+        self.payload = np.empty(info.payload_bytes + DEVICE_PAD_BYTES, np.uint8)
+        self.sm = np.empty(info.sm_bytes + DEVICE_PAD_BYTES, np.uint8)
+        self.descs = np.zeros(info.n_chunks, CHUNK_DESC_DTYPE)
+        self.tables = np.zeros(n * TABLE_BYTES, np.uint8)
+        self.tensor_first_chunk = np.zeros(n, np.uint32)
+        out_base = np.zeros(n, np.uint64)
+        _check("zipmoe_launch_plan",
+               _lib.zipmoe_launch_plan(ptrs, sizes, n, _ptr(self.payload), _ptr(self.sm), _ptr(self.descs),
+                                       _ptr(self.tables), _ptr(self.tensor_first_chunk), _ptr(out_base), ctypes.byref(info)))
         self.infos = [zipmoe_blob_info_get(b) for b in blobs]
-        pay = sm = out = 0
-        self.payload_base, self.sm_base, self.out_base = [], [], []
-        for inf in self.infos:
-            self.payload_base.append(pay)
-            self.sm_base.append(sm)
-            self.out_base.append(out)
-            pay += inf.payload_bytes                      # multiples of 16 by construction
-            sm += (inf.sm_bytes + 15) // 16 * 16
-            out += (inf.n_elems + 7) // 8 * 8
-        self.payload_bytes, self.sm_bytes, self.out_elems = pay, sm, out
-        self.payload = np.zeros(pay + DEVICE_PAD_BYTES, np.uint8)
-        self.sm = np.zeros(sm + DEVICE_PAD_BYTES, np.uint8)
-        descs, tables = [], []
-        chunk_base = tile_base = 0
-        for i, (b, inf) in enumerate(zip(blobs, self.infos)):
-            b = np.ascontiguousarray(b, dtype=np.uint8)
-            self.payload[self.payload_base[i]: self.payload_base[i] + inf.payload_bytes] = \
-                b[inf.payload_off: inf.payload_off + inf.payload_bytes]
-            self.sm[self.sm_base[i]: self.sm_base[i] + inf.sm_bytes] = b[inf.sm_off: inf.sm_off + inf.sm_bytes]
-            d, t = zipmoe_blob_plan(b, self.payload_base[i], self.sm_base[i], self.out_base[i], i, chunk_base,
-                                    tile_base)
-            descs.append(d)
-            tables.append(t)
-            chunk_base += inf.n_chunks
-            tile_base += inf.n_tiles
-        self.descs = np.concatenate(descs) if descs else np.zeros(0, CHUNK_DESC_DTYPE)
-        self.tables = np.concatenate(tables) if tables else np.zeros(0, np.uint8)
-        self.n_chunks, self.n_tiles, self.n_tables = chunk_base, tile_base, len(blobs)
-        self.max_record_bytes = int(self.descs["max_record_bytes"].max()) if self.n_chunks else 0
-        # what the fastest kernel variant wants promised: no code longer than 8 bits, no record higher than 16 rows
-        self.max_code_len = int(self.tables.max()) if self.tables.size else 0
-        self.flags = DECODE_SHORT_CODES if (0 < self.max_record_bytes <= NARROW_RECORD_BYTES and self.max_code_len <= 8) else 0
+        self.out_base = [int(v) for v in out_base]
+        self.payload_base = [int(self.descs["payload_off"][int(c)]) if inf.n_chunks else 0
+                             for c, inf in zip(self.tensor_first_chunk, self.infos)]
+        self.sm_base = [int(self.descs["sm_off"][int(c)]) if inf.n_chunks else 0
+                        for c, inf in zip(self.tensor_first_chunk, self.infos)]
+        self.payload_bytes, self.sm_bytes, self.out_elems = info.payload_bytes, info.sm_bytes, info.out_elems
+        self.n_chunks, self.n_tiles, self.n_tables = info.n_chunks, info.n_tiles, info.n_tables
+        self.max_record_bytes, self.max_code_len, self.flags = info.max_record_bytes, info.max_code_len, info.flags
 
     def algorithmic_bytes(self):
         """Bytes one decode must move: E-chunk section + SM bytes read, bf16 written."""
@@ -426,8 +437,7 @@ class DeviceExperts:
         assert len(blobs) % 3 == 0
         self.plan = DecodePlan(blobs)
         self.dev = self.plan.to_device(device)
-        first = np.cumsum([0] + [inf.n_chunks for inf in self.plan.infos])[:-1].astype(np.uint32)
-        self.tensor_first_chunk = torch.from_numpy(first.view(np.int32).copy()).to(self.dev.device)
+        self.tensor_first_chunk = torch.from_numpy(self.plan.tensor_first_chunk.view(np.int32).copy()).to(self.dev.device)
         p, d = self.plan, self.dev
         self.struct = CompressedExperts(len(blobs) // 3, hidden, inter, p.n_chunks, d.descs.data_ptr(),
                                         self.tensor_first_chunk.data_ptr(), d.tables.data_ptr(), p.n_tables, 0,

@@ -236,6 +236,9 @@ struct LaunchArgs {
   uint32_t *work_counter;   // two words zeroed before the launch (dynamic distribution only): the next tile not yet
                             // handed to a CTA, and the tag of the launch that uses the counter
   uint32_t work_tag;
+  uint32_t wait_tries;      // tries of a wait on an asynchronous copy before the kernel gives up on it
+  uint32_t extra_tx;        // 0; the library's own tests arm record barriers for this many bytes more than the
+                            // copy delivers, so that the give-up path can be exercised without any fault
 };
 
 // Which descriptor holds global tile g: exact guess for launches whose chunks all hold the same number of tiles,
@@ -636,3 +639,9 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
 }
 
 }  // namespace zipmoe_dev
+
+namespace zipmoe_host {
+constexpr uint32_t kWaitTries = 1u << 20;
+// what zipmoe_test_wait_fault last set (0 extra bytes and kWaitTries unless a test is running)
+void wait_fault_setting(uint32_t *extra_tx, uint32_t *tries);
+}  // namespace zipmoe_host

@@ -61,13 +61,14 @@ struct Cfg {
 struct WarpPipe {
   uint32_t pay_addr, sm_addr, bar_addr;   // shared addresses: record stages, SM slots, barriers
   uint32_t stage_bytes;                   // bytes of a record stage
+  uint32_t tries, extra_tx;               // wait limit; test-only surplus a record barrier is armed with
   uint32_t phase;                         // bit b = parity to wait for on barrier b
   uint32_t pending;                       // bit b = a copy on barrier b has been started and not waited for
   uint32_t lane;
 
   __device__ __forceinline__ uint32_t bar(uint32_t b) const { return bar_addr + 8 * b; }
   __device__ __forceinline__ bool wait(uint32_t b) {
-    if (!mbar_wait_bounded(bar(b), (phase >> b) & 1u)) return false;
+    if (!mbar_wait_bounded(bar(b), (phase >> b) & 1u, tries)) return false;
     phase ^= 1u << b;
     pending &= ~(1u << b);
     return true;
@@ -75,7 +76,10 @@ struct WarpPipe {
   // all lanes call these; one lane starts the copy
   __device__ __forceinline__ void load_record(const TileWork &t, uint32_t stage) {
     if (!t.staged) return;
-    if (lane == 0) bulk_load(pay_addr + stage * stage_bytes, t.rec, t.rec_bytes, bar(stage));
+    if (lane == 0) {
+      mbar_expect_tx(bar(stage), t.rec_bytes + extra_tx);
+      bulk_g2s(pay_addr + stage * stage_bytes, t.rec, t.rec_bytes, bar(stage));
+    }
     pending |= 1u << stage;
   }
   __device__ __forceinline__ void load_sm_piece(const TileWork &t, uint32_t p) {
@@ -87,7 +91,7 @@ struct WarpPipe {
   // after a wait ran out: give what is still in flight one short, bounded chance to land
   __device__ __forceinline__ void drain() {
     for (uint32_t b = 0; b < (uint32_t)kBarsPerWarp; ++b)
-      if (pending & (1u << b)) mbar_wait_bounded(bar(b), (phase >> b) & 1u, 1u << 14);
+      if (pending & (1u << b)) mbar_wait_bounded(bar(b), (phase >> b) & 1u, min(tries, 1u << 14));
   }
 };
 
@@ -190,6 +194,8 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
   pipe.stage_bytes = Cfg<WIDE>::kStage;
   pipe.sm_addr = pipe.pay_addr + kPayStages * Cfg<WIDE>::kStage;
   pipe.bar_addr = smem_addr(bars + warp * kBarsPerWarp);
+  pipe.tries = a.wait_tries;
+  pipe.extra_tx = a.extra_tx;
   pipe.phase = 0;
   pipe.pending = 0;
   pipe.lane = lane;
@@ -397,6 +403,7 @@ namespace {
 constexpr uint32_t kCounterSlots = 1024;
 static __device__ unsigned long long g_work_counters[kCounterSlots];   // per slot: tag of the owning launch << 32 | next tile
 std::atomic<uint32_t> g_next_slot{0};
+std::atomic<uint32_t> g_test_extra_tx{0}, g_test_tries{zipmoe_host::kWaitTries};
 
 struct DeviceInfo {
   int sm_count = 0;
@@ -434,6 +441,16 @@ zipmoe_status prepare_device(int *sm_count, uint32_t **counters) {
 }
 }  // namespace
 
+void zipmoe_host::wait_fault_setting(uint32_t *extra_tx, uint32_t *tries) {
+  *extra_tx = g_test_extra_tx.load();
+  *tries = g_test_tries.load();
+}
+
+extern "C" void zipmoe_test_wait_fault(uint32_t extra_tx_bytes, uint32_t tries) {
+  g_test_extra_tx.store(extra_tx_bytes & ~15u);
+  g_test_tries.store(tries ? tries : zipmoe_host::kWaitTries);
+}
+
 extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t n_chunks, uint32_t n_tiles,
                                        const zipmoe_table *tables, uint32_t n_tables, const uint8_t *payload,
                                        uint64_t payload_bytes, const uint8_t *sm, uint64_t sm_bytes,
@@ -463,6 +480,7 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
   a.n_chunks = n_chunks;
   a.n_tiles = n_tiles;
   a.n_tables = n_tables;
+  zipmoe_host::wait_fault_setting(&a.extra_tx, &a.wait_tries);
   // CTAs to fill the SMs once, each with a contiguous range of tiles
   const bool narrow = max_record_bytes != 0 && max_record_bytes <= (uint32_t)zipmoe_dev::Cfg<false>::kBuf;
   uint32_t ctas = (uint32_t)sms * (narrow ? zipmoe_dev::Cfg<false>::kCtasPerSm : zipmoe_dev::Cfg<true>::kCtasPerSm);

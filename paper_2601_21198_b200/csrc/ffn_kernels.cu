@@ -319,7 +319,10 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
     uint2 sm[8];   // sign+mantissa bytes of the lane's groups in the 8 rows of a half-tile
     if (!failed) {
       cur = tile(0);
-      if (cur.staged && lane == 0) bulk_load(my + stage * kPayStage, cur.rec, cur.rec_bytes, rec_bar + 8 * stage);
+      if (cur.staged && lane == 0) {
+        mbar_expect_tx(rec_bar + 8 * stage, cur.rec_bytes + a.la.extra_tx);
+        bulk_g2s(my + stage * kPayStage, cur.rec, cur.rec_bytes, rec_bar + 8 * stage);
+      }
 #pragma unroll
       for (int k = 0; k < 8; ++k) sm[k] = ldg_v2_early(cur.sm + k * 256 + lane * 8);
     }
@@ -426,14 +429,16 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
         const bool have_next = !failed && s + 1 < n_steps;
         if (have_next) {
           nxt = tile(s + 1);
-          if (nxt.staged && lane == 0)
-            bulk_load(my + (stage ^ 1) * kPayStage, nxt.rec, nxt.rec_bytes, rec_bar + 8 * (stage ^ 1));
+          if (nxt.staged && lane == 0) {
+            mbar_expect_tx(rec_bar + 8 * (stage ^ 1), nxt.rec_bytes + a.la.extra_tx);
+            bulk_g2s(my + (stage ^ 1) * kPayStage, nxt.rec, nxt.rec_bytes, rec_bar + 8 * (stage ^ 1));
+          }
         }
         bool step_done = false;
         if (!failed) {
           bool good = true;
           if (cur.staged) {
-            good = mbar_wait_bounded(rec_bar + 8 * stage, (rec_phase >> stage) & 1);
+            good = mbar_wait_bounded(rec_bar + 8 * stage, (rec_phase >> stage) & 1, a.la.wait_tries);
             rec_phase ^= 1u << stage;
             if (!good) {
               report(a.la.status, kStatusWaitTimeout);
@@ -819,6 +824,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.la.tiles_per_cta = 0;
   a.la.work_counter = nullptr;
   a.la.work_tag = 0;
+  zipmoe_host::wait_fault_setting(&a.la.extra_tx, &a.la.wait_tries);
   a.tensor_first_chunk = ex->tensor_first_chunk;
   a.expert_offset = expert_offset;
   a.active = active;

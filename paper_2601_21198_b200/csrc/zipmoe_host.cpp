@@ -520,3 +520,69 @@ zipmoe_status zipmoe_blob_plan(const void *blob_v, uint64_t bytes, uint64_t payl
 }
 
 }  // extern "C"
+
+// ---- planning one launch over several blobs ---------------------------------------------------
+extern "C" {
+
+zipmoe_status zipmoe_launch_plan_size(const void *const *blobs, const uint64_t *blob_bytes, uint32_t n_blobs,
+                                      zipmoe_launch_info *info) {
+  if (!info || (n_blobs && (!blobs || !blob_bytes))) return ZIPMOE_ERR_INVALID_ARG;
+  zipmoe_launch_info li = {};
+  for (uint32_t i = 0; i < n_blobs; ++i) {
+    zipmoe_blob_info bi;
+    zipmoe_status rc = zipmoe_blob_info_get(blobs[i], blob_bytes[i], &bi);
+    if (rc != ZIPMOE_OK) return rc;
+    li.payload_bytes += bi.payload_bytes;              // multiples of 16 by construction
+    li.sm_bytes += align_up(bi.sm_bytes, 16);
+    li.out_elems += align_up(bi.n_elems, 8);
+    if ((uint64_t)li.n_chunks + bi.n_chunks > 0xFFFFFFFFull || (uint64_t)li.n_tiles + bi.n_tiles > 0xFFFFFFFFull)
+      return ZIPMOE_ERR_UNSUPPORTED;
+    li.n_chunks += bi.n_chunks;
+    li.n_tiles += bi.n_tiles;
+  }
+  li.n_tables = n_blobs;
+  *info = li;
+  return ZIPMOE_OK;
+}
+
+zipmoe_status zipmoe_launch_plan(const void *const *blobs, const uint64_t *blob_bytes, uint32_t n_blobs, uint8_t *payload,
+                                 uint8_t *sm, zipmoe_chunk_desc *descs, zipmoe_table *tables, uint32_t *tensor_first_chunk,
+                                 uint64_t *out_base, zipmoe_launch_info *info) {
+  zipmoe_launch_info li;
+  zipmoe_status rc = zipmoe_launch_plan_size(blobs, blob_bytes, n_blobs, &li);
+  if (rc != ZIPMOE_OK) return rc;
+  if (!info || (n_blobs && (!payload || !sm || !tables)) || (li.n_chunks && !descs)) return ZIPMOE_ERR_INVALID_ARG;
+  uint64_t pay = 0, smo = 0, out = 0;
+  uint32_t chunk_base = 0, tile_base = 0;
+  li.max_record_bytes = 0;
+  li.max_code_len = 0;
+  for (uint32_t i = 0; i < n_blobs; ++i) {
+    const uint8_t *blob = static_cast<const uint8_t *>(blobs[i]);
+    zipmoe_blob_info bi;
+    zipmoe_blob_info_get(blob, blob_bytes[i], &bi);
+    std::memcpy(payload + pay, blob + bi.payload_off, bi.payload_bytes);
+    std::memcpy(sm + smo, blob + bi.sm_off, bi.sm_bytes);
+    std::memset(sm + smo + bi.sm_bytes, 0, align_up(bi.sm_bytes, 16) - bi.sm_bytes);
+    rc = zipmoe_blob_plan(blob, blob_bytes[i], pay, smo, out, i, chunk_base, tile_base, descs + chunk_base, tables + i);
+    if (rc != ZIPMOE_OK) return rc;
+    if (tensor_first_chunk) tensor_first_chunk[i] = chunk_base;
+    if (out_base) out_base[i] = out;
+    if (bi.n_chunks) li.max_record_bytes = std::max(li.max_record_bytes, descs[chunk_base].max_record_bytes);
+    for (int s = 0; s < 256; ++s) li.max_code_len = std::max<uint32_t>(li.max_code_len, tables[i].code_len[s]);
+    pay += bi.payload_bytes;
+    smo += align_up(bi.sm_bytes, 16);
+    out += align_up(bi.n_elems, 8);
+    chunk_base += bi.n_chunks;
+    tile_base += bi.n_tiles;
+  }
+  std::memset(payload + pay, 0, ZIPMOE_DEVICE_PAD_BYTES);
+  std::memset(sm + smo, 0, ZIPMOE_DEVICE_PAD_BYTES);
+  // the promise the fastest kernel variant wants holds exactly when the plan says so
+  li.flags = (li.max_record_bytes > 0 && li.max_record_bytes <= ZIPMOE_NARROW_RECORD_BYTES && li.max_code_len <= 8)
+                 ? ZIPMOE_DECODE_SHORT_CODES
+                 : 0u;
+  *info = li;
+  return ZIPMOE_OK;
+}
+
+}  // extern "C"
