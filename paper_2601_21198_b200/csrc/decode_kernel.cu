@@ -112,14 +112,17 @@ struct SmFeed {
   }
 };
 
+// PITCH = 256: the rows of a tile follow one another (linear layout), so that a row's offset is a constant of the
+// unrolled decode loop; PITCH = 0: the pitch is the tensor's (blocked layout).
+template <uint32_t PITCH>
 struct GlobalSink {
   uint16_t *out;
   uint32_t pitch;
   __device__ __forceinline__ void group(uint32_t i, uint32_t lane, const uint4 &v) const {
-    __stcs(reinterpret_cast<uint4 *>(out + (size_t)i * pitch + lane * 8), v);
+    __stcs(reinterpret_cast<uint4 *>(out + (size_t)i * (PITCH ? PITCH : pitch) + lane * 8), v);
   }
   __device__ __forceinline__ void elem(uint32_t i, uint32_t lane, uint32_t j, uint16_t v) const {
-    out[(size_t)i * pitch + lane * 8 + j] = v;
+    out[(size_t)i * (PITCH ? PITCH : pitch) + lane * 8 + j] = v;
   }
 };
 
@@ -342,11 +345,16 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
         if (rc == 0) {
           const uint32_t rec_s = pipe.pay_addr + stage * pipe.stage_bytes;
           SmFeed feed{pipe, nxt, nxt_issued};
-          GlobalSink sink{cur.out, cur.pitch};
+          GlobalSink<0> sink{cur.out, cur.pitch};
           if (LEAN) {
-            rc = (cur.staged && fast) ? decode_tile<true, true, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid,
-                                                                        cur.iters, lane, feed, sink)
-                                      : kStatusBrokenPromise;
+            if (!(cur.staged && fast)) {
+              rc = kStatusBrokenPromise;
+            } else if (cur.pitch == 256u) {
+              GlobalSink<256> rows{cur.out, 256u};
+              rc = decode_tile<true, true, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid, cur.iters, lane, feed, rows);
+            } else {
+              rc = decode_tile<true, true, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid, cur.iters, lane, feed, sink);
+            }
           } else if (cur.staged) {
             rc = fast ? decode_tile<true, true, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid,
                                                   cur.iters, lane, feed, sink)

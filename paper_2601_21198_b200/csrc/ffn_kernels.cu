@@ -710,7 +710,7 @@ zipmoe_status make_plan(uint32_t T, uint32_t k, const zipmoe_compressed_experts 
   // as many decode warps as fit beside the activation ring and the lookup table
   uint32_t nw = zipmoe_dev::kFfnMaxWarps;
   while (nw > (uint32_t)zipmoe_dev::kGroupWarps && zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u)
-    nw -= zipmoe_dev::kGroupWarps;
+    nw -= nw % zipmoe_dev::kGroupWarps ? nw % zipmoe_dev::kGroupWarps : zipmoe_dev::kGroupWarps;   // first the incomplete group
   if (zipmoe_dev::ffn_smem_bytes(nw, p->groups) > 227u * 1024u) return ZIPMOE_ERR_UNSUPPORTED;
   p->n_warps = nw;
   p->smem = zipmoe_dev::ffn_smem_bytes(nw, p->groups);
