@@ -36,7 +36,7 @@ def build(force=False, verbose=False):
     tmp = LIB + ".tmp%d" % os.getpid()
     extra = os.environ.get("ZIPMOE_NVCC_EXTRA", "").split()   # e.g. -DZIPMOE_WARPS=20 when tuning
     cmd = [_nvcc()] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + \
-          [os.path.join(CSRC, s) for s in SOURCES] + ["-o", tmp, "-lcudart"]
+          [os.path.join(CSRC, s) for s in SOURCES] + ["-o", tmp, "-lcudart", "-ldl"]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)
     return LIB

@@ -4,6 +4,7 @@
 // tile decoder.  sm_100a only.
 #pragma once
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <cstdint>
 #include <type_traits>
@@ -641,6 +642,12 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
 }  // namespace zipmoe_dev
 
 namespace zipmoe_host {
+// A named range around an entry point's host work and launches, for timeline profilers (costs nothing unless a
+// tool is attached).
+struct TraceRange {
+  explicit TraceRange(const char *name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+};
 constexpr uint32_t kWaitTries = 1u << 20;
 // what zipmoe_test_wait_fault last set (0 extra bytes and kWaitTries unless a test is running)
 void wait_fault_setting(uint32_t *extra_tx, uint32_t *tries);

@@ -464,6 +464,7 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
                                        uint64_t payload_bytes, const uint8_t *sm, uint64_t sm_bytes,
                                        uint16_t *out_bf16, uint64_t out_elems, uint32_t *status_word,
                                        zipmoe_stream stream, uint32_t max_record_bytes, uint32_t flags) {
+  zipmoe_host::TraceRange trace("zipmoe_decode");
   if (n_chunks == 0 || n_tiles == 0) return (n_chunks == 0 && n_tiles == 0) ? ZIPMOE_OK : ZIPMOE_ERR_INVALID_ARG;
   if (!chunks || !tables || n_tables == 0 || !payload || !sm || !out_bf16) return ZIPMOE_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(payload) | reinterpret_cast<uintptr_t>(sm) | reinterpret_cast<uintptr_t>(out_bf16) |

@@ -772,6 +772,7 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
                                                   uint64_t workspace_bytes, uint32_t *status_word,
                                                   zipmoe_stream stream_) {
   using namespace zipmoe_dev;
+  zipmoe_host::TraceRange trace("zipmoe_decode_expert_ffn");
   FfnPlan p;
   zipmoe_status rc = make_plan(T, k, ex, plan_grid(), &p);
   if (rc != ZIPMOE_OK) return rc;

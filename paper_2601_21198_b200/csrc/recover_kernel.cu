@@ -6,6 +6,7 @@
 // reference point for the fused decode kernel, and the recovery step for callers
 // that keep E-chunks decompressed.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <cstdint>
 
@@ -62,6 +63,8 @@ __global__ void __launch_bounds__(256) recover_kernel(const uint8_t *__restrict_
 
 extern "C" zipmoe_status zipmoe_recover(const uint8_t *exp, const uint8_t *sm, uint64_t n_elems, uint16_t *out_bf16,
                                         zipmoe_stream stream) {
+  nvtxRangePushA("zipmoe_recover");
+  struct Pop { ~Pop() { nvtxRangePop(); } } pop;
   if (n_elems == 0) return ZIPMOE_OK;
   if (!exp || !sm || !out_bf16) return ZIPMOE_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(exp) | reinterpret_cast<uintptr_t>(sm) | reinterpret_cast<uintptr_t>(out_bf16)) & 15)
