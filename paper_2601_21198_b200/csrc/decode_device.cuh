@@ -222,6 +222,8 @@ struct TileWork {
   const uint8_t *sm;    // global address of the tile's sign+mantissa bytes
   uint16_t *out;        // global address of the tile's first element
   uint32_t rec_bytes, pitch, valid, iters, pieces;
+  uint32_t n_sub;       // 1, or the number of small consecutive tiles taken in one step (see decode_step): rec_bytes,
+                        // valid, iters and pieces are then those of the whole step
   bool ok, staged;      // staged: the record fits a record stage of the calling kernel
 };
 
@@ -274,6 +276,7 @@ __device__ __forceinline__ TileWork resolve_tile(const LaunchArgs &a, uint32_t c
   TileWork w;
   w.ok = false;
   w.staged = false;
+  w.n_sub = 1;
   if (c >= a.n_chunks) return w;
   const uint4 *d = reinterpret_cast<const uint4 *>(a.chunks + c);
   const uint4 d0 = __ldg(d), d1 = __ldg(d + 1), d2 = __ldg(d + 2), d3 = __ldg(d + 3);
@@ -632,6 +635,40 @@ __device__ __forceinline__ uint32_t decode_tile(uint32_t rec_s, const uint8_t *r
       } else {
         ragged(std::integral_constant<int, 0>{}, i, sm_s);
         if (i + 1 < i_end) ragged(std::integral_constant<int, 1>{}, i + 1, sm_s);
+      }
+    }
+    feed.end(p);
+  }
+  return 0;
+}
+
+// Decodes a step of n_sub small tiles with the 32 lanes of a warp: consecutive full tiles of one linear tensor, each
+// of `sub_iters` (2, 4 or 8) iterations with a record of its own, whose records were staged by one copy (lane i holds
+// the offset of record i in the stage and its size), whose sign+mantissa bytes are one contiguous run served in the
+// usual pieces, and whose outputs are one contiguous run of rows.  The per-tile costs of the pipeline (copies,
+// waits, bookkeeping) are paid once per step.  Codes of at most 8 bits only.
+template <class Feed, class Sink>
+__device__ __forceinline__ uint32_t decode_step(uint32_t rec_s, uint32_t sub_off, uint32_t sub_bytes, uint32_t n_sub,
+                                                uint32_t sub_iters, uint32_t lut, uint32_t lane, Feed &feed, Sink &sink) {
+  const uint32_t per_piece = kPieceIters / sub_iters;          // tiles served by one piece of sign+mantissa bytes
+  const uint32_t pieces = (n_sub + per_piece - 1) / per_piece;
+  for (uint32_t p = 0; p < pieces; ++p) {
+    const uint32_t sm_s = feed.begin(p);
+    if (sm_s == 0xFFFFFFFFu) return kStatusWaitTimeout;
+    const uint32_t i_end = min(n_sub, (p + 1) * per_piece);
+#pragma unroll 1
+    for (uint32_t i = p * per_piece; i < i_end; ++i) {
+      const uint32_t off = __shfl_sync(0xFFFFFFFFu, sub_off, i), bytes = __shfl_sync(0xFFFFFFFFu, sub_bytes, i);
+      LaneDecoder<true, true> dec;
+      dec.init(rec_s + off, nullptr, bytes, lut, lane);
+      const uint32_t row0 = i * sub_iters;                     // first row of the tile within the step
+      const uint32_t sm_lane = sm_s + (row0 % kPieceIters) * 256 + lane * 8;
+#pragma unroll 1
+      for (uint32_t k = 0; k < sub_iters; k += 2) {
+        uint4 o0, o1;
+        dec.group2(lds_v2(sm_lane + k * 256), lds_v2(sm_lane + (k + 1) * 256), o0, o1);
+        sink.group(row0 + k, lane, o0);
+        sink.group(row0 + k + 1, lane, o1);
       }
     }
     feed.end(p);

@@ -47,7 +47,9 @@ struct Cfg {
   static constexpr int kCtasPerSm = WIDE ? 1 : ZIPMOE_CTAS_PER_SM;
   static constexpr int kWarps = WIDE ? ZIPMOE_WARPS - 1 : ZIPMOE_WARPS / kCtasPerSm;   // warps per CTA
   static constexpr int kThreads = kWarps * 32;
-  static constexpr int kStage = WIDE ? (int)(kRecHead + 32 * kRowBytes) + kPaySlack : kPayStage;   // bytes of a record stage
+  // bytes of a record stage: 32 rows; or 16 rows and a little more, so that a step of four small tiles with four
+  // rows each (and the tile tables of their chunks in between) still fits
+  static constexpr int kStage = WIDE ? (int)(kRecHead + 32 * kRowBytes) + kPaySlack : 2432 + kPaySlack;
   static constexpr int kBuf = kStage - kPaySlack;                         // longest staged record
   static constexpr int kWarpBytes = kPayStages * kStage + kSmPieces * kSmPieceBytes;
   static constexpr int kSmemBytes = kLutBytes + kWarps * kWarpBytes + kWarps * kBarsPerWarp * 8 + kLutScratchBytes;
@@ -157,6 +159,7 @@ __device__ __forceinline__ TileWork fetch_tile(const LaunchArgs &a, const Packed
   const uint32_t sm16 = __reduce_or_sync(0xFFFFFFFFu, me ? mine.sm16 : 0u);
   const uint32_t out8 = __reduce_or_sync(0xFFFFFFFFu, me ? mine.out8 : 0u);
   TileWork w;
+  w.n_sub = 1;
   w.pitch = __reduce_or_sync(0xFFFFFFFFu, me ? mine.pitch : 0u);
   w.ok = bits >> 31;
   w.staged = (bits >> 30) & 1u;
@@ -170,6 +173,43 @@ __device__ __forceinline__ TileWork fetch_tile(const LaunchArgs &a, const Packed
   return w;
 }
 
+// Like fetch_tile, but small tiles are taken several at a time: if the tile of lane `at` is a full tile of fewer
+// than 16 (an even number of) iterations of a linear tensor, the tiles of the following lanes join it as long as they
+// are full tiles of the same size, their sign+mantissa bytes and outputs continue where the previous tile's end,
+// their records ascend, the whole span of records fits the record stage and the step stays within 4096 elements.
+// Lane i comes back with offset and size of the step's i-th record (sub_off, sub_bytes) and every lane with the tile
+// size in iterations (sub_iters).
+__device__ __forceinline__ TileWork fetch_step(const LaunchArgs &a, const PackedTile &mine, uint32_t at, uint32_t stage_buf,
+                                               uint32_t &sub_off, uint32_t &sub_bytes, uint32_t &sub_iters) {
+  TileWork w = fetch_tile(a, mine, at);
+  sub_off = 0;
+  sub_bytes = w.rec_bytes;
+  sub_iters = w.iters;
+  if (!w.ok || !w.staged || w.pitch != 256u || w.iters >= 16u || (w.iters & 1u) || w.valid != w.iters * 256u) return w;
+  const uint32_t lane = threadIdx.x & 31u, i = lane - at, most = 16u / w.iters;
+  const uint32_t first_rec = __shfl_sync(0xFFFFFFFFu, mine.rec16, at), first_sm = __shfl_sync(0xFFFFFFFFu, mine.sm16, at);
+  const uint32_t first_out = __shfl_sync(0xFFFFFFFFu, mine.out8, at);
+  const uint32_t my_units = (mine.bits >> 18) & 0x3FFu, my_end = mine.rec16 + my_units;
+  const uint32_t prev_end = __shfl_up_sync(0xFFFFFFFFu, my_end, 1);
+  const bool joins = lane >= at && i < most && (mine.bits >> 30) == 3u /* ok and staged */ &&
+                     ((mine.bits >> 13) & 31u) == w.iters && (mine.bits & 0x1FFFu) == w.valid && mine.pitch == 256u &&
+                     mine.sm16 == first_sm + i * (w.valid >> 4) && mine.out8 == first_out + i * (w.valid >> 3) &&
+                     (i == 0 || mine.rec16 >= prev_end) && mine.rec16 >= first_rec &&
+                     (uint64_t)(my_end - first_rec) * 16u <= stage_buf;
+  const uint32_t run = ~(__ballot_sync(0xFFFFFFFFu, joins) >> at);   // zero bits = consecutive tiles that join
+  const uint32_t n = min(most, run ? (uint32_t)__ffs(run) - 1u : 32u - at);
+  if (n < 2) return w;
+  const uint32_t src = min(at + lane, 31u);
+  sub_off = (__shfl_sync(0xFFFFFFFFu, mine.rec16, src) - first_rec) * 16u;
+  sub_bytes = __shfl_sync(0xFFFFFFFFu, my_units, src) * 16u;
+  w.n_sub = n;
+  w.rec_bytes = (__shfl_sync(0xFFFFFFFFu, my_end, at + n - 1) - first_rec) * 16u;
+  w.valid *= n;
+  w.iters *= n;
+  w.pieces = sm_pieces_of_tile(w.valid);
+  return w;
+}
+
 // BATCHED: tiles are resolved 32 at a time, one per lane, instead of one by one by the whole warp.  That pays when
 // tiles are small or tensors many; with few large tensors of full tiles the one-by-one form keeps the hot loop leaner
 // and is 3 % faster.  The host picks by the launch's tiles per tensor.
@@ -178,8 +218,9 @@ __device__ __forceinline__ TileWork fetch_tile(const LaunchArgs &a, const Packed
 // left undecoded.  The shorter code is worth 2-3 %.
 template <bool WIDE, bool BATCHED, bool LEAN = false>
 __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) decode_kernel(const LaunchArgs a) {
-  constexpr int kWarps = Cfg<WIDE>::kWarps, kThreads = Cfg<WIDE>::kThreads, kWarpBytes = Cfg<WIDE>::kWarpBytes;
-  constexpr uint32_t kBuf = Cfg<WIDE>::kBuf;
+  using C = Cfg<WIDE>;
+  constexpr int kWarps = C::kWarps, kThreads = C::kThreads, kWarpBytes = C::kWarpBytes;
+  constexpr uint32_t kBuf = C::kBuf;
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t *lut_raw = smem;
   uint8_t *warp_base = smem + kLutBytes;
@@ -194,8 +235,8 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
 
   WarpPipe pipe;
   pipe.pay_addr = smem_addr(warp_base + warp * kWarpBytes);
-  pipe.stage_bytes = Cfg<WIDE>::kStage;
-  pipe.sm_addr = pipe.pay_addr + kPayStages * Cfg<WIDE>::kStage;
+  pipe.stage_bytes = C::kStage;
+  pipe.sm_addr = pipe.pay_addr + kPayStages * C::kStage;
   pipe.bar_addr = smem_addr(bars + warp * kBarsPerWarp);
   pipe.tries = a.wait_tries;
   pipe.extra_tx = a.extra_tx;
@@ -298,10 +339,14 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
     PackedTile batch = {0, 0, 0, 0, 0};
     TileWork cur;
     cur.ok = false;
+    cur.n_sub = 1;
+    // small tiles are taken several at a time (only where codes of at most 8 bits are promised: decode_step)
+    constexpr bool steps = BATCHED && LEAN;
+    uint32_t cur_off = 0, cur_bytes = 0, cur_sub_iters = 0, nxt_off = 0, nxt_bytes = 0, nxt_sub_iters = 0;
     if (g < g_end && !dead) {
       if (batched) {
         batch = resolve_batch(g);
-        cur = fetch_tile(a, batch, 0);
+        cur = steps ? fetch_step(a, batch, 0, kBuf, cur_off, cur_bytes, cur_sub_iters) : fetch_tile(a, batch, 0);
       } else {
         cur = resolve_tile(a, tc, tt, kBuf, table_id);
       }
@@ -317,17 +362,21 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
       lut_table = table_id;
     }
 
-    for (uint32_t in_batch = 0; g < g_end && !dead; ++g) {
+    uint32_t advance = 1;   // tiles of the step being decoded
+    for (uint32_t in_batch = cur.n_sub; g < g_end && !dead; g += advance) {   // in_batch: tiles of the batch handed out
       TileWork nxt;
       nxt.ok = false;
+      nxt.n_sub = 1;
       uint32_t nxt_issued = 0;
-      if (g + 1 < g_end) {
+      advance = cur.n_sub;
+      if (g + advance < g_end) {
         if (batched) {
-          if (++in_batch == 32) {   // the batch is used up (the current tile was fetched from it one step ago)
-            batch = resolve_batch(g + 1);
+          if (in_batch == 32) {   // the batch is used up
+            batch = resolve_batch(g + advance);
             in_batch = 0;
           }
-          nxt = fetch_tile(a, batch, in_batch);
+          nxt = steps ? fetch_step(a, batch, in_batch, kBuf, nxt_off, nxt_bytes, nxt_sub_iters) : fetch_tile(a, batch, in_batch);
+          in_batch += nxt.n_sub;
         } else {
           if (++tt == tpc) {
             tt = 0;
@@ -351,7 +400,10 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
               rc = kStatusBrokenPromise;
             } else if (cur.pitch == 256u) {
               GlobalSink<256> rows{cur.out, 256u};
-              rc = decode_tile<true, true, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid, cur.iters, lane, feed, rows);
+              if (steps && cur.n_sub > 1)
+                rc = decode_step(rec_s, cur_off, cur_bytes, cur.n_sub, cur_sub_iters, lut, lane, feed, rows);
+              else
+                rc = decode_tile<true, true, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid, cur.iters, lane, feed, rows);
             } else {
               rc = decode_tile<true, true, BATCHED>(rec_s, nullptr, cur.rec_bytes, lut, cur.valid, cur.iters, lane, feed, sink);
             }
@@ -389,6 +441,9 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
       if (nxt.ok)
         for (; nxt_issued < nxt.pieces; ++nxt_issued) pipe.load_sm_piece(nxt, nxt_issued);
       cur = nxt;
+      cur_off = nxt_off;
+      cur_bytes = nxt_bytes;
+      cur_sub_iters = nxt_sub_iters;
       stage ^= 1;
     }
     g0 = seg_end;
@@ -514,9 +569,11 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
     if (ctas > most) ctas = most;
   }
   const bool lean = narrow && (flags & ZIPMOE_DECODE_SHORT_CODES);
-  if (lean && batched) zipmoe_dev::decode_kernel<false, true, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
+  if (lean && batched)
+    zipmoe_dev::decode_kernel<false, true, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
   else if (lean) zipmoe_dev::decode_kernel<false, false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
-  else if (narrow && batched) zipmoe_dev::decode_kernel<false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
+  else if (narrow && batched)
+    zipmoe_dev::decode_kernel<false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
   else if (narrow) zipmoe_dev::decode_kernel<false, false><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
   else if (batched) zipmoe_dev::decode_kernel<true, true><<<ctas, Wide::kThreads, Wide::kSmemBytes, st>>>(a);
   else zipmoe_dev::decode_kernel<true, false><<<ctas, Wide::kThreads, Wide::kSmemBytes, st>>>(a);
