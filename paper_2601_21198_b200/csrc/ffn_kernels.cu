@@ -77,6 +77,14 @@ struct FfnArgs {
   uint32_t smem_bytes;                 // dynamic shared memory of the launch
 };
 
+// The kernels of one call are launched with programmatic stream serialization: each may be set up on the SMs while
+// its predecessor is still running, waits here until that one has completed and its memory is visible, and then
+// lets its own successor do the same.  (Launched the ordinary way, the wait returns at once.)
+__device__ __forceinline__ void after_previous_kernel() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---- how the steps of a launch are shared out --------------------------------------------------
 // U units (steps of all jobs, job-major) go to P CTAs; CTA c takes [c*U/P, (c+1)*U/P).  P is chosen so that
 // every CTA gets at least min_units units, hence a job of `steps` units is cut between at most
@@ -152,6 +160,7 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
   // never read back)
   const uint32_t NACC = kGroupWarps == 16 ? (NCOL + 15u) & ~15u : NCOL;
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  after_previous_kernel();
 
   // ---- this CTA's share of the launch's steps ----
   const uint32_t n_active = __ldg(a.active);   // experts that have tokens
@@ -572,6 +581,7 @@ __global__ void route_kernel(const int32_t *topk_ids, uint32_t S, uint32_t k, ui
                              uint32_t *expert_offset, uint32_t *active, uint32_t *slot_token, uint32_t *slot_of,
                              uint32_t *slot_active, uint32_t *status) {
   extern __shared__ uint32_t sh[];   // [E] counts, [E] cursors, [E] position in the active list, [S] ids
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // (the first kernel of a call: launched the ordinary way)
   uint32_t *cnt = sh, *cursor = sh + E, *apos = sh + 2 * E;
   int32_t *ids = reinterpret_cast<int32_t *>(sh + 3 * E);
   for (uint32_t i = threadIdx.x; i < 3 * E; i += blockDim.x) sh[i] = 0;
@@ -635,6 +645,7 @@ __global__ void swiglu_kernel(const float *gu, const PartsOf po, const uint32_t 
   // block's first row, and again by the threads whose row lies in another group
   __shared__ uint32_t s_parts[2];
   const uint32_t slot = blockIdx.y, row0 = blockIdx.x * blockDim.x, row = row0 + threadIdx.x;
+  after_previous_kernel();
   if (slot >= __ldg(expert_offset + E)) return;
   if (threadIdx.x < 2) s_parts[threadIdx.x] = po.parts(slot, threadIdx.x, row0);
   __syncthreads();
@@ -656,6 +667,7 @@ __global__ void combine_kernel(const float *y, const PartsOf po, const uint32_t 
   // block's first column, are looked up once per block
   __shared__ uint32_t s_parts[8];
   const uint32_t t = blockIdx.y, c0 = blockIdx.x * blockDim.x, c = c0 + threadIdx.x;
+  after_previous_kernel();
   if (threadIdx.x < k && threadIdx.x < 8) {
     const uint32_t slot = slot_of[t * k + threadIdx.x];
     s_parts[threadIdx.x] = slot == 0xFFFFFFFFu ? 0u : po.parts(slot, 0, c0);
@@ -851,14 +863,31 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.n_groups = p.groups_gu;
   a.min_units = p.min_gu;
   a.max_parts = p.parts_gu;
-  ffn_matmul_kernel<<<p.grid, threads, p.smem, stream>>>(a);
+  // every kernel after the first may start while its predecessor drains (it waits for it before it reads anything)
+  cudaLaunchAttribute overlap;
+  overlap.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  overlap.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = stream;
+  cfg.attrs = &overlap;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3(p.grid);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = p.smem;
+  if (cudaLaunchKernelEx(&cfg, ffn_matmul_kernel, a) != cudaSuccess) return ZIPMOE_ERR_CUDA;
 
   po.n_mats = 2;
   po.n_groups = p.groups_gu;
   po.steps = H / 256;
   po.min_units = p.min_gu;
   po.max_parts = p.parts_gu;
-  swiglu_kernel<<<dim3((I + 255) / 256, S), 256, 0, stream>>>(gu, po, expert_offset, E, S, I, h);
+  cudaLaunchConfig_t small = cfg;
+  small.gridDim = dim3((I + 255) / 256, S);
+  small.blockDim = dim3(256);
+  small.dynamicSmemBytes = 0;
+  if (cudaLaunchKernelEx(&small, swiglu_kernel, (const float *)gu, po, (const uint32_t *)expert_offset, E, S, I, h) !=
+      cudaSuccess)
+    return ZIPMOE_ERR_CUDA;
 
   // down: partial sums of W_2 H
   a.slot_token = nullptr;
@@ -871,14 +900,17 @@ extern "C" zipmoe_status zipmoe_decode_expert_ffn(const uint16_t *tokens, uint32
   a.n_groups = p.groups_dn;
   a.min_units = p.min_dn;
   a.max_parts = p.parts_dn;
-  ffn_matmul_kernel<<<p.grid, threads, p.smem, stream>>>(a);
+  if (cudaLaunchKernelEx(&cfg, ffn_matmul_kernel, a) != cudaSuccess) return ZIPMOE_ERR_CUDA;
 
   po.n_mats = 1;
   po.n_groups = p.groups_dn;
   po.steps = I / 256;
   po.min_units = p.min_dn;
   po.max_parts = p.parts_dn;
-  combine_kernel<<<dim3((H + 255) / 256, T), 256, 0, stream>>>(y, po, slot_of, topk_weights, T, k, S, H, out);
+  small.gridDim = dim3((H + 255) / 256, T);
+  if (cudaLaunchKernelEx(&small, combine_kernel, (const float *)y, po, (const uint32_t *)slot_of, topk_weights, T, k, S,
+                         H, out) != cudaSuccess)
+    return ZIPMOE_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? ZIPMOE_OK : ZIPMOE_ERR_CUDA;
 }
 
