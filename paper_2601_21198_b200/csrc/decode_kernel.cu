@@ -173,8 +173,9 @@ __device__ __forceinline__ TileWork fetch_tile(const LaunchArgs &a, const Packed
   return w;
 }
 
-// Like fetch_tile, but small tiles are taken several at a time: if the tile of lane `at` is a full tile of fewer
-// than 16 (an even number of) iterations of a linear tensor, the tiles of the following lanes join it as long as they
+// Like fetch_tile, but small tiles are taken several at a time: if the tile of lane `at` is a full tile of 2, 4 or 8
+// iterations of a linear tensor (a whole number of tiles per piece of sign+mantissa bytes, so that no tile lies
+// across two pieces), the tiles of the following lanes join it as long as they
 // are full tiles of the same size, their sign+mantissa bytes and outputs continue where the previous tile's end,
 // their records ascend, the whole span of records fits the record stage and the step stays within 4096 elements.
 // Lane i comes back with offset and size of the step's i-th record (sub_off, sub_bytes) and every lane with the tile
@@ -185,7 +186,9 @@ __device__ __forceinline__ TileWork fetch_step(const LaunchArgs &a, const Packed
   sub_off = 0;
   sub_bytes = w.rec_bytes;
   sub_iters = w.iters;
-  if (!w.ok || !w.staged || w.pitch != 256u || w.iters >= 16u || (w.iters & 1u) || w.valid != w.iters * 256u) return w;
+  if (!w.ok || !w.staged || w.pitch != 256u || w.iters > kPieceIters || (w.iters & 1u) || kPieceIters % w.iters != 0 ||
+      w.valid != w.iters * 256u)
+    return w;
   const uint32_t lane = threadIdx.x & 31u, i = lane - at, most = 16u / w.iters;
   const uint32_t first_rec = __shfl_sync(0xFFFFFFFFu, mine.rec16, at), first_sm = __shfl_sync(0xFFFFFFFFu, mine.sm16, at);
   const uint32_t first_out = __shfl_sync(0xFFFFFFFFu, mine.out8, at);

@@ -96,23 +96,29 @@ def test_many_tensors_mixed_tiles_layouts_and_tables_in_one_launch(zb):
     assert (host[mask] == 0x5555).all()
 
 
-@pytest.mark.parametrize("chunk", [512, 1024, 2048])
+@pytest.mark.parametrize("chunk", [512, 768, 1024, 1536, 2048])
 def test_small_tiles_taken_several_at_a_time(zb, chunk):
     """Tiles of 512, 1024 or 2048 elements (chunks below 4096) are decoded several per step when they follow one
-    another in a tensor: whole multiples of a step, one tile more, one tile fewer, a ragged last tile, a tensor of a
-    single tile, a tensor with wide records (near-uniform exponents: fewer tiles fit the stage) -- all in one
-    launch, next to each other."""
+    another in a tensor and a warp is handed several of them: sixty tensors of about 400 tiles make the ranges of
+    tiles long enough for that (a launch of a few hundred tiles hands them out one by one) while the launch still
+    counts as one of many tensors, and next to them, in the same launch: whole multiples of a step, one tile more,
+    one tile fewer, a ragged last tile, a tensor of a single tile, a tensor with wide records (near-uniform
+    exponents: fewer tiles fit the stage).  Tiles of 768 or 1536
+    elements would lie across two pieces of sign+mantissa bytes and must go one by one."""
     rng = np.random.default_rng(chunk)
-    sizes = [8 * 4096, 8 * 4096 + chunk, 8 * 4096 - chunk, 5 * 4096 + chunk // 2 + 3, chunk, chunk - 1, 3 * chunk + 1, 40 * chunk]
-    xs = [inputs.gaussian((n,), 0.02 * (1 + k), 1000 * chunk + k) for k, n in enumerate(sizes)]
-    xs.append(rng.integers(0, 1 << 16, 6 * 4096 + 77, dtype=np.uint16))      # 8-bit codes everywhere
+    sizes = [8 * 4096, 8 * 4096 + chunk, 8 * 4096 - chunk, 5 * 4096 + chunk // 2 + 3, chunk, chunk - 1, 3 * chunk + 1,
+             40 * chunk]
+    sizes += [(400 + k % 5) * chunk + (k % 7) * (chunk // 3 + 1) for k in range(60)]
+    xs = [inputs.gaussian((n,), 0.02 * (1 + k % 9), 1000 * chunk + k) for k, n in enumerate(sizes)]
+    xs.append(rng.integers(0, 1 << 16, 100 * 4096 + 77, dtype=np.uint16))    # 8-bit codes everywhere
     xs.append(inputs.stress_tensor(5, max_elems=50000)[0])
     blobs = [zb.zipmoe_encode(x, chunk_elems=chunk) for x in xs]
     plan, got, host = gpu_decode(zb, blobs)
     assert plan.flags == zb.DECODE_SHORT_CODES and plan.n_tiles < 512 * plan.n_tables
+    assert plan.n_tiles > 148 * 16 * 8                                        # several tiles per warp and range
     for g, x, b in zip(got, xs, blobs):
         assert np.array_equal(g, x.ravel())
-    for i in (3, 6, 8):
+    for i in (3, 6, 9, len(xs) - 2):
         assert np.array_equal(got[i], codec.decode(blobs[i]))
     mask = np.ones(plan.out_elems, bool)
     for i, inf in enumerate(plan.infos):
