@@ -149,6 +149,52 @@ def test_long_records_of_near_uniform_exponents(zb):
     assert np.array_equal(got, codec.decode(blob)) and np.array_equal(got, x)
 
 
+def _mostly_one_exponent(n_tiles, rare_tiles, layout, seed):
+    """bf16 patterns with one exponent nearly everywhere and, in the given tiles (4096 consecutive elements; in the
+    blocked layout 16 rows x 256 columns of a matrix 4096 wide), exponents drawn from 200 other values: at a
+    code-length limit of 12 those get codes of 9 bits or more, so the records of these tiles are higher than 32
+    rows."""
+    rng = np.random.default_rng(seed)
+    n = n_tiles * 4096
+    e = np.full(n, 120, np.uint16)
+    rare = np.array([v for v in range(1, 202) if v != 120], np.uint16)
+    if layout:
+        e = e.reshape(-1, 4096)
+    for t in rare_tiles:
+        if layout:
+            e[16 * (t // 16):16 * (t // 16) + 16, 256 * (t % 16):256 * (t % 16) + 256] = rng.choice(rare, (16, 256))
+        else:
+            e[t * 4096:(t + 1) * 4096] = rng.choice(rare, 4096)
+    sm = (rng.integers(0, 2, n, dtype=np.uint16) << 15) | rng.integers(0, 128, n, dtype=np.uint16)
+    return ((e << 7) | sm.reshape(e.shape)).astype(np.uint16)
+
+
+@pytest.mark.parametrize("n_tiles,layout", [(64, 0), (64, 1), (600, 0), (640, 1)])
+def test_records_too_high_for_a_stage_are_read_from_global_memory(zb, n_tiles, layout):
+    """Tiles whose codes average above 8 bits have records of more than 32 rows, which no record stage holds: the
+    decoder reads them from global memory.  With few tiles the launch hands tiles out dynamically, with 600 it
+    gives every CTA a fixed range; both layouts."""
+    x = _mostly_one_exponent(n_tiles, (0, 5, 6, n_tiles // 2, n_tiles - 1), layout, n_tiles + layout)
+    blob = zb.zipmoe_encode(x, layout=layout, chunk_elems=16384, max_code_len=12)
+    plan, (got,), _ = gpu_decode(zb, [blob])
+    assert plan.max_record_bytes > 32 + 32 * 128 and plan.max_code_len > 8 and plan.flags == 0
+    assert (plan.n_tiles >= 512) == (n_tiles >= 600)
+    assert np.array_equal(got, x.ravel())
+    assert np.array_equal(got, codec.decode(blob))
+
+
+def test_fixed_ranges_with_wide_records(zb):
+    """A single large tensor of near-uniform exponents (8-bit codes, records of 32 rows): fixed ranges of tiles per
+    CTA in the kernel instantiation with the larger record stages, linear and blocked layout."""
+    rng = np.random.default_rng(77)
+    for layout, shape in ((0, (700 * 4096 + 1234,)), (1, (176, 16384))):
+        x = rng.integers(0, 1 << 16, shape, dtype=np.uint16)
+        blob = zb.zipmoe_encode(x, layout=layout, chunk_elems=65536)
+        plan, (got,), _ = gpu_decode(zb, [blob])
+        assert plan.n_tiles >= 512 * plan.n_tables and plan.max_record_bytes > zb.NARROW_RECORD_BYTES
+        assert np.array_equal(got, x.ravel())
+
+
 def test_stress_set_sample(zb):
     xs, blobs = [], []
     for i in range(0, 96):
