@@ -85,20 +85,27 @@ def test_small_experts_match_oracle(zb, T, max_code_len):
         check(out.cpu().numpy().view(np.uint16), want, y, (T, max_code_len, weights is None))
 
 
-def test_experts_whose_records_do_not_fit_the_record_stage(zb):
+@pytest.mark.parametrize("long_codes", [False, True])
+def test_experts_whose_records_do_not_fit_the_record_stage(zb, long_codes):
     """Weights with forty equally likely exponents take more than 5 bits per code: tile records of about 22 rows,
-    more than the fused kernel's record stages hold, so the decode warps read them from global memory."""
+    more than the fused kernel's record stages hold, so the decode warps read them from global memory.  With a
+    thin tail of forty more (tiny) exponents and a code-length limit of 12 the tail's codes are longer than 8 bits
+    and the wide table is used as well."""
     import torch
     E, H, I, k, T = 2, 512, 1024, 2, 5
     rng = np.random.default_rng(123)
     ws, blobs = [], []
     for j in range(3 * E):
         shape = (I, H) if j % 3 < 2 else (H, I)
-        w = ((rng.integers(0, 2, shape, dtype=np.uint16) << 15) | (rng.integers(84, 124, shape, dtype=np.uint16) << 7) |
+        e = rng.integers(84, 124, shape, dtype=np.uint16)
+        if long_codes:
+            e = np.where(rng.random(shape) < 2e-3, rng.integers(40, 80, shape, dtype=np.uint16), e)
+        w = ((rng.integers(0, 2, shape, dtype=np.uint16) << 15) | (e << 7) |
              rng.integers(0, 128, shape, dtype=np.uint16)).astype(np.uint16)
         ws.append(w)
-        blobs.append(zb.zipmoe_encode(w, layout=zb.LAYOUT_BLOCKED, chunk_elems=65536))
-    assert zb.DecodePlan(blobs).max_record_bytes > 2432
+        blobs.append(zb.zipmoe_encode(w, layout=zb.LAYOUT_BLOCKED, chunk_elems=65536, max_code_len=12 if long_codes else 8))
+    plan = zb.DecodePlan(blobs)
+    assert plan.max_record_bytes > 2432 and (plan.max_code_len > 8) == long_codes
     ex = zb.DeviceExperts(blobs, H, I)
     tok = inputs.tokens(T, H, seed=9)
     ids, wts = inputs.routing(T, n_experts=E, k=k, seed=9)
@@ -106,7 +113,7 @@ def test_experts_whose_records_do_not_fit_the_record_stage(zb):
     torch.cuda.synchronize()
     assert int(ex.dev.status.item()) == 0
     want, y = oracle_out(ws, tok, ids, wts, np.arange(T))
-    check(out.cpu().numpy().view(np.uint16), want, y, "records read from global memory")
+    check(out.cpu().numpy().view(np.uint16), want, y, ("records read from global memory", long_codes))
 
 
 def test_single_expert_k1_and_unused_experts(zb):
