@@ -416,6 +416,14 @@ zipmoe_status zipmoe_plan_schedule(const zipmoe_sched_task *tasks, uint32_t n_ta
  * up after `tries` tries.  (0, 0) restores normal operation.  Process-wide; not for concurrent use. */
 void zipmoe_test_wait_fault(uint32_t extra_tx_bytes, uint32_t tries);
 
+/* For the library's own tests (the paper has no counterpart).  A launch that hands its tiles out dynamically owns
+ * a work counter of the library's ring for its duration; should it ever find the tag of another launch there, it
+ * stops, decodes nothing more and sets status_word to code 6.  With more than a thousand such launches in flight
+ * that could happen; a test cannot bring it about on purpose.  While this switch is on, zipmoe_decode therefore
+ * fills the counter of such a launch with a tag that no launch carries instead of zeroing it.  0 restores normal
+ * operation.  Process-wide; not for concurrent use. */
+void zipmoe_test_foreign_counter(uint32_t on);
+
 /* Name of a status code (static string). */
 const char *zipmoe_status_string(zipmoe_status s);
 

@@ -112,6 +112,15 @@ def zipmoe_test_wait_fault(extra_tx_bytes, tries):
     _lib.zipmoe_test_wait_fault(int(extra_tx_bytes), int(tries))
 
 
+_lib.zipmoe_test_foreign_counter.argtypes = [_u32]
+_lib.zipmoe_test_foreign_counter.restype = None
+
+
+def zipmoe_test_foreign_counter(on):
+    """Test switch: dynamically distributed launches find another launch's tag in their work counter; 0 = normal."""
+    _lib.zipmoe_test_foreign_counter(int(on))
+
+
 def zipmoe_version():
     return int(_lib.zipmoe_version())
 

@@ -469,7 +469,7 @@ namespace {
 constexpr uint32_t kCounterSlots = 1024;
 static __device__ unsigned long long g_work_counters[kCounterSlots];   // per slot: tag of the owning launch << 32 | next tile
 std::atomic<uint32_t> g_next_slot{0};
-std::atomic<uint32_t> g_test_extra_tx{0}, g_test_tries{zipmoe_host::kWaitTries};
+std::atomic<uint32_t> g_test_extra_tx{0}, g_test_tries{zipmoe_host::kWaitTries}, g_test_foreign_counter{0};
 
 struct DeviceInfo {
   int sm_count = 0;
@@ -511,6 +511,8 @@ void zipmoe_host::wait_fault_setting(uint32_t *extra_tx, uint32_t *tries) {
   *extra_tx = g_test_extra_tx.load();
   *tries = g_test_tries.load();
 }
+
+extern "C" void zipmoe_test_foreign_counter(uint32_t on) { g_test_foreign_counter.store(on ? 1u : 0u); }
 
 extern "C" void zipmoe_test_wait_fault(uint32_t extra_tx_bytes, uint32_t tries) {
   g_test_extra_tx.store(extra_tx_bytes & ~15u);
@@ -566,7 +568,8 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
     const uint32_t seq = g_next_slot.fetch_add(1);
     a.work_counter = counters + 2 * (seq % kCounterSlots);
     a.work_tag = seq | 0x80000000u;   // never zero; differs between any two launches that can meet on a slot
-    if (cudaMemsetAsync(a.work_counter, 0, 8, st) != cudaSuccess) return ZIPMOE_ERR_CUDA;
+    // (the library's own tests can have the counter filled with 0x7F7F7F7F, a tag no launch carries: tags have bit 31 set)
+    if (cudaMemsetAsync(a.work_counter, g_test_foreign_counter.load() ? 0x7F : 0, 8, st) != cudaSuccess) return ZIPMOE_ERR_CUDA;
     ctas = (uint32_t)sms * (narrow ? zipmoe_dev::Cfg<false>::kCtasPerSm : 1u);
     const uint32_t most = (n_tiles + 15 - 1) / 15;   // a tile per warp at least
     if (ctas > most) ctas = most;

@@ -236,6 +236,35 @@ def test_dynamic_distribution_many_launches_in_a_row(zb):
                 assert np.array_equal(got, want), it
 
 
+def test_launch_that_finds_its_work_counter_taken_says_so(zb):
+    """A dynamically distributed launch that finds another launch's tag in its work counter (possible only with
+    more than a thousand such launches in flight) must stop, leave the output alone and set status 6; the library's
+    test switch fills the counter with a tag no launch carries.  Launches with fixed ranges use no counter; the next
+    ordinary launch is exact."""
+    import torch
+    xs = [inputs.gaussian((n,), 0.02, n) for n in (30000, 5000, 70000)]
+    plan = zb.DecodePlan([zb.zipmoe_encode(x, chunk_elems=1024) for x in xs])
+    assert plan.n_tiles < 512 * plan.n_tables
+    dev = plan.to_device()
+    out = dev.new_output()
+    out.fill_(0x5555)
+    zb.zipmoe_test_foreign_counter(1)
+    try:
+        dev.decode(out)
+        torch.cuda.synchronize()
+    finally:
+        zb.zipmoe_test_foreign_counter(0)
+    assert int(dev.status.item()) == 6
+    assert bool((out == 0x5555).all())
+    dev.status.zero_()
+    dev.decode(out)
+    torch.cuda.synchronize()
+    assert int(dev.status.item()) == 0
+    host = out.cpu().numpy().view(np.uint16)
+    for i, x in enumerate(xs):
+        assert np.array_equal(plan.tensor_slice(host, i), x)
+
+
 def test_short_codes_promise_kept_and_broken(zb):
     """ZIPMOE_DECODE_SHORT_CODES selects the kernel variant that carries only the common path.  The plan gives the
     promise exactly when it holds; a launch that gives it falsely must leave the offending tiles undecoded and say
