@@ -292,6 +292,51 @@ def test_short_codes_promise_kept_and_broken(zb):
     assert bool((out == 0x5555).all())                              # nothing was written
 
 
+@pytest.mark.parametrize("damage", ["incomplete", "overfull", "length 13"])
+@pytest.mark.parametrize("promise", [False, True])
+def test_code_lengths_that_are_no_prefix_code_set_status_4(zb, damage, promise):
+    """A table whose 256 code lengths do not form a complete prefix code (one code dropped, one code too many, a
+    length above 12) is reported in the status word; what is decoded with it is garbage but every access stays
+    inside the call's buffers (the elements between and after the tensors keep their fill), and with the
+    short-codes promise nothing is decoded at all.  The same launch with the sound table is exact afterwards."""
+    import torch
+    xs = [inputs.gaussian((n,), 0.02, n) for n in (50000, 4096, 9000)]
+    plan = zb.DecodePlan([zb.zipmoe_encode(x, chunk_elems=4096) for x in xs])
+    sound = plan.tables.copy()
+    used = np.nonzero(sound[:256])[0]
+    if damage == "incomplete":
+        plan.tables[used[0]] = 0                                     # a code of the first tensor's table goes missing
+    elif damage == "overfull":
+        plan.tables[int(np.flatnonzero(sound[:256] == 0)[0])] = 2    # a short code more than the code space holds
+    else:
+        plan.tables[used[0]] = 13
+    if not promise:
+        plan.flags = 0
+    dev = plan.to_device()
+    out = dev.new_output()
+    out.fill_(0x5555)
+    dev.decode(out)
+    torch.cuda.synchronize()
+    assert int(dev.status.item()) == 4
+    host = out.cpu().numpy().view(np.uint16)
+    mask = np.ones(plan.out_elems, bool)
+    for i, inf in enumerate(plan.infos):
+        mask[plan.out_base[i]: plan.out_base[i] + inf.n_elems] = False
+    assert (host[mask] == 0x5555).all()
+    if promise:
+        assert (plan.tensor_slice(host, 0) == 0x5555).all()          # the tensor with the bad table: left alone
+    for i in (1, 2):                                                 # the other tensors have sound tables
+        assert np.array_equal(plan.tensor_slice(host, i), xs[i])
+    dev.tables.copy_(torch.from_numpy(sound))
+    dev.status.zero_()
+    dev.decode(out)
+    torch.cuda.synchronize()
+    assert int(dev.status.item()) == 0
+    host = out.cpu().numpy().view(np.uint16)
+    for i, x in enumerate(xs):
+        assert np.array_equal(plan.tensor_slice(host, i), x)
+
+
 def test_empty_launch_and_bad_arguments(zb):
     import torch
     zb.zipmoe_decode(None, 0, 0, None, 0, None, 0, None, 0, None, 0)       # nothing to do: OK
