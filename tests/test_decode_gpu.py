@@ -337,6 +337,43 @@ def test_code_lengths_that_are_no_prefix_code_set_status_4(zb, damage, promise):
         assert np.array_equal(plan.tensor_slice(host, i), x)
 
 
+@pytest.mark.parametrize("chunk,max_code_len", [(1024, 8), (4096, 8), (16384, 12)])
+def test_damaged_code_streams_decode_to_other_data_but_stay_in_bounds(zb, chunk, max_code_len):
+    """Bytes of the payload buffer (tile tables, column tables, code words) are overwritten at random.  The kernel
+    cannot know the right data any more, but it must stay inside the call's buffers: a tile table entry that no
+    longer describes a record is reported (status 1) and the tile skipped, everything else decodes to something, the
+    elements between and after the tensors keep their fill, and the launch after it, on sound data, is exact."""
+    import torch
+    rng = np.random.default_rng(chunk + max_code_len)
+    xs = [inputs.gaussian((n,), 0.02, n) for n in (70000, 33000, 4096 * 9 + 5)] + [inputs.stress_tensor(3, max_elems=60000)[0]]
+    plan = zb.DecodePlan([zb.zipmoe_encode(x, chunk_elems=chunk, max_code_len=max_code_len) for x in xs])
+    dev = plan.to_device()
+    sound = dev.payload.clone()
+    out = dev.new_output()
+    mask = np.ones(plan.out_elems, bool)
+    for i, inf in enumerate(plan.infos):
+        mask[plan.out_base[i]: plan.out_base[i] + inf.n_elems] = False
+    for n_bytes in (1, 30, 3000):
+        bad = plan.payload.copy()
+        at = rng.integers(0, plan.payload_bytes, n_bytes)
+        bad[at] = rng.integers(0, 256, n_bytes).astype(np.uint8)
+        dev.payload.copy_(torch.from_numpy(bad))
+        dev.status.zero_()
+        out.fill_(0x5555)
+        dev.decode(out)
+        torch.cuda.synchronize()
+        assert int(dev.status.item()) in (0, 1)
+        assert (out.cpu().numpy().view(np.uint16)[mask] == 0x5555).all()
+    dev.payload.copy_(sound)
+    dev.status.zero_()
+    dev.decode(out)
+    torch.cuda.synchronize()
+    assert int(dev.status.item()) == 0
+    host = out.cpu().numpy().view(np.uint16)
+    for i, x in enumerate(xs):
+        assert np.array_equal(plan.tensor_slice(host, i), x.ravel())
+
+
 def test_empty_launch_and_bad_arguments(zb):
     import torch
     zb.zipmoe_decode(None, 0, 0, None, 0, None, 0, None, 0, None, 0)       # nothing to do: OK
