@@ -266,7 +266,10 @@ zipmoe_status zipmoe_ffn_workspace_bytes(uint32_t T, uint32_t k, const zipmoe_co
  * bf16 inputs, fp32 accumulation on the tensor cores (tcgen05, accumulators in
  * tensor memory), weights decoded tile by tile into shared memory.  The paper
  * does not define the expert network; this is the gated FFN of the models it
- * evaluates.  Five kernels on `stream`, asynchronous.
+ * evaluates.  Five kernels on `stream`, asynchronous; the last four are launched
+ * with programmatic stream serialization (each is set up while its predecessor
+ * drains and waits for it before it reads anything), so work queued on `stream`
+ * before and after the call is ordered against it as against one kernel.
  * device in : tokens [T, hidden] bf16 patterns; topk_ids [T, k] (each token's ids
  *             distinct); topk_weights [T, k] fp32 or NULL (= 1.0)
  * device out: out [T, hidden] bf16 patterns; workspace: scratch of at least
