@@ -284,6 +284,28 @@ def measure_decode(w, dev, steps, warmup, target_s, sampler=None, world=1, barri
     times = max_over_ranks([a.elapsed_time(b) for a, b in evs], dev)
     verified = verified and all(int(d.status.item()) == 0 for d in dplans)
     med, best = float(np.median(times)), float(min(times))
+    # small launches with fixed ranges (nothing but the kernel on the stream): also replayed from a CUDA graph that
+    # holds one launch per buffer copy, which takes the host's launch cost out of the figure
+    in_graph = None
+    if copies > 1 and barrier is None and plan.n_tiles >= 512 * plan.n_tables:
+        side = torch.cuda.Stream(dev)
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(copies):
+                    dplans[i].decode(outs[i])
+            for _ in range(3):
+                g.replay()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(side)
+            for _ in range(20):
+                g.replay()
+            b.record(side)
+        torch.cuda.synchronize(dev)
+        in_graph = a.elapsed_time(b) / (20 * copies)
+        verified = verified and all(int(d.status.item()) == 0 for d in dplans)
+        del g
     peaks, _ = measured_peaks()
     res = {
         "workload": w.label, "tensors": len(w.blobs), "elements": w.n_elems,
@@ -296,6 +318,7 @@ def measure_decode(w, dev, steps, warmup, target_s, sampler=None, world=1, barri
         "frac": alg * steps / (med / 1e3) / 1e9 / peaks["hbm_gbs"],
         "frac_best": alg * steps / (best / 1e3) / 1e9 / peaks["hbm_gbs"],
         "buffer_copies_rotated": copies, "status_clean": all(int(d.status.item()) == 0 for d in dplans),
+        "ms_per_launch_in_cuda_graph": in_graph,
         "verified_bit_exact": verified, "timed_seconds": sum(times) / 1e3,
     }
     if sampler is not None:
@@ -420,8 +443,25 @@ def bench_ffn(dev, iters=20, cpu_tokens=2, token_counts=(1, 16, 64), config="lar
         ref = unfused().float()
         diff = (y.view(torch.bfloat16).float() - ref).abs().max().item()
         us_f, us_u = timed(fused), timed(unfused)
+        # the same call replayed from a CUDA graph (what a decode loop would do with it)
+        side = torch.cuda.Stream(dev)
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                fused()
+            for _ in range(3):
+                g.replay()
+            ga, gb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ga.record(side)
+            for _ in range(iters):
+                g.replay()
+            gb.record(side)
+        torch.cuda.synchronize(dev)
+        us_g = ga.elapsed_time(gb) / iters * 1e3
+        del g
         nbytes = sum(expert_bytes[e] for e in active)
-        out["T%d" % T] = {"us": us_f, "tokens_per_s": T / us_f * 1e6, "active_experts": len(active),
+        out["T%d" % T] = {"us": us_f, "us_in_cuda_graph": us_g, "tokens_per_s": T / us_f * 1e6, "active_experts": len(active),
                           "compressed_gbs": nbytes / us_f / 1e3,
                           # the fused call must at least read the routed experts' compressed bytes once
                           "frac_of_hbm_roofline": nbytes / us_f / 1e3 / measured_peaks()[0]["hbm_gbs"],
