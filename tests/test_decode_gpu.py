@@ -374,6 +374,22 @@ def test_damaged_code_streams_decode_to_other_data_but_stay_in_bounds(zb, chunk,
         assert np.array_equal(plan.tensor_slice(host, i), x.ravel())
 
 
+def test_status_word_is_optional(zb):
+    """A caller that passes no status word gets the same decode (errors would then go unreported: its choice)."""
+    import torch
+    xs = [inputs.gaussian((n,), 0.02, n) for n in (100000, 3000)]
+    for chunk in (1024, 65536):
+        plan = zb.DecodePlan([zb.zipmoe_encode(x, chunk_elems=chunk) for x in xs])
+        dev = plan.to_device()
+        out = dev.new_output()
+        zb.zipmoe_decode(dev.descs, plan.n_chunks, plan.n_tiles, dev.tables, plan.n_tables, dev.payload, plan.payload_bytes,
+                         dev.sm, plan.sm_bytes, out, plan.out_elems, None, None, plan.max_record_bytes, plan.flags)
+        torch.cuda.synchronize()
+        host = out.cpu().numpy().view(np.uint16)
+        for i, x in enumerate(xs):
+            assert np.array_equal(plan.tensor_slice(host, i), x)
+
+
 def test_empty_launch_and_bad_arguments(zb):
     import torch
     zb.zipmoe_decode(None, 0, 0, None, 0, None, 0, None, 0, None, 0)       # nothing to do: OK

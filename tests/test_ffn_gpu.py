@@ -130,6 +130,23 @@ def test_single_expert_k1_and_unused_experts(zb):
     check(out.cpu().numpy().view(np.uint16), want, y, "k1")
 
 
+def test_status_word_is_optional(zb):
+    import torch
+    E, H, I = 2, 256, 512
+    ws, blobs = make_layer(zb, E, H, I, seed=70)
+    ex = zb.DeviceExperts(blobs, H, I)
+    tok = torch.from_numpy(inputs.tokens(3, H, seed=4).view(np.int16)).cuda()
+    ids_np, wts_np = inputs.routing(3, n_experts=E, k=2, seed=4)
+    ids, wts = torch.from_numpy(ids_np).cuda(), torch.from_numpy(wts_np).cuda()
+    want = ex.ffn(tok, ids, wts).clone()
+    n = zb.zipmoe_ffn_workspace_bytes(3, 2, ex.struct)
+    wsp = torch.empty(n, dtype=torch.uint8, device="cuda")
+    out = torch.zeros(3, H, dtype=torch.int16, device="cuda")
+    zb.zipmoe_decode_expert_ffn(tok, 3, ids, wts, 2, ex.struct, out, wsp, n, None, None)
+    torch.cuda.synchronize()
+    assert torch.equal(out, want)
+
+
 def test_bad_arguments(zb):
     import torch
     E, H, I = 1, 256, 1024
