@@ -139,8 +139,17 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
 // over-full code is reported and leaves zero entries in the holes: decoding
 // then yields garbage but stays in bounds.
 // lut_raw holds the lane table when the result is <= 8, the wide table otherwise.
+// A barrier of the whole CTA (id 0) or of `threads` threads that share a named barrier (a team of warps with a
+// table of its own).
+__device__ __forceinline__ void group_sync(uint32_t bar_id, uint32_t threads) {
+  if (bar_id == 0) __syncthreads();
+  else asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(threads) : "memory");
+}
+
+// (tid: the thread's index among the THREADS that call, bar_id: their barrier -- by default the whole CTA)
 __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint8_t *code_len, uint8_t *lut_raw,
-                                              uint8_t *scratch, uint32_t *status) {
+                                              uint8_t *scratch, uint32_t *status, const uint32_t tid_in = 0xFFFFFFFFu,
+                                              const uint32_t bar_id = 0) {
   uint8_t *s_len = scratch;                                           // [256]
   uint32_t *s_first = reinterpret_cast<uint32_t *>(scratch + 256);    // [16] left-aligned 12-bit start of each length
   uint32_t *s_wcnt = s_first + 16;                                    // [8][16] per-warp symbol counts by length
@@ -149,7 +158,7 @@ __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint
   uint32_t *s_max = s_short + 256;                                    // [1] longest length
   uint32_t *lane_lut = reinterpret_cast<uint32_t *>(lut_raw);
   uint32_t *wide_lut = reinterpret_cast<uint32_t *>(lut_raw);
-  const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t tid = tid_in == 0xFFFFFFFFu ? threadIdx.x : tid_in, warp = tid >> 5, lane = tid & 31;
 
   uint32_t len = 0;
   if (tid < 256) {
@@ -166,7 +175,7 @@ __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint
       if (lane == 0) s_wcnt[warp * 16 + L] = __popc(b);
     }
   }
-  __syncthreads();
+  group_sync(bar_id, THREADS);
   if (tid == 0) {
     uint32_t code = 0, longest = 0;
     for (uint32_t L = 1; L <= ZIPMOE_MAX_CODE_LEN; ++L) {
@@ -183,7 +192,7 @@ __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint
     }
     *s_max = longest;
   }
-  __syncthreads();
+  group_sync(bar_id, THREADS);
   const uint32_t longest = *s_max;
   if (tid < 256 && len) {
     uint32_t rank = rank_in_warp;
@@ -193,7 +202,7 @@ __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint
   }
   if (longest > (uint32_t)kLaneLutBits)
     for (uint32_t k = tid; k < (uint32_t)kWideLutEntries; k += THREADS) wide_lut[k] = 0;
-  __syncthreads();
+  group_sync(bar_id, THREADS);
   // every symbol fills the range of windows its code is a prefix of
   for (uint32_t s = warp; s < 256; s += THREADS / 32) {
     const uint32_t L = s_len[s];
@@ -208,11 +217,11 @@ __device__ __forceinline__ uint32_t build_lut(const uint32_t THREADS, const uint
     if (longest > (uint32_t)kLaneLutBits)
       for (uint32_t k = lane; k < n; k += 32) wide_lut[start + k] = entry;
   }
-  __syncthreads();
+  group_sync(bar_id, THREADS);
   // replicate the 8-bit table once per lane
   if (longest <= (uint32_t)kLaneLutBits)
     for (uint32_t k = tid; k < (1u << kLaneLutBits) * 32; k += THREADS) lane_lut[k] = s_short[k >> 5];
-  __syncthreads();
+  group_sync(bar_id, THREADS);
   return longest;
 }
 

@@ -52,8 +52,14 @@ struct Cfg {
   static constexpr int kStage = WIDE ? (int)(kRecHead + 32 * kRowBytes) + kPaySlack : 2432 + kPaySlack;
   static constexpr int kBuf = kStage - kPaySlack;                         // longest staged record
   static constexpr int kWarpBytes = kPayStages * kStage + kSmPieces * kSmPieceBytes;
-  static constexpr int kSmemBytes = kLutBytes + kWarps * kWarpBytes + kWarps * kBarsPerWarp * 8 + kLutScratchBytes;
-  static_assert(kCtasPerSm * (kSmemBytes + 1024) <= 228 * 1024, "shared memory per SM");
+  // lookup tables: one, or two where the narrow stages leave room and the launch is dynamically distributed (two
+  // teams of warps, see decode_kernel); a launch asks for no more shared memory than it uses, because what it
+  // leaves is first-level cache (the fixed-range launches are 2 % slower with 35 KB less of it)
+  static constexpr int kMaxLuts = WIDE ? 1 : 2;
+  static constexpr int smem_bytes(int luts) {
+    return luts * (kLutBytes + kLutScratchBytes) + kWarps * kWarpBytes + kWarps * kBarsPerWarp * 8;
+  }
+  static_assert(kCtasPerSm * (smem_bytes(kMaxLuts) + 1024) <= 228 * 1024, "shared memory per SM");
 };
 
 // Per-warp asynchronous pipeline.  A warp decodes its tiles one after the other;
@@ -222,19 +228,28 @@ __device__ __forceinline__ TileWork fetch_step(const LaunchArgs &a, const Packed
 template <bool WIDE, bool BATCHED, bool LEAN = false>
 __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) decode_kernel(const LaunchArgs a) {
   using C = Cfg<WIDE>;
-  constexpr int kWarps = C::kWarps, kThreads = C::kThreads, kWarpBytes = C::kWarpBytes;
+  constexpr int kWarps = C::kWarps, kWarpBytes = C::kWarpBytes;
   constexpr uint32_t kBuf = C::kBuf;
   extern __shared__ __align__(128) uint8_t smem[];
-  uint8_t *lut_raw = smem;
-  uint8_t *warp_base = smem + kLutBytes;
-  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kLutBytes + kWarps * kWarpBytes);
-  uint8_t *lut_scratch = reinterpret_cast<uint8_t *>(bars + kWarps * kBarsPerWarp);
-
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // Teams: a dynamically distributed launch with narrow stages splits its warps into two teams, each with its own
+  // table, its own ranges of tiles and its own barrier, so that while one team changes tensors (waits for its
+  // last warp, builds the table, fetches the first records) the other keeps decoding, and a tensor of a few
+  // tiles leaves half as many warps without work.  Otherwise the CTA is one team.
+  constexpr int kTeams = (BATCHED && !WIDE) ? 2 : 1;
+  constexpr int kTeamWarps = kWarps / kTeams, kTeamThreads = kTeamWarps * 32;
+  static_assert(kTeams <= C::kMaxLuts && kWarps % kTeams == 0 && kTeamThreads >= 256, "teams");
+  const uint32_t team = warp / kTeamWarps, tw = warp - team * kTeamWarps, ttid = tid - team * kTeamThreads;
+  const uint32_t bar_id = kTeams > 1 ? team + 1 : 0;
+  uint8_t *lut_raw = smem + team * kLutBytes;
+  uint8_t *warp_base = smem + kTeams * kLutBytes;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(warp_base + kWarps * kWarpBytes);
+  uint8_t *lut_scratch = reinterpret_cast<uint8_t *>(bars + kWarps * kBarsPerWarp) + team * kLutScratchBytes;
+
   uint32_t g0 = blockIdx.x * a.tiles_per_cta;
   uint32_t g1 = min(g0 + a.tiles_per_cta, a.n_tiles);
   if (!BATCHED && g0 >= g1) return;
-  __shared__ uint32_t s_grab[2];   // BATCHED: the range of tiles the CTA took last
+  __shared__ uint32_t s_grab[2][2];   // BATCHED: the range of tiles each team took last
 
   WarpPipe pipe;
   pipe.pay_addr = smem_addr(warp_base + warp * kWarpBytes);
@@ -264,11 +279,11 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
 #ifndef ZIPMOE_GRAB_DIV
 #define ZIPMOE_GRAB_DIV 2
 #endif
-  constexpr uint32_t kMinGrab = ZIPMOE_GRAB_MIN * kWarps;
+  constexpr uint32_t kMinGrab = ZIPMOE_GRAB_MIN * kTeamWarps;
   for (;;) {
   if (BATCHED) {
-    __syncthreads();   // s_grab of the previous round has been read by every thread
-    if (tid == 0) {
+    group_sync(bar_id, kTeamThreads);   // s_grab of the previous round has been read by every thread of the team
+    if (ttid == 0) {
       // The counter is one 64-bit word: the tag of the launch that owns it above the next tile not yet handed out.
       // It was zeroed on the stream before this kernel; the first CTA to arrive installs the launch's tag.  Should
       // two launches ever be given the same counter while both are in flight (more of them queued than the ring
@@ -287,18 +302,18 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
       if (tag != a.work_tag) {
         report(a.status, kStatusCounterShared);
       } else if (seen < a.n_tiles) {
-        take = (a.n_tiles - seen) / (ZIPMOE_GRAB_DIV * gridDim.x);
-        take = max(take, max(1u, min(kMinGrab, a.n_tiles / gridDim.x)));   // small launches: spread over all CTAs
+        take = (a.n_tiles - seen) / (ZIPMOE_GRAB_DIV * kTeams * gridDim.x);
+        take = max(take, max(1u, min(kMinGrab, a.n_tiles / (kTeams * gridDim.x))));   // small launches: spread over all teams
         first = (uint32_t)atomicAdd(ctr, (unsigned long long)take);
         take = first < a.n_tiles ? min(a.n_tiles - first, take) : 0u;
         if (take == 0) first = a.n_tiles;
       }
-      s_grab[0] = first;
-      s_grab[1] = first + take;
+      s_grab[team][0] = first;
+      s_grab[team][1] = first + take;
     }
-    __syncthreads();
-    g0 = s_grab[0];
-    g1 = s_grab[1];
+    group_sync(bar_id, kTeamThreads);
+    g0 = s_grab[team][0];
+    g1 = s_grab[team][1];
     if (g0 >= g1) break;
   }
   uint32_t c = find_chunk(a, g0);
@@ -315,8 +330,8 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
     }
     // Each warp takes a contiguous share of the segment's tiles: consecutive tiles sit in the same chunk, so the
     // descriptor and the tile-table entries of the next tile are usually in the first-level cache already.
-    const uint32_t share = (seg_end - g0 + kWarps - 1) / kWarps;
-    uint32_t g = g0 + warp * share;
+    const uint32_t share = (seg_end - g0 + kTeamWarps - 1) / kTeamWarps;
+    uint32_t g = g0 + tw * share;
     const uint32_t g_end = min(seg_end, g + share);
     uint32_t stage = 0;
     constexpr bool batched = BATCHED;
@@ -360,8 +375,9 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
       }
     }
     if (!BATCHED || table_id != lut_table) {
-      __syncthreads();  // every warp is done with the previous table
-      fast = build_lut(kThreads, a.tables[table_id].code_len, lut_raw, lut_scratch, a.status) <= (uint32_t)kLaneLutBits;
+      group_sync(bar_id, kTeamThreads);  // every warp of the team is done with the previous table
+      fast = build_lut(kTeamThreads, a.tables[table_id].code_len, lut_raw, lut_scratch, a.status, ttid, bar_id) <=
+             (uint32_t)kLaneLutBits;
       lut_table = table_id;
     }
 
@@ -488,12 +504,12 @@ zipmoe_status prepare_device(int *sm_count, uint32_t **counters) {
     if (major != 10) return ZIPMOE_ERR_UNSUPPORTED;
     using namespace zipmoe_dev;
     const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    if (cudaFuncSetAttribute(decode_kernel<true, true>, at, Cfg<true>::kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(decode_kernel<true, false>, at, Cfg<true>::kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(decode_kernel<false, true>, at, Cfg<false>::kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(decode_kernel<false, false>, at, Cfg<false>::kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(decode_kernel<false, true, true>, at, Cfg<false>::kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(decode_kernel<false, false, true>, at, Cfg<false>::kSmemBytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(decode_kernel<true, true>, at, Cfg<true>::smem_bytes(1)) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_kernel<true, false>, at, Cfg<true>::smem_bytes(1)) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_kernel<false, true>, at, Cfg<false>::smem_bytes(2)) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_kernel<false, false>, at, Cfg<false>::smem_bytes(1)) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_kernel<false, true, true>, at, Cfg<false>::smem_bytes(2)) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_kernel<false, false, true>, at, Cfg<false>::smem_bytes(1)) != cudaSuccess)
       return ZIPMOE_ERR_CUDA;
     void *ptr = nullptr;   // (in host code the array's name is not a device address: ask for it)
     if (cudaGetSymbolAddress(&ptr, g_work_counters) != cudaSuccess || !ptr) return ZIPMOE_ERR_CUDA;
@@ -576,12 +592,12 @@ extern "C" zipmoe_status zipmoe_decode(const zipmoe_chunk_desc *chunks, uint32_t
   }
   const bool lean = narrow && (flags & ZIPMOE_DECODE_SHORT_CODES);
   if (lean && batched)
-    zipmoe_dev::decode_kernel<false, true, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
-  else if (lean) zipmoe_dev::decode_kernel<false, false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
+    zipmoe_dev::decode_kernel<false, true, true><<<ctas, Narrow::kThreads, Narrow::smem_bytes(2), st>>>(a);
+  else if (lean) zipmoe_dev::decode_kernel<false, false, true><<<ctas, Narrow::kThreads, Narrow::smem_bytes(1), st>>>(a);
   else if (narrow && batched)
-    zipmoe_dev::decode_kernel<false, true><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
-  else if (narrow) zipmoe_dev::decode_kernel<false, false><<<ctas, Narrow::kThreads, Narrow::kSmemBytes, st>>>(a);
-  else if (batched) zipmoe_dev::decode_kernel<true, true><<<ctas, Wide::kThreads, Wide::kSmemBytes, st>>>(a);
-  else zipmoe_dev::decode_kernel<true, false><<<ctas, Wide::kThreads, Wide::kSmemBytes, st>>>(a);
+    zipmoe_dev::decode_kernel<false, true><<<ctas, Narrow::kThreads, Narrow::smem_bytes(2), st>>>(a);
+  else if (narrow) zipmoe_dev::decode_kernel<false, false><<<ctas, Narrow::kThreads, Narrow::smem_bytes(1), st>>>(a);
+  else if (batched) zipmoe_dev::decode_kernel<true, true><<<ctas, Wide::kThreads, Wide::smem_bytes(1), st>>>(a);
+  else zipmoe_dev::decode_kernel<true, false><<<ctas, Wide::kThreads, Wide::smem_bytes(1), st>>>(a);
   return cudaGetLastError() == cudaSuccess ? ZIPMOE_OK : ZIPMOE_ERR_CUDA;
 }
