@@ -271,8 +271,9 @@ __global__ void __launch_bounds__(Cfg<WIDE>::kThreads, Cfg<WIDE>::kCtasPerSm) de
   uint32_t lut_table = 0xFFFFFFFFu;   // BATCHED: the table in shared memory
   bool fast = true;
   // BATCHED: the launch's tiles are handed out dynamically, in ranges that shrink as the work runs out (half of what
-  // an even split of the rest would give, at least kMinGrab tiles: measured best among halves, thirds, quarters and minima of 1..32 tiles per warp), because tiles and tensors of such launches differ
-  // too much in cost for equal shares to finish together.  Otherwise the CTA has its one fixed range.
+  // an even split of the rest would give, at least kMinGrab tiles: measured best among halves, thirds, quarters
+  // and minima of 1..32 tiles per warp), because tiles and tensors of such launches differ too much in cost for
+  // equal shares to finish together.  Otherwise the CTA has its one fixed range.
 #ifndef ZIPMOE_GRAB_MIN
 #define ZIPMOE_GRAB_MIN 8
 #endif

@@ -214,8 +214,8 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
 
   // (an incomplete last group: the MMA operand then also covers the bytes after the last warp's buffer, which
   // are the lookup table's, inside the allocation; the accumulator rows they produce are never read)
-  const bool shape_ok = 2 * Q * NACC <= 512 && (kGroupWarps * Q - NW) * kFfnWarpBytes <= kMyLutBytes && steps > 0 && steps <= 64 && a.n_mats > 0 &&
-                        a.n_groups > 0;
+  const bool shape_ok = 2 * Q * NACC <= 512 && (kGroupWarps * Q - NW) * kFfnWarpBytes <= kMyLutBytes && steps > 0 &&
+                        steps <= 64 && a.n_mats > 0 && a.n_groups > 0;
   if (!shape_ok) report(a.la.status, kStatusBadDescriptor);
 
   // The barriers are initialised once; every role counts what it has put through them since the kernel began,
@@ -377,7 +377,9 @@ __global__ void __launch_bounds__(kFfnMaxThreads, 1) ffn_matmul_kernel(const Ffn
       }
     } else if (is_mma) {
       // ---- one MMA warp per group; one lane issues, per half-tile: D[64 x N] (+)= A[64 x 256] * X[N x 256]^T ----
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((NACC >> 3) << 17) | ((uint32_t)(kGroupWarps / 2) << 24);   // bf16 x bf16 -> fp32, N = NACC, M = 8 * kGroupWarps
+      // instruction descriptor: bf16 x bf16 -> fp32, N = NACC, M = 8 * kGroupWarps
+      const uint32_t idesc =
+          (1u << 4) | (1u << 7) | (1u << 10) | ((NACC >> 3) << 17) | ((uint32_t)(kGroupWarps / 2) << 24);
       const uint32_t q = warp - NW;
       const uint32_t abuf = smem_addr(warp_raw) + 2 * kPayStage + kGroupWarps * q * kFfnWarpBytes;
       const uint64_t a_desc0 = smem_desc(abuf, kBLbo, kFfnWarpBytes);
